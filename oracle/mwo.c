@@ -1,0 +1,327 @@
+/*
+ * mwo -- CPU oracle for the MultiWrite dispatch / AllGather pack-and-deliver path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, sequential statement of
+ * what the path computes.  It shares no code with the CUDA library and is never
+ * used by it; only the tests, the smoke check and the benchmark's CPU-baseline leg
+ * may call it.
+ *
+ * What is being computed (paper, Section 4.3.1): MultiWrite(S, M, B_S) writes the
+ * content of the source buffer B_S into the target buffer B_i of every destination
+ * D_i in M.  For MoE dispatch (Sections 1 and 2.3.2) the destinations of a token
+ * are the nodes that host its gate-selected top-k experts; the destination set is
+ * carried as a bitmap with one bit per rank, ranks numbered from zero
+ * (Section 4.1, "Encoding scheme of metadata"; Section 6.4 for more than 64 ranks).
+ * The unicast comparison sends one copy per destination (Section 2.2).  The
+ * AllGather form (Section 5.2) delivers every rank's shard to every rank.
+ *
+ * The paper fixes the *content* each destination must end up with; it leaves the
+ * slot layout open.  The layout used here (also listed in the design notes):
+ *   - bit (r mod 64) of 64-bit word (r / 64) stands for rank r, least significant
+ *     bit first; bits at or above R are zero;
+ *   - the destination set is per rank: several experts of one token on the same
+ *     rank set one bit;
+ *   - a group is the set of all tokens with a bit-identical, non-empty bitmap;
+ *     groups are numbered by first occurrence while walking tokens 0..T-1;
+ *   - inside a group, and inside every receive region, rows keep ascending token
+ *     order;
+ *   - an expert id of -1 is padding; any other id outside [0,E), or a table entry
+ *     outside [0,R), is ignored and reported as MWO_ERR_BAD_INDEX;
+ *   - a token whose bitmap is empty gets no group, no send row and no bytes;
+ *   - src_rank >= 0 names the sender's own rank: its bit is still delivered, but
+ *     that copy is local and is left out of both transmitted-byte counts.
+ *
+ * Parity pins for every function live in tests/test_oracle_*.py (brute-force
+ * enumeration of (token, rank) pairs written independently in Python, closed
+ * forms, library counting-sort / bincount / concatenate special cases, the
+ * constants printed in the paper).  The numbering rules themselves (first
+ * occurrence, ascending token order) are this implementation's reading, not the
+ * paper's: parity for those choices is pinned only to the independent brute force.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define MWO_OK 0
+#define MWO_ERR_INVALID_ARG (-1)
+#define MWO_ERR_BAD_INDEX (-5)
+
+typedef struct {
+    int64_t T_nonempty;               /* T' : tokens with a non-empty destination set        */
+    int64_t G;                        /* number of distinct non-empty destination sets       */
+    int64_t total_dest;               /* sum over tokens of |D_t| (rows delivered)           */
+    int64_t mw_bytes;                 /* bytes transmitted when each row is sent once        */
+    int64_t unicast_bytes;            /* bytes transmitted with one copy per destination     */
+    int64_t unicast_per_expert_bytes; /* bytes if one copy were sent per valid expert slot   */
+    int64_t meta_bytes;               /* in-payload bitmap bytes when R > 64 (Section 6.4)   */
+    int32_t status;
+    int32_t reserved;
+} mwo_totals;
+
+static int mwo_words(int32_t R) { return (R + 63) / 64; }
+
+static int popcount64(uint64_t v)
+{
+    int c = 0;
+    while (v) { v &= v - 1; ++c; }
+    return c;
+}
+
+/*
+ * Plan: bitmaps, groups, offsets, slots, byte accounting.
+ *
+ * Output arrays (caller allocated, Kd = min(K, R), W = ceil(R / 64)):
+ *   token_mask   [T, W]   token_ndest [T]   token_group [T]   token_mw_row [T]
+ *   mw_row_token [T]      (first T' entries defined, rest -1)
+ *   group_offsets[T + 1]  (first G + 1 entries defined, rest -1)
+ *   group_mask   [T, W]   (first G rows defined, rest 0)
+ *   rank_offsets [R + 1]  rank_tokens [T * Kd] (first total_dest defined, rest -1)
+ *   dest_rank    [T, Kd]  dest_pos    [T, Kd]  (-1 padded)
+ */
+int mwo_plan(const int32_t *topk_ids, const int32_t *expert_to_rank,
+             int32_t T, int32_t K, int32_t E, int32_t R, int64_t row_bytes, int32_t src_rank,
+             uint64_t *token_mask, int32_t *token_ndest, int32_t *token_group,
+             int32_t *token_mw_row, int32_t *mw_row_token, int32_t *group_offsets,
+             uint64_t *group_mask, int32_t *rank_offsets, int32_t *rank_tokens,
+             int32_t *dest_rank, int32_t *dest_pos, mwo_totals *totals)
+{
+    if (T < 0 || K <= 0 || E <= 0 || R <= 0 || row_bytes <= 0 || src_rank >= R) return MWO_ERR_INVALID_ARG;
+    const int W = mwo_words(R);
+    const int Kd = K < R ? K : R;
+    int32_t status = MWO_OK;
+    int64_t valid_slots = 0;
+
+    /* Step 1 -- destination bitmap per token (Section 4.1: one bit per rank, 1 = target). */
+    for (int32_t t = 0; t < T; ++t) {
+        uint64_t *m = token_mask + (int64_t)t * W;
+        for (int w = 0; w < W; ++w) m[w] = 0;
+        for (int32_t k = 0; k < K; ++k) {
+            int32_t id = topk_ids[(int64_t)t * K + k];
+            if (id == -1) continue;                         /* padding slot            */
+            if (id < 0 || id >= E) { status = MWO_ERR_BAD_INDEX; continue; }
+            int32_t r = expert_to_rank[id];
+            if (r < 0 || r >= R) { status = MWO_ERR_BAD_INDEX; continue; }
+            ++valid_slots;
+            m[r / 64] |= (uint64_t)1 << (r % 64);            /* OR: per-rank dedup      */
+        }
+        int nd = 0;
+        for (int w = 0; w < W; ++w) nd += popcount64(m[w]);
+        token_ndest[t] = nd;
+    }
+
+    /* Step 2 -- groups of identical bitmap, numbered by first occurrence. */
+    int64_t G = 0, Tn = 0;
+    int32_t *group_count = (int32_t *)calloc((size_t)T + 1, sizeof(int32_t));
+    if (!group_count) return MWO_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < (int64_t)T * W; ++i) group_mask[i] = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        const uint64_t *m = token_mask + (int64_t)t * W;
+        if (token_ndest[t] == 0) { token_group[t] = -1; continue; }
+        int64_t g = 0;
+        for (; g < G; ++g)
+            if (memcmp(group_mask + g * W, m, (size_t)W * sizeof(uint64_t)) == 0) break;
+        if (g == G) { memcpy(group_mask + G * W, m, (size_t)W * sizeof(uint64_t)); ++G; }
+        token_group[t] = (int32_t)g;
+        ++group_count[g];
+        ++Tn;
+    }
+
+    /* Step 3 -- group offsets (exclusive prefix sum) and send rows in token order. */
+    for (int32_t i = 0; i <= T; ++i) group_offsets[i] = -1;
+    group_offsets[0] = 0;
+    for (int64_t g = 0; g < G; ++g) group_offsets[g + 1] = group_offsets[g] + group_count[g];
+    for (int32_t t = 0; t < T; ++t) mw_row_token[t] = -1;
+    for (int64_t g = 0; g < G; ++g) group_count[g] = 0;       /* reuse as "members seen so far" */
+    for (int32_t t = 0; t < T; ++t) {
+        int32_t g = token_group[t];
+        if (g < 0) { token_mw_row[t] = -1; continue; }
+        int32_t row = group_offsets[g] + group_count[g]++;
+        token_mw_row[t] = row;
+        mw_row_token[row] = t;
+    }
+    free(group_count);
+
+    /* Step 4 -- per-rank counts, offsets, and each token's slot in each receive region. */
+    int32_t *rank_seen = (int32_t *)calloc((size_t)R, sizeof(int32_t));
+    if (!rank_seen) return MWO_ERR_INVALID_ARG;
+    for (int32_t t = 0; t < T; ++t)
+        for (int32_t r = 0; r < R; ++r)
+            if (token_mask[(int64_t)t * W + r / 64] >> (r % 64) & 1) ++rank_seen[r];
+    rank_offsets[0] = 0;
+    for (int32_t r = 0; r < R; ++r) rank_offsets[r + 1] = rank_offsets[r] + rank_seen[r];
+    const int64_t total_dest = rank_offsets[R];
+    for (int64_t i = 0; i < (int64_t)T * Kd; ++i) { rank_tokens[i] = -1; dest_rank[i] = -1; dest_pos[i] = -1; }
+    for (int32_t r = 0; r < R; ++r) rank_seen[r] = 0;          /* reuse as "tokens seen so far" */
+    for (int32_t t = 0; t < T; ++t) {
+        int i = 0;
+        for (int32_t r = 0; r < R; ++r) {
+            if (!(token_mask[(int64_t)t * W + r / 64] >> (r % 64) & 1)) continue;
+            dest_rank[(int64_t)t * Kd + i] = r;
+            dest_pos[(int64_t)t * Kd + i] = rank_seen[r];
+            rank_tokens[rank_offsets[r] + rank_seen[r]] = t;
+            ++rank_seen[r];
+            ++i;
+        }
+    }
+    free(rank_seen);
+
+    /* Step 5 -- transmitted bytes, exactly, from the plan. */
+    int64_t sent_rows = 0, sent_copies = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        int nd = token_ndest[t];
+        if (src_rank >= 0 && (token_mask[(int64_t)t * W + src_rank / 64] >> (src_rank % 64) & 1)) --nd;
+        if (nd > 0) ++sent_rows;
+        sent_copies += nd;
+    }
+    totals->T_nonempty = Tn;
+    totals->G = G;
+    totals->total_dest = total_dest;
+    totals->mw_bytes = sent_rows * row_bytes;
+    totals->unicast_bytes = sent_copies * row_bytes;
+    totals->unicast_per_expert_bytes = valid_slots * row_bytes;
+    /* Section 6.4: above 64 ranks the bitmap rides in the payload, once per 4096-byte packet. */
+    totals->meta_bytes = R <= 64 ? 0 : sent_rows * ((row_bytes + 4095) / 4096) * (int64_t)(8 * W);
+    totals->status = status;
+    totals->reserved = 0;
+    return MWO_OK;
+}
+
+/* Region r of a receive area: explicit stride, or compact (stride 0: region r begins at row rank_offsets[r]). */
+static uint8_t *region(uint8_t *recv_base, int64_t stride, const int32_t *rank_offsets, int32_t r, int64_t row_bytes)
+{
+    return stride ? recv_base + (int64_t)r * stride : recv_base + (int64_t)rank_offsets[r] * row_bytes;
+}
+
+/* MultiWrite send layout: row j holds the hidden row of token mw_row_token[j], each token once. */
+void mwo_pack_mw(const uint8_t *x, int64_t row_bytes, const int32_t *mw_row_token, int64_t T_nonempty, uint8_t *send_mw)
+{
+    for (int64_t j = 0; j < T_nonempty; ++j)
+        memcpy(send_mw + j * row_bytes, x + (int64_t)mw_row_token[j] * row_bytes, (size_t)row_bytes);
+}
+
+/* Unicast send layout: one copy per destination, rank-major, token order inside a rank. */
+void mwo_pack_uc(const uint8_t *x, int64_t row_bytes, const int32_t *rank_tokens, int64_t total_dest, uint8_t *send_uc)
+{
+    for (int64_t i = 0; i < total_dest; ++i)
+        memcpy(send_uc + i * row_bytes, x + (int64_t)rank_tokens[i] * row_bytes, (size_t)row_bytes);
+}
+
+/*
+ * Deliver from the MultiWrite send buffer: every send row is written to every
+ * destination named by its group's bitmap (Section 4.3.1; Section 4.3.3 with each
+ * destination as its own next hop: one plain write per set bit).
+ */
+void mwo_deliver_mw(const uint8_t *send_mw, int64_t row_bytes, int64_t T_nonempty, int32_t R, int32_t K,
+                    const int32_t *mw_row_token, const int32_t *token_group, const uint64_t *group_mask,
+                    const int32_t *dest_pos, const int32_t *rank_offsets,
+                    uint8_t *recv_base, int64_t recv_stride_bytes)
+{
+    const int W = mwo_words(R);
+    const int Kd = K < R ? K : R;
+    for (int64_t j = 0; j < T_nonempty; ++j) {
+        int32_t t = mw_row_token[j];
+        const uint64_t *m = group_mask + (int64_t)token_group[t] * W;
+        int i = 0;
+        for (int32_t r = 0; r < R; ++r) {
+            if (!(m[r / 64] >> (r % 64) & 1)) continue;
+            int64_t slot = dest_pos[(int64_t)t * Kd + i++];
+            memcpy(region(recv_base, recv_stride_bytes, rank_offsets, r, row_bytes) + slot * row_bytes,
+                   send_mw + j * row_bytes, (size_t)row_bytes);
+        }
+    }
+}
+
+/* Deliver from the unicast send buffer: region r receives its contiguous slice. */
+void mwo_deliver_uc(const uint8_t *send_uc, int64_t row_bytes, int32_t R, const int32_t *rank_offsets,
+                    uint8_t *recv_base, int64_t recv_stride_bytes)
+{
+    for (int32_t r = 0; r < R; ++r) {
+        int64_t n = rank_offsets[r + 1] - rank_offsets[r];
+        memcpy(region(recv_base, recv_stride_bytes, rank_offsets, r, row_bytes),
+               send_uc + (int64_t)rank_offsets[r] * row_bytes, (size_t)(n * row_bytes));
+    }
+}
+
+/*
+ * Delivery straight from the definition, using only the router output and the
+ * table: for each rank, walk tokens in ascending order and append the hidden row
+ * of every token that selected an expert on that rank.
+ */
+void mwo_deliver_definition(const uint8_t *x, int64_t row_bytes, const int32_t *topk_ids, const int32_t *expert_to_rank,
+                            int32_t T, int32_t K, int32_t E, int32_t R, const int32_t *rank_offsets,
+                            uint8_t *recv_base, int64_t recv_stride_bytes)
+{
+    for (int32_t r = 0; r < R; ++r) {
+        uint8_t *dst = region(recv_base, recv_stride_bytes, rank_offsets, r, row_bytes);
+        int64_t n = 0;
+        for (int32_t t = 0; t < T; ++t) {
+            int hit = 0;
+            for (int32_t k = 0; k < K && !hit; ++k) {
+                int32_t id = topk_ids[(int64_t)t * K + k];
+                if (id >= 0 && id < E && expert_to_rank[id] == r) hit = 1;
+            }
+            if (hit) memcpy(dst + (n++) * row_bytes, x + (int64_t)t * row_bytes, (size_t)row_bytes);
+        }
+    }
+}
+
+/*
+ * AllGather (Section 5.2): R ranks each hold one shard of shard_bytes; afterwards
+ * every destination rank holds shard_0 | shard_1 | ... | shard_{R-1}.
+ *
+ * Only destination ranks [dst_begin, dst_begin + dst_count) are materialised (the
+ * full R x R result does not fit in memory for large shards); byte accounting is
+ * always for the full domain.  A rank's own shard reaches its own region by a
+ * local copy, never over the network (Section 2.3.1: N1 sends its partition seven
+ * times in an 8-node domain), so it is delivered but not counted.
+ *
+ * layout 0 (MultiWrite): send_buf [R, shard_bytes] holds every shard once.
+ * layout 1 (unicast):    send_buf [R, dst_count, shard_bytes]; slot (i, d) holds the
+ *                        copy of shard i addressed to rank dst_begin + d.  The slot
+ *                        with dst_begin + d == i is never transmitted; it is left
+ *                        untouched and the self copy is taken from the shard itself.
+ * Region d of recv (rank dst_begin + d) starts at recv_base + d * stride
+ * (stride 0: compact, d * R * shard_bytes).
+ */
+int mwo_allgather(const uint8_t *shards, int32_t R, int64_t shard_bytes, int layout,
+                  int32_t dst_begin, int32_t dst_count, uint8_t *send_buf,
+                  uint8_t *recv_base, int64_t recv_stride_bytes, mwo_totals *totals)
+{
+    if (R <= 0 || shard_bytes <= 0 || dst_begin < 0 || dst_count < 0 || dst_begin + dst_count > R) return MWO_ERR_INVALID_ARG;
+    if (layout != 0 && layout != 1) return MWO_ERR_INVALID_ARG;
+    const int64_t stride = recv_stride_bytes ? recv_stride_bytes : (int64_t)R * shard_bytes;
+    if (layout == 0) {
+        for (int32_t i = 0; i < R; ++i)
+            memcpy(send_buf + (int64_t)i * shard_bytes, shards + (int64_t)i * shard_bytes, (size_t)shard_bytes);
+        for (int32_t i = 0; i < R; ++i)
+            for (int32_t d = 0; d < dst_count; ++d)
+                memcpy(recv_base + d * stride + (int64_t)i * shard_bytes,
+                       send_buf + (int64_t)i * shard_bytes, (size_t)shard_bytes);
+    } else {
+        for (int32_t i = 0; i < R; ++i)
+            for (int32_t d = 0; d < dst_count; ++d) {
+                if (dst_begin + d == i) continue;
+                memcpy(send_buf + ((int64_t)i * dst_count + d) * shard_bytes,
+                       shards + (int64_t)i * shard_bytes, (size_t)shard_bytes);
+            }
+        for (int32_t i = 0; i < R; ++i)
+            for (int32_t d = 0; d < dst_count; ++d) {
+                const uint8_t *src = (dst_begin + d == i) ? shards + (int64_t)i * shard_bytes
+                                                           : send_buf + ((int64_t)i * dst_count + d) * shard_bytes;
+                memcpy(recv_base + d * stride + (int64_t)i * shard_bytes, src, (size_t)shard_bytes);
+            }
+    }
+    if (totals) {
+        const int W = mwo_words(R);
+        memset(totals, 0, sizeof(*totals));
+        totals->T_nonempty = R;
+        totals->G = R;                                   /* every shard has its own destination set (all but itself) */
+        totals->total_dest = (int64_t)R * R;             /* rows delivered, self copies included */
+        totals->mw_bytes = R > 1 ? (int64_t)R * shard_bytes : 0;
+        totals->unicast_bytes = (int64_t)R * (R - 1) * shard_bytes;
+        totals->unicast_per_expert_bytes = totals->unicast_bytes;
+        totals->meta_bytes = (R <= 64 || R == 1) ? 0 : (int64_t)R * ((shard_bytes + 4095) / 4096) * (8 * W);
+        totals->status = MWO_OK;
+    }
+    return MWO_OK;
+}

@@ -1,0 +1,180 @@
+"""ctypes front end of the CPU oracle (oracle/mwo.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library never imports or links this.
+It marshals numpy arrays into the C functions; it does no arithmetic of its own.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mwo.c")
+_LIB = os.path.join(_HERE, "libmwo.so")
+
+MWO_OK = 0
+MWO_ERR_INVALID_ARG = -1
+MWO_ERR_BAD_INDEX = -5
+
+LAYOUT_MULTIWRITE = 0
+LAYOUT_UNICAST = 1
+
+
+class Totals(C.Structure):
+    _fields_ = [("T_nonempty", C.c_int64), ("G", C.c_int64), ("total_dest", C.c_int64),
+                ("mw_bytes", C.c_int64), ("unicast_bytes", C.c_int64),
+                ("unicast_per_expert_bytes", C.c_int64), ("meta_bytes", C.c_int64),
+                ("status", C.c_int32), ("reserved", C.c_int32)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle/mwo.c into oracle/libmwo.so with gcc (plain C, no CUDA)."""
+    stale = force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if stale:
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.mwo_plan.restype = C.c_int
+        _lib.mwo_allgather.restype = C.c_int
+        for name in ("mwo_pack_mw", "mwo_pack_uc", "mwo_deliver_mw", "mwo_deliver_uc", "mwo_deliver_definition"):
+            getattr(_lib, name).restype = None
+    return _lib
+
+
+def _p(a: np.ndarray):
+    assert a.flags["C_CONTIGUOUS"]
+    return C.c_void_p(a.ctypes.data)
+
+
+@dataclass
+class Plan:
+    T: int
+    K: int
+    E: int
+    R: int
+    W: int
+    Kd: int
+    row_bytes: int
+    token_mask: np.ndarray     # uint64 [T, W]
+    token_ndest: np.ndarray    # int32  [T]
+    token_group: np.ndarray    # int32  [T]
+    token_mw_row: np.ndarray   # int32  [T]
+    mw_row_token: np.ndarray   # int32  [T]      first T' defined
+    group_offsets: np.ndarray  # int32  [T + 1]  first G + 1 defined
+    group_mask: np.ndarray     # uint64 [T, W]   first G defined
+    rank_offsets: np.ndarray   # int32  [R + 1]
+    rank_tokens: np.ndarray    # int32  [T * Kd] first total_dest defined
+    dest_rank: np.ndarray      # int32  [T, Kd]
+    dest_pos: np.ndarray       # int32  [T, Kd]
+    totals: dict
+    ret: int
+
+
+def plan(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: int, src_rank: int = -1) -> Plan:
+    ids = np.ascontiguousarray(topk_ids, dtype=np.int32)
+    e2r = np.ascontiguousarray(expert_to_rank, dtype=np.int32)
+    T, K = ids.shape
+    E = e2r.shape[0]
+    W = (R + 63) // 64
+    Kd = min(K, R)
+    o = dict(
+        token_mask=np.zeros((T, W), np.uint64), token_ndest=np.zeros(T, np.int32),
+        token_group=np.zeros(T, np.int32), token_mw_row=np.zeros(T, np.int32),
+        mw_row_token=np.zeros(T, np.int32), group_offsets=np.zeros(T + 1, np.int32),
+        group_mask=np.zeros((T, W), np.uint64), rank_offsets=np.zeros(R + 1, np.int32),
+        rank_tokens=np.zeros(T * Kd, np.int32), dest_rank=np.zeros((T, Kd), np.int32),
+        dest_pos=np.zeros((T, Kd), np.int32))
+    tot = Totals()
+    ret = lib().mwo_plan(_p(ids), _p(e2r), C.c_int32(T), C.c_int32(K), C.c_int32(E), C.c_int32(R),
+                         C.c_int64(row_bytes), C.c_int32(src_rank),
+                         _p(o["token_mask"]), _p(o["token_ndest"]), _p(o["token_group"]), _p(o["token_mw_row"]),
+                         _p(o["mw_row_token"]), _p(o["group_offsets"]), _p(o["group_mask"]), _p(o["rank_offsets"]),
+                         _p(o["rank_tokens"]), _p(o["dest_rank"]), _p(o["dest_pos"]), C.byref(tot))
+    return Plan(T=T, K=K, E=E, R=R, W=W, Kd=Kd, row_bytes=row_bytes, totals=tot.as_dict(), ret=ret, **o)
+
+
+def _bytes2d(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x)
+    return x.view(np.uint8).reshape(x.shape[0], -1) if x.ndim == 2 else x.view(np.uint8)
+
+
+def recv_bytes_needed(p: Plan, recv_stride_bytes: int) -> int:
+    if recv_stride_bytes:
+        return p.R * recv_stride_bytes
+    return int(p.totals["total_dest"]) * p.row_bytes
+
+
+def pack_mw(p: Plan, x: np.ndarray) -> np.ndarray:
+    xb = _bytes2d(x)
+    Tn = p.totals["T_nonempty"]
+    out = np.zeros((Tn, p.row_bytes), np.uint8)
+    lib().mwo_pack_mw(_p(xb), C.c_int64(p.row_bytes), _p(p.mw_row_token), C.c_int64(Tn), _p(out))
+    return out
+
+
+def pack_uc(p: Plan, x: np.ndarray) -> np.ndarray:
+    xb = _bytes2d(x)
+    n = p.totals["total_dest"]
+    out = np.zeros((n, p.row_bytes), np.uint8)
+    lib().mwo_pack_uc(_p(xb), C.c_int64(p.row_bytes), _p(p.rank_tokens), C.c_int64(n), _p(out))
+    return out
+
+
+def deliver_mw(p: Plan, send_mw: np.ndarray, recv_stride_bytes: int = 0, fill: int = 0) -> np.ndarray:
+    recv = np.full(recv_bytes_needed(p, recv_stride_bytes), fill, np.uint8)
+    lib().mwo_deliver_mw(_p(send_mw), C.c_int64(p.row_bytes), C.c_int64(p.totals["T_nonempty"]), C.c_int32(p.R),
+                         C.c_int32(p.K), _p(p.mw_row_token), _p(p.token_group), _p(p.group_mask), _p(p.dest_pos),
+                         _p(p.rank_offsets), _p(recv), C.c_int64(recv_stride_bytes))
+    return recv
+
+
+def deliver_uc(p: Plan, send_uc: np.ndarray, recv_stride_bytes: int = 0, fill: int = 0) -> np.ndarray:
+    recv = np.full(recv_bytes_needed(p, recv_stride_bytes), fill, np.uint8)
+    lib().mwo_deliver_uc(_p(send_uc), C.c_int64(p.row_bytes), C.c_int32(p.R), _p(p.rank_offsets), _p(recv),
+                         C.c_int64(recv_stride_bytes))
+    return recv
+
+
+def deliver_definition(p: Plan, x: np.ndarray, topk_ids: np.ndarray, expert_to_rank: np.ndarray,
+                       recv_stride_bytes: int = 0, fill: int = 0) -> np.ndarray:
+    xb = _bytes2d(x)
+    ids = np.ascontiguousarray(topk_ids, dtype=np.int32)
+    e2r = np.ascontiguousarray(expert_to_rank, dtype=np.int32)
+    recv = np.full(recv_bytes_needed(p, recv_stride_bytes), fill, np.uint8)
+    lib().mwo_deliver_definition(_p(xb), C.c_int64(p.row_bytes), _p(ids), _p(e2r), C.c_int32(p.T), C.c_int32(p.K),
+                                 C.c_int32(p.E), C.c_int32(p.R), _p(p.rank_offsets), _p(recv),
+                                 C.c_int64(recv_stride_bytes))
+    return recv
+
+
+def allgather(shards: np.ndarray, layout: int, dst_begin: int = 0, dst_count: int | None = None,
+              recv_stride_bytes: int = 0, fill: int = 0):
+    """Returns (send_buf, recv, totals, ret).  shards: uint8 [R, S]."""
+    sh = np.ascontiguousarray(shards).view(np.uint8)
+    R, S = sh.shape
+    dst_count = R if dst_count is None else dst_count
+    stride = recv_stride_bytes or R * S
+    send = np.full(R * S if layout == LAYOUT_MULTIWRITE else R * dst_count * S, fill, np.uint8)
+    recv = np.full(max(dst_count, 0) * stride, fill, np.uint8)
+    tot = Totals()
+    ret = lib().mwo_allgather(_p(sh), C.c_int32(R), C.c_int64(S), C.c_int(layout), C.c_int32(dst_begin),
+                              C.c_int32(dst_count), _p(send), _p(recv), C.c_int64(recv_stride_bytes), C.byref(tot))
+    return send, recv, tot.as_dict(), ret
