@@ -1,0 +1,236 @@
+/*
+ * mw.h -- C ABI of the MultiWrite dispatch / AllGather pack-and-deliver library (CUDA, sm_100a).
+ *
+ * The library emulates a communication domain of R ranks as R receive regions in one
+ * GPU's memory and performs, on the device, the source-side and relay-side work of
+ * the paper's MultiWrite semantic:
+ *
+ *   MultiWrite(S, M, B_S), M = {(D_i, B_i)}: the content of the source buffer B_S is
+ *   written into the target buffer B_i of every destination D_i   (Section 4.3.1).
+ *
+ * For MoE dispatch the destinations of a token are the ranks hosting its top-k experts
+ * (Sections 1, 2.3.2); the destination set travels as a bitmap, one bit per rank, ranks
+ * numbered from zero (Section 4.1; Section 6.4 for more than 64 ranks).  The unicast
+ * layout sends one copy per destination (Section 2.2) and is kept as the comparison.
+ *
+ * Conventions for every call
+ *   - All pointers marked "device" are CUDA device pointers valid on the context's
+ *     device; "host" pointers are ordinary host memory.  `stream` is a cudaStream_t
+ *     passed as void* (NULL = the legacy default stream).
+ *   - The caller owns every buffer it passes.  The context owns the plan metadata and
+ *     its scratch, all allocated in mw_create; no other call allocates device memory,
+ *     except mw_dispatch_host, which uses staging buffers allocated in mw_create when
+ *     MW_FLAG_HOST_STAGING is set.
+ *   - Calls are asynchronous on `stream` unless stated otherwise; results are defined
+ *     once the stream has completed ("atomic per destination, no ordering between
+ *     destinations", Section 4.3.4).  A context must be driven from one stream at a time.
+ *   - Every call returns MW_OK or a negative MW_ERR_* code.  Errors that the host can
+ *     see (null pointer, misalignment, sizes beyond the configured maxima) are returned
+ *     at once and nothing is launched.  Errors that depend on device data (an expert id
+ *     outside {-1} U [0,E), a table entry outside [0,R), a row that would land beyond a
+ *     buffer's capacity, a wait that gave up) are recorded in mw_totals.status on the
+ *     device, the offending write is suppressed, and mw_get_totals reports them.
+ *     Nothing traps or aborts.
+ *
+ * Layout rules (the paper fixes the bytes each destination receives; the slots are this
+ * library's choice)
+ *   - rank r is bit (r mod 64), least significant first, of 64-bit word (r / 64);
+ *     W = ceil(R / 64) words per bitmap; bits >= R are zero;
+ *   - destination sets are per rank: experts of one token on the same rank set one bit;
+ *   - a group is the set of all tokens with the same non-empty bitmap; groups are numbered
+ *     by first occurrence in token order; rows of a group, and rows of a receive region,
+ *     keep ascending token order;
+ *   - expert id -1 is padding and is skipped; a token whose bitmap is empty has no group,
+ *     no send row (token_group = token_mw_row = -1) and moves no bytes.
+ */
+#ifndef MW_H_
+#define MW_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define MW_API __attribute__((visibility("default")))
+#else
+#define MW_API
+#endif
+
+#define MW_OK                0
+#define MW_ERR_INVALID_ARG  (-1)  /* null pointer, size out of range, unknown layout          */
+#define MW_ERR_ALIGNMENT    (-2)  /* pointer, stride or row size not a multiple of 16 bytes   */
+#define MW_ERR_CAPACITY     (-3)  /* a buffer cannot hold the rows the plan assigns to it     */
+#define MW_ERR_CUDA         (-4)  /* a CUDA runtime call failed                               */
+#define MW_ERR_BAD_INDEX    (-5)  /* expert id or expert->rank entry out of range (ignored)   */
+#define MW_ERR_TIMEOUT      (-6)  /* a bounded device-side wait gave up; the plan is invalid  */
+#define MW_ERR_NO_PLAN      (-7)  /* dispatch called before any plan                          */
+
+#define MW_LAYOUT_MULTIWRITE 0    /* send buffer holds each row once (one row per group member) */
+#define MW_LAYOUT_UNICAST    1    /* send buffer holds one copy per destination                */
+
+#define MW_FLAG_HOST_STAGING   0x1u  /* allocate device staging so mw_dispatch_host can be used */
+#define MW_FLAG_PLAN_MULTIPASS 0x2u  /* always take the tiled multi-kernel plan, even for small T */
+#define MW_FLAG_COPY_LDST      0x4u  /* row copies by 16-byte register loads/stores, not bulk copies */
+
+#define MW_MAX_RANKS   1024
+#define MW_MAX_TOPK    64
+
+typedef struct mw_ctx mw_ctx;   /* opaque: configuration, device workspace, plan metadata */
+
+typedef struct {
+    int32_t  R;           /* ranks in the emulated domain, 1..MW_MAX_RANKS                         */
+    int32_t  E;           /* experts (length of expert_to_rank), >= 1                              */
+    int32_t  K;           /* router top-k (columns of topk_ids), 1..MW_MAX_TOPK                    */
+    int32_t  max_tokens;  /* largest T any mw_plan call will pass, >= 1                            */
+    int64_t  row_bytes;   /* B: bytes per hidden row, a positive multiple of 16                    */
+    int32_t  src_rank;    /* sender's own rank, or -1 if it is outside the domain (Section 2.3.1:  */
+                          /* the copy to oneself is local and not counted as transmitted)          */
+    int32_t  device;      /* CUDA device ordinal                                                   */
+    uint32_t flags;       /* MW_FLAG_*                                                             */
+    uint32_t reserved;
+} mw_config;
+
+/* Exact byte accounting of the last plan (64-bit integers; no measurement involved). */
+typedef struct {
+    int64_t T_nonempty;               /* T': tokens with at least one destination                   */
+    int64_t G;                        /* distinct non-empty destination sets = MultiWrite groups    */
+    int64_t total_dest;               /* sum over tokens of |D_t| = rows delivered                   */
+    int64_t mw_bytes;                 /* transmitted when every row is sent once (Section 1)        */
+    int64_t unicast_bytes;            /* transmitted with one copy per destination (Section 2.2)    */
+    int64_t unicast_per_expert_bytes; /* one copy per valid expert slot (no per-rank dedup)         */
+    int64_t meta_bytes;               /* bitmap bytes carried in the payload when R > 64, one       */
+                                      /* bitmap per 4096-byte packet (Section 6.4); 0 otherwise     */
+    int32_t status;                   /* MW_OK or the first device-side MW_ERR_* of plan/dispatch   */
+    int32_t reserved;
+} mw_totals;
+
+/*
+ * Device pointers into the context's workspace, valid until mw_destroy; contents are those
+ * of the latest mw_plan once its stream work has completed.  Kd = min(K, R).
+ * Entries past the defined prefix hold -1 (masks: 0).
+ */
+typedef struct {
+    const uint64_t  *token_mask;    /* [T, W]    destination bitmap of each token                   */
+    const int32_t   *token_ndest;   /* [T]       |D_t|                                              */
+    const int32_t   *token_group;   /* [T]       group id, -1 if D_t is empty                       */
+    const int32_t   *token_mw_row;  /* [T]       row of the token in the MultiWrite send buffer     */
+    const int32_t   *mw_row_token;  /* [T]       inverse of the above; first T' entries defined     */
+    const int32_t   *group_offsets; /* [T + 1]   exclusive prefix sum of group sizes; G + 1 defined */
+    const uint64_t  *group_mask;    /* [T, W]    bitmap of each group; first G rows defined         */
+    const int32_t   *rank_offsets;  /* [R + 1]   exclusive prefix sum of rows per receive region    */
+    const int32_t   *rank_tokens;   /* [T * Kd]  token of every delivered row, region-major         */
+    const int32_t   *dest_rank;     /* [T, Kd]   ascending destination ranks of the token, -1 pad   */
+    const int32_t   *dest_pos;      /* [T, Kd]   slot of the token inside that rank's region        */
+    const mw_totals *totals;        /* device copy of the accounting                                */
+    int32_t T, W, Kd, reserved;
+} mw_plan_view;
+
+/*
+ * Creates a context: validates the configuration, selects cfg->device, allocates all
+ * device workspace (sized for max_tokens and the worst case of Kd destinations per token).
+ * Corresponds to the paper's initialisation module, which loads the node configuration
+ * (Section 5.1, cs_ini).  Synchronous.  *out is NULL on failure.
+ */
+MW_API int mw_create(mw_ctx **out, const mw_config *cfg);
+
+/* Frees everything mw_create allocated.  Synchronises the device first.  NULL is accepted. */
+MW_API int mw_destroy(mw_ctx *ctx);
+
+/*
+ * Source-side planning (Section 4.1 step 1: the source turns the destination information
+ * into bitmap metadata; Section 5.1, cs_send: task decomposition).  From the router output
+ * it builds bitmaps, groups, per-group and per-rank counts with exclusive prefix sums, every
+ * token's send row and receive slots, and the byte accounting.
+ *
+ *   topk_ids        device, int32 [T, K] row-major; -1 = padding
+ *   expert_to_rank  device, int32 [E], values in [0, R)  (the preconfigured table of Section 4.1)
+ *   T               0 <= T <= max_tokens
+ *   view            host, optional: receives the workspace pointers (same every call)
+ */
+MW_API int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
+            mw_plan_view *view, void *stream);
+
+/* Waits for `stream`, then copies the accounting of the latest plan to host memory. */
+MW_API int mw_get_totals(mw_ctx *ctx, mw_totals *host_out, void *stream);
+
+/*
+ * Pack: fill the send buffer from the hidden rows, using the latest plan (Section 5.2 step 1:
+ * "loads its local message data into the pre-allocated send buffer").
+ *   MW_LAYOUT_MULTIWRITE  send_buf[j] = x[mw_row_token[j]],            j < T'
+ *   MW_LAYOUT_UNICAST     send_buf[rank_offsets[r] + i] = x[rank_tokens[rank_offsets[r] + i]]
+ *   x         device, [T, row_bytes], 16-byte aligned
+ *   send_buf  device, send_capacity_rows * row_bytes bytes, 16-byte aligned; rows beyond the
+ *             capacity are not written and set MW_ERR_CAPACITY in the status
+ */
+MW_API int mw_pack(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows, void *stream);
+
+/*
+ * Deliver: expand the send buffer into the R receive regions (Section 4.1 steps 3-5 and
+ * Section 4.3.3 with every destination as its own next hop: the relay reads the payload it
+ * holds and writes one copy per set bit of the bitmap).
+ *   MW_LAYOUT_MULTIWRITE  for each send row j and each set bit r of its group's bitmap:
+ *                         region(r)[dest_pos(token, r)] = send_buf[j]
+ *   MW_LAYOUT_UNICAST     region(r)[i] = send_buf[rank_offsets[r] + i]
+ * Both give region(r) = the rows of all tokens bound for r, in ascending token order.
+ *   recv_base           device, 16-byte aligned
+ *   recv_stride_bytes   > 0: region(r) starts at recv_base + r * stride (multiple of 16) and holds
+ *                       at most recv_capacity_rows rows;
+ *                       0: compact, region(r) starts at row rank_offsets[r] and the whole area
+ *                       holds at most recv_capacity_rows rows
+ */
+MW_API int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_base, int64_t recv_stride_bytes,
+               int64_t recv_capacity_rows, void *stream);
+
+/* mw_pack followed by mw_deliver on the same stream: the whole data movement of one dispatch. */
+MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows,
+                void *recv_base, int64_t recv_stride_bytes, int64_t recv_capacity_rows, void *stream);
+
+/*
+ * AllGather pack + deliver (Section 5.2): R ranks each contribute one shard of shard_bytes;
+ * every destination rank ends with shard_0 | shard_1 | ... | shard_{R-1}.  Uses cfg.R only.
+ *   shards       device, [R, shard_bytes] contiguous, 16-byte aligned; shard_bytes multiple of 16
+ *   layout       MW_LAYOUT_MULTIWRITE: send_buf [R, shard_bytes], every shard once;
+ *                MW_LAYOUT_UNICAST:    send_buf [R, dst_rank_count, shard_bytes]; slot (i, d) is the
+ *                copy of shard i addressed to rank dst_rank_begin + d; the slot addressed to
+ *                rank i itself is never written (that copy is local: Section 2.3.1)
+ *   recv_base    device; region d (rank dst_rank_begin + d) starts at recv_base + d * stride,
+ *                stride = recv_stride_bytes, or R * shard_bytes when 0
+ *   dst_rank_begin, dst_rank_count   the window of destination ranks that is materialised
+ *                (the full R x R result need not fit in memory); accounting is for the full domain
+ *   host_totals  host, optional: receives the accounting (filled synchronously, no device work)
+ */
+MW_API int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int layout, void *send_buf,
+                      void *recv_base, int64_t recv_stride_bytes, int32_t dst_rank_begin, int32_t dst_rank_count,
+                      mw_totals *host_totals, void *stream);
+
+/*
+ * One whole dispatch from host memory (plan, pack, deliver) for callers whose data lives on
+ * the host: copies topk_ids, expert_to_rank and x to the device, runs mw_plan and mw_dispatch
+ * into context-owned staging, and copies the compact receive area (total_dest rows), the
+ * rank offsets and the accounting back.  Needs MW_FLAG_HOST_STAGING.  Synchronises `stream`.
+ *   recv_host              host, at least recv_capacity_rows * row_bytes bytes
+ *   rank_offsets_host      host, int32 [R + 1]
+ * Pinned host memory makes the copies asynchronous; pageable memory also works.
+ */
+MW_API int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int32_t *expert_to_rank_host,
+                     const void *x_host, int32_t T, int layout, void *recv_host, int64_t recv_capacity_rows,
+                     int32_t *rank_offsets_host, mw_totals *totals_host, void *stream);
+
+/*
+ * Convenience for reading plan metadata: waits for `stream`, then copies `bytes` from a device
+ * pointer of the plan view (or any device memory of the context's device) into host memory.
+ */
+MW_API int mw_read_device(mw_ctx *ctx, void *host_dst, const void *device_src, int64_t bytes, void *stream);
+
+/* Number of kernels this context has launched since mw_create (for launch accounting). */
+MW_API int64_t mw_kernel_launches(const mw_ctx *ctx);
+
+/* Static description of an error code. */
+MW_API const char *mw_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MW_H_ */

@@ -1,0 +1,234 @@
+"""ctypes binding of libmw.so: same names as the C ABI in include/mw.h, argument marshalling only.
+
+Device buffers are torch CUDA tensors (or raw integer device pointers); streams are torch streams.
+Every step of the path runs in the library's CUDA kernels.  If the library cannot be loaded this
+module raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+from . import build as _build
+
+MW_OK = 0
+MW_ERR_INVALID_ARG = -1
+MW_ERR_ALIGNMENT = -2
+MW_ERR_CAPACITY = -3
+MW_ERR_CUDA = -4
+MW_ERR_BAD_INDEX = -5
+MW_ERR_TIMEOUT = -6
+MW_ERR_NO_PLAN = -7
+
+MW_LAYOUT_MULTIWRITE = 0
+MW_LAYOUT_UNICAST = 1
+
+MW_FLAG_HOST_STAGING = 0x1
+MW_FLAG_PLAN_MULTIPASS = 0x2
+MW_FLAG_COPY_LDST = 0x4
+
+EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch",
+           "mw_allgather_pack", "mw_dispatch_host", "mw_read_device", "mw_kernel_launches", "mw_strerror")
+
+
+class mw_config(C.Structure):
+    _fields_ = [("R", C.c_int32), ("E", C.c_int32), ("K", C.c_int32), ("max_tokens", C.c_int32),
+                ("row_bytes", C.c_int64), ("src_rank", C.c_int32), ("device", C.c_int32),
+                ("flags", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class mw_totals(C.Structure):
+    _fields_ = [("T_nonempty", C.c_int64), ("G", C.c_int64), ("total_dest", C.c_int64),
+                ("mw_bytes", C.c_int64), ("unicast_bytes", C.c_int64),
+                ("unicast_per_expert_bytes", C.c_int64), ("meta_bytes", C.c_int64),
+                ("status", C.c_int32), ("reserved", C.c_int32)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
+
+
+class mw_plan_view(C.Structure):
+    _fields_ = [("token_mask", C.c_void_p), ("token_ndest", C.c_void_p), ("token_group", C.c_void_p),
+                ("token_mw_row", C.c_void_p), ("mw_row_token", C.c_void_p), ("group_offsets", C.c_void_p),
+                ("group_mask", C.c_void_p), ("rank_offsets", C.c_void_p), ("rank_tokens", C.c_void_p),
+                ("dest_rank", C.c_void_p), ("dest_pos", C.c_void_p), ("totals", C.c_void_p),
+                ("T", C.c_int32), ("W", C.c_int32), ("Kd", C.c_int32), ("reserved", C.c_int32)]
+
+
+class MwError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib():
+    """Loads libmw.so (built in-tree by build.build_library); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run `python -m paper_2605_22428_b200.build` "
+                               "(or __graft_entry__.build()); there is no CPU fallback")
+        L = C.CDLL(path)
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        L.mw_create.argtypes = [C.POINTER(vp), C.POINTER(mw_config)]
+        L.mw_destroy.argtypes = [vp]
+        L.mw_plan.argtypes = [vp, vp, vp, i32, C.POINTER(mw_plan_view), vp]
+        L.mw_get_totals.argtypes = [vp, C.POINTER(mw_totals), vp]
+        L.mw_pack.argtypes = [vp, vp, C.c_int, vp, i64, vp]
+        L.mw_deliver.argtypes = [vp, C.c_int, vp, vp, i64, i64, vp]
+        L.mw_dispatch.argtypes = [vp, vp, C.c_int, vp, i64, vp, i64, i64, vp]
+        L.mw_allgather_pack.argtypes = [vp, vp, i64, C.c_int, vp, vp, i64, i32, i32, C.POINTER(mw_totals), vp]
+        L.mw_dispatch_host.argtypes = [vp, vp, vp, vp, i32, C.c_int, vp, i64, vp, C.POINTER(mw_totals), vp]
+        L.mw_read_device.argtypes = [vp, vp, vp, i64, vp]
+        L.mw_kernel_launches.argtypes = [vp]
+        L.mw_kernel_launches.restype = C.c_int64
+        L.mw_strerror.argtypes = [C.c_int]
+        L.mw_strerror.restype = C.c_char_p
+        for name in EXPORTS[:10]:
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().mw_strerror(int(code)).decode()
+
+
+def _ptr(t) -> C.c_void_p:
+    """Device (or host) address of a torch tensor / numpy array / integer address / None."""
+    if t is None:
+        return C.c_void_p(0)
+    if isinstance(t, int):
+        return C.c_void_p(t)
+    if hasattr(t, "data_ptr"):
+        return C.c_void_p(t.data_ptr())
+    return C.c_void_p(t.ctypes.data)
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return C.c_void_p(stream)
+    return C.c_void_p(stream.cuda_stream)
+
+
+class Context:
+    """Owns one mw_ctx.  Methods mirror the C entry points and return the C return code checked."""
+
+    def __init__(self, R: int, E: int, K: int, max_tokens: int, row_bytes: int, src_rank: int = -1,
+                 device: int = 0, flags: int = 0):
+        self.cfg = mw_config(R, E, K, max_tokens, row_bytes, src_rank, device, flags, 0)
+        self._h = C.c_void_p()
+        rc = lib().mw_create(C.byref(self._h), C.byref(self.cfg))
+        if rc != MW_OK:
+            raise MwError(rc, "mw_create")
+        self.R, self.E, self.K, self.row_bytes = R, E, K, row_bytes
+        self.W = (R + 63) // 64
+        self.Kd = min(K, R)
+        self.device = device
+        self.view = None
+
+    def close(self):
+        if self._h:
+            lib().mw_destroy(self._h)
+            self._h = C.c_void_p()
+
+    __del__ = close
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- C ABI mirrors ----------------------------------------------------------------------
+    def mw_plan(self, topk_ids, expert_to_rank, T: int | None = None, stream=None, check: bool = True) -> int:
+        T = int(topk_ids.shape[0]) if T is None else T
+        view = mw_plan_view()
+        rc = lib().mw_plan(self._h, _ptr(topk_ids), _ptr(expert_to_rank), T, C.byref(view), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_plan")
+        self.view = view
+        return rc
+
+    def mw_get_totals(self, stream=None) -> dict:
+        tot = mw_totals()
+        rc = lib().mw_get_totals(self._h, C.byref(tot), _stream(stream))
+        if rc != MW_OK:
+            raise MwError(rc, "mw_get_totals")
+        return tot.as_dict()
+
+    def mw_pack(self, x, layout: int, send_buf, send_capacity_rows: int, stream=None, check: bool = True) -> int:
+        rc = lib().mw_pack(self._h, _ptr(x), layout, _ptr(send_buf), send_capacity_rows, _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_pack")
+        return rc
+
+    def mw_deliver(self, layout: int, send_buf, recv, recv_stride_bytes: int, recv_capacity_rows: int,
+                   stream=None, check: bool = True) -> int:
+        rc = lib().mw_deliver(self._h, layout, _ptr(send_buf), _ptr(recv), recv_stride_bytes, recv_capacity_rows,
+                              _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_deliver")
+        return rc
+
+    def mw_dispatch(self, x, layout: int, send_buf, send_capacity_rows: int, recv, recv_stride_bytes: int,
+                    recv_capacity_rows: int, stream=None, check: bool = True) -> int:
+        rc = lib().mw_dispatch(self._h, _ptr(x), layout, _ptr(send_buf), send_capacity_rows, _ptr(recv),
+                               recv_stride_bytes, recv_capacity_rows, _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_dispatch")
+        return rc
+
+    def mw_allgather_pack(self, shards, shard_bytes: int, layout: int, send_buf, recv, recv_stride_bytes: int = 0,
+                          dst_rank_begin: int = 0, dst_rank_count: int | None = None, stream=None,
+                          check: bool = True):
+        tot = mw_totals()
+        cnt = self.R if dst_rank_count is None else dst_rank_count
+        rc = lib().mw_allgather_pack(self._h, _ptr(shards), shard_bytes, layout, _ptr(send_buf), _ptr(recv),
+                                     recv_stride_bytes, dst_rank_begin, cnt, C.byref(tot), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_allgather_pack")
+        return rc, tot.as_dict()
+
+    def mw_dispatch_host(self, topk_ids_host, expert_to_rank_host, x_host, T: int, layout: int, recv_host,
+                         recv_capacity_rows: int, rank_offsets_host, stream=None, check: bool = True):
+        tot = mw_totals()
+        rc = lib().mw_dispatch_host(self._h, _ptr(topk_ids_host), _ptr(expert_to_rank_host), _ptr(x_host), T, layout,
+                                    _ptr(recv_host), recv_capacity_rows, _ptr(rank_offsets_host), C.byref(tot),
+                                    _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_dispatch_host")
+        return rc, tot.as_dict()
+
+    def mw_kernel_launches(self) -> int:
+        return int(lib().mw_kernel_launches(self._h))
+
+    # -- reading the plan back (tests, diagnostics) -------------------------------------------
+    def plan_arrays(self, T: int, stream=None) -> dict:
+        """Copies the plan metadata of the latest mw_plan to numpy arrays (synchronises)."""
+        import numpy as np
+        v = self.view
+        W, Kd, R = self.W, self.Kd, self.R
+        spec = dict(token_mask=(np.uint64, (T, W)), token_ndest=(np.int32, (T,)), token_group=(np.int32, (T,)),
+                    token_mw_row=(np.int32, (T,)), mw_row_token=(np.int32, (T,)), group_offsets=(np.int32, (T + 1,)),
+                    group_mask=(np.uint64, (T, W)), rank_offsets=(np.int32, (R + 1,)),
+                    rank_tokens=(np.int32, (T * Kd,)), dest_rank=(np.int32, (T, Kd)), dest_pos=(np.int32, (T, Kd)))
+        out = {}
+        for name, (dt, shape) in spec.items():
+            a = np.empty(shape, dt)
+            rc = lib().mw_read_device(self._h, _ptr(a), C.c_void_p(getattr(v, name)), a.nbytes, _stream(stream))
+            if rc != MW_OK:
+                raise MwError(rc, "mw_read_device")
+            out[name] = a
+        return out

@@ -1,0 +1,348 @@
+// C ABI entry points (declared and documented in include/mw.h): argument checks, workspace
+// carving, and the launch sequences.  No step of the path runs on the host.
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+#include "mw_internal.cuh"
+
+namespace {
+
+inline bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+inline size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+struct Carver {
+    uint8_t *base;
+    size_t used;
+    template <class T> T *take(size_t count)
+    {
+        T *p = base ? (T *)(base + used) : nullptr;
+        used += round256(count * sizeof(T));
+        return p;
+    }
+};
+
+// Lays the workspace out inside one slab; with base == nullptr it only measures.
+size_t carve(mw_ctx *c, uint8_t *base)
+{
+    Carver k{base, 0};
+    const size_t Tm = (size_t)c->cfg.max_tokens, W = (size_t)c->W, Kd = (size_t)c->Kd, R = (size_t)c->cfg.R;
+    mw_dev &d = c->d;
+    d.token_mask = k.take<uint64_t>(Tm * W);
+    d.token_ndest = k.take<int32_t>(Tm);
+    d.token_group = k.take<int32_t>(Tm);
+    d.token_mw_row = k.take<int32_t>(Tm);
+    d.mw_row_token = k.take<int32_t>(Tm);
+    d.group_offsets = k.take<int32_t>(Tm + 1);
+    d.group_mask = k.take<uint64_t>(Tm * W);
+    d.rank_offsets = k.take<int32_t>(R + 1);
+    d.rank_tokens = k.take<int32_t>(Tm * Kd);
+    d.dest_rank = k.take<int32_t>(Tm * Kd);
+    d.dest_pos = k.take<int32_t>(Tm * Kd);
+    d.totals = k.take<mw_totals>(1);
+    d.token_slot = k.take<int32_t>(Tm);
+    d.token_leader = k.take<int32_t>(Tm);
+    d.token_gcount = k.take<int32_t>(Tm);
+    d.gid_at = k.take<int32_t>(Tm);
+    d.goff_at = k.take<int32_t>(Tm);
+    d.row_ndest = k.take<int32_t>(Tm);
+    d.row_dest_rank = k.take<int32_t>(Tm * Kd);
+    d.row_dest_pos = k.take<int32_t>(Tm * Kd);
+    d.uc_row_rank = k.take<int32_t>(Tm * Kd);
+    d.slot_rep = k.take<int32_t>((size_t)c->HS);
+    d.slot_leader = k.take<int32_t>((size_t)c->HS);
+    d.slot_count = k.take<int32_t>((size_t)c->HS);
+    d.tile_state = k.take<unsigned long long>((size_t)c->max_tiles * (size_t)c->NC);
+    d.ticket = k.take<unsigned int>(1);
+    d.acc = k.take<mw_acc>(2);
+    if (c->cfg.flags & MW_FLAG_HOST_STAGING) {
+        const size_t B = (size_t)c->cfg.row_bytes;
+        c->st_ids = k.take<int32_t>(Tm * (size_t)c->cfg.K);
+        c->st_e2r = k.take<int32_t>((size_t)c->cfg.E);
+        c->st_x = k.take<uint8_t>(Tm * B);
+        c->st_send = k.take<uint8_t>(Tm * Kd * B);  // large enough for the unicast layout
+        c->st_recv = k.take<uint8_t>(Tm * Kd * B);
+        c->st_recv_rows = (int64_t)(Tm * Kd);
+    }
+    return k.used;
+}
+
+__global__ void k_fill_i32(int32_t *p, int64_t n, int32_t v)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = v;
+}
+
+inline cudaStream_t as_stream(void *s) { return (cudaStream_t)s; }
+
+int check_layout(int layout) { return (layout == MW_LAYOUT_MULTIWRITE || layout == MW_LAYOUT_UNICAST) ? MW_OK : MW_ERR_INVALID_ARG; }
+
+mw_copy_args base_args(mw_ctx *ctx)
+{
+    mw_copy_args a;
+    memset(&a, 0, sizeof(a));
+    a.row_bytes = ctx->cfg.row_bytes;
+    a.host_rows = -1;
+    a.Kd = ctx->Kd;
+    a.R = ctx->cfg.R;
+    a.rank_offsets = ctx->d.rank_offsets;
+    a.uc_row_rank = ctx->d.uc_row_rank;
+    a.totals = ctx->d.totals;
+    return a;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mw_create(mw_ctx **out, const mw_config *cfg)
+{
+    if (!out) return MW_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return MW_ERR_INVALID_ARG;
+    if (cfg->R < 1 || cfg->R > MW_MAX_RANKS || cfg->E < 1 || cfg->K < 1 || cfg->K > MW_MAX_TOPK ||
+        cfg->max_tokens < 1 || cfg->max_tokens > (1 << 24) || cfg->row_bytes < 16 || cfg->src_rank < -1 ||
+        cfg->src_rank >= cfg->R || cfg->device < 0)
+        return MW_ERR_INVALID_ARG;
+    if (cfg->row_bytes % 16) return MW_ERR_ALIGNMENT;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device >= ndev) return MW_ERR_CUDA;
+    if (cudaSetDevice(cfg->device) != cudaSuccess) return MW_ERR_CUDA;
+
+    mw_ctx *c = new (std::nothrow) mw_ctx();
+    if (!c) return MW_ERR_INVALID_ARG;
+    memset(c, 0, sizeof(*c));
+    c->cfg = *cfg;
+    c->W = (cfg->R + 63) / 64;
+    c->Kd = cfg->K < cfg->R ? cfg->K : cfg->R;
+    c->NC = cfg->R + 2;
+    c->max_tiles = (cfg->max_tokens + MW_TILE - 1) / MW_TILE;
+    int hs = 256;
+    while (hs < 2 * cfg->max_tokens) hs <<= 1;
+    c->HS = hs;
+    c->planned_T = -1;
+    cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
+    cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
+
+    const size_t bytes = carve(c, nullptr);
+    if (cudaMalloc(&c->slab, bytes) != cudaSuccess) { cudaGetLastError(); delete c; return MW_ERR_CUDA; }
+    carve(c, (uint8_t *)c->slab);
+    int rc = MW_OK;
+    if (cudaMemset(c->slab, 0, bytes) != cudaSuccess) rc = MW_ERR_CUDA;
+    // empty table: no representative, no leader
+    if (rc == MW_OK) {
+        k_fill_i32<<<64, 256>>>(c->d.slot_rep, c->HS, -1);
+        k_fill_i32<<<64, 256>>>(c->d.slot_leader, c->HS, 0x7fffffff);
+        if (cudaDeviceSynchronize() != cudaSuccess) rc = MW_ERR_CUDA;
+    }
+    if (rc == MW_OK) rc = mw_plan_smem_setup(c);
+    if (rc == MW_OK) rc = mw_copy_smem_setup(c);
+    if (rc != MW_OK) { cudaFree(c->slab); cudaGetLastError(); delete c; return rc; }
+    *out = c;
+    return MW_OK;
+}
+
+int mw_destroy(mw_ctx *ctx)
+{
+    if (!ctx) return MW_OK;
+    cudaSetDevice(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    const cudaError_t e = cudaFree(ctx->slab);
+    delete ctx;
+    return e == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}
+
+int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, mw_plan_view *view, void *stream)
+{
+    if (!ctx || !expert_to_rank || T < 0 || T > ctx->cfg.max_tokens || (T > 0 && !topk_ids)) return MW_ERR_INVALID_ARG;
+    if (view) {
+        const mw_dev &d = ctx->d;
+        view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
+        view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
+        view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
+        view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
+        view->T = T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
+    }
+    return mw_plan_launch(ctx, topk_ids, expert_to_rank, T, as_stream(stream));
+}
+
+int mw_get_totals(mw_ctx *ctx, mw_totals *host_out, void *stream)
+{
+    if (!ctx || !host_out) return MW_ERR_INVALID_ARG;
+    if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
+    if (cudaMemcpyAsync(host_out, ctx->d.totals, sizeof(mw_totals), cudaMemcpyDeviceToHost, as_stream(stream)) != cudaSuccess)
+        return MW_ERR_CUDA;
+    return cudaStreamSynchronize(as_stream(stream)) == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}
+
+int mw_pack(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows, void *stream)
+{
+    if (!ctx || !x || !send_buf || send_capacity_rows < 0 || check_layout(layout)) return MW_ERR_INVALID_ARG;
+    if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
+    if (!aligned16(x) || !aligned16(send_buf)) return MW_ERR_ALIGNMENT;
+    mw_copy_args a = base_args(ctx);
+    a.src = (const uint8_t *)x;
+    a.dst = (uint8_t *)send_buf;
+    a.capacity_rows = send_capacity_rows;
+    if (layout == MW_LAYOUT_MULTIWRITE) {
+        a.mode = MW_CP_PACK_MW;
+        a.rows_from = 1;                       // T' send rows, known on the device
+        a.src_index = ctx->d.mw_row_token;
+        a.host_rows = ctx->planned_T;          // estimate for the chunking heuristic
+    } else {
+        // one pass over the tokens: each hidden row is read once and written to its |D_t| unicast slots
+        a.mode = MW_CP_SCATTER;
+        a.rows_from = 0;
+        a.host_rows = ctx->planned_T;
+        a.ndst = ctx->d.token_ndest;
+        a.d_rank = ctx->d.dest_rank;
+        a.d_pos = ctx->d.dest_pos;
+        a.dst_stride = 0;
+    }
+    return mw_copy_launch(ctx, a, as_stream(stream));
+}
+
+int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_base, int64_t recv_stride_bytes,
+               int64_t recv_capacity_rows, void *stream)
+{
+    if (!ctx || !send_buf || !recv_base || recv_stride_bytes < 0 || recv_capacity_rows < 0 || check_layout(layout))
+        return MW_ERR_INVALID_ARG;
+    if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
+    if (!aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
+    if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
+    mw_copy_args a = base_args(ctx);
+    a.src = (const uint8_t *)send_buf;
+    a.dst = (uint8_t *)recv_base;
+    a.dst_stride = recv_stride_bytes;
+    a.capacity_rows = recv_capacity_rows;
+    if (layout == MW_LAYOUT_MULTIWRITE) {
+        a.mode = MW_CP_SCATTER;
+        a.rows_from = 1;
+        a.ndst = ctx->d.row_ndest;
+        a.d_rank = ctx->d.row_dest_rank;
+        a.d_pos = ctx->d.row_dest_pos;
+        a.host_rows = ctx->planned_T;          // estimate for the chunking heuristic
+    } else {
+        a.mode = MW_CP_DELIVER_UC;
+        a.rows_from = 2;
+        a.host_rows = (int64_t)ctx->planned_T * ctx->Kd;
+    }
+    return mw_copy_launch(ctx, a, as_stream(stream));
+}
+
+int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows,
+                void *recv_base, int64_t recv_stride_bytes, int64_t recv_capacity_rows, void *stream)
+{
+    if (!ctx || !x || !send_buf || !recv_base) return MW_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
+    int rc = mw_pack(ctx, x, layout, send_buf, send_capacity_rows, stream);
+    if (rc != MW_OK) return rc;
+    return mw_deliver(ctx, layout, send_buf, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
+}
+
+int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int layout, void *send_buf,
+                      void *recv_base, int64_t recv_stride_bytes, int32_t dst_rank_begin, int32_t dst_rank_count,
+                      mw_totals *host_totals, void *stream)
+{
+    if (!ctx || !shards || !send_buf || !recv_base || shard_bytes < 16 || recv_stride_bytes < 0 || check_layout(layout))
+        return MW_ERR_INVALID_ARG;
+    const int R = ctx->cfg.R;
+    if (dst_rank_begin < 0 || dst_rank_count < 0 || dst_rank_begin + dst_rank_count > R) return MW_ERR_INVALID_ARG;
+    if (shard_bytes % 16 || recv_stride_bytes % 16 || !aligned16(shards) || !aligned16(send_buf) || !aligned16(recv_base))
+        return MW_ERR_ALIGNMENT;
+    const int64_t stride = recv_stride_bytes ? recv_stride_bytes : (int64_t)R * shard_bytes;
+    if (stride < (int64_t)R * shard_bytes) return MW_ERR_CAPACITY;
+    if (host_totals) {
+        memset(host_totals, 0, sizeof(*host_totals));
+        host_totals->T_nonempty = R;
+        host_totals->G = R;
+        host_totals->total_dest = (int64_t)R * R;
+        host_totals->mw_bytes = R > 1 ? (int64_t)R * shard_bytes : 0;
+        host_totals->unicast_bytes = (int64_t)R * (R - 1) * shard_bytes;     // Section 2.3.1: R - 1 copies per source
+        host_totals->unicast_per_expert_bytes = host_totals->unicast_bytes;
+        host_totals->meta_bytes = (R <= 64) ? 0 : (int64_t)R * ((shard_bytes + 4095) / 4096) * (8 * ctx->W);
+    }
+    if (dst_rank_count == 0 && layout == MW_LAYOUT_UNICAST) return MW_OK;   // empty window: no unicast slot exists
+    mw_copy_args a = base_args(ctx);
+    a.row_bytes = shard_bytes;
+    a.rows_from = 0;
+    a.dst_begin = dst_rank_begin;
+    a.dst_count = dst_rank_count;
+    a.capacity_rows = INT64_MAX;
+    int rc;
+    if (layout == MW_LAYOUT_MULTIWRITE) {
+        a.mode = MW_CP_AG_PACK_MW;
+        a.src = (const uint8_t *)shards; a.dst = (uint8_t *)send_buf; a.host_rows = R;
+        if ((rc = mw_copy_launch(ctx, a, as_stream(stream))) != MW_OK || dst_rank_count == 0) return rc;
+        a.mode = MW_CP_AG_DELIVER_MW;
+        a.src = (const uint8_t *)send_buf; a.dst = (uint8_t *)recv_base; a.dst_stride = stride;
+        return mw_copy_launch(ctx, a, as_stream(stream));
+    }
+    a.mode = MW_CP_AG_PACK_UC;
+    a.src = (const uint8_t *)shards; a.dst = (uint8_t *)send_buf; a.host_rows = R;
+    if ((rc = mw_copy_launch(ctx, a, as_stream(stream))) != MW_OK) return rc;
+    a.mode = MW_CP_AG_DELIVER_UC;
+    a.src = (const uint8_t *)send_buf; a.src2 = (const uint8_t *)shards; a.dst = (uint8_t *)recv_base;
+    a.dst_stride = stride; a.host_rows = (int64_t)R * dst_rank_count;
+    return mw_copy_launch(ctx, a, as_stream(stream));
+}
+
+int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int32_t *expert_to_rank_host,
+                     const void *x_host, int32_t T, int layout, void *recv_host, int64_t recv_capacity_rows,
+                     int32_t *rank_offsets_host, mw_totals *totals_host, void *stream)
+{
+    if (!ctx || !expert_to_rank_host || !recv_host || !rank_offsets_host || !totals_host || T < 0 ||
+        T > ctx->cfg.max_tokens || (T > 0 && (!topk_ids_host || !x_host)) || check_layout(layout))
+        return MW_ERR_INVALID_ARG;
+    if (!(ctx->cfg.flags & MW_FLAG_HOST_STAGING)) return MW_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    const int64_t B = ctx->cfg.row_bytes;
+    if (cudaMemcpyAsync(ctx->st_e2r, expert_to_rank_host, sizeof(int32_t) * (size_t)ctx->cfg.E, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return MW_ERR_CUDA;
+    if (T > 0) {
+        if (cudaMemcpyAsync(ctx->st_ids, topk_ids_host, sizeof(int32_t) * (size_t)T * ctx->cfg.K, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return MW_ERR_CUDA;
+        if (cudaMemcpyAsync(ctx->st_x, x_host, (size_t)T * B, cudaMemcpyHostToDevice, st) != cudaSuccess) return MW_ERR_CUDA;
+    }
+    int rc = mw_plan(ctx, ctx->st_ids, ctx->st_e2r, T, nullptr, stream);
+    if (rc != MW_OK) return rc;
+    rc = mw_dispatch(ctx, ctx->st_x, layout, ctx->st_send, ctx->st_recv_rows, ctx->st_recv, 0, ctx->st_recv_rows, stream);
+    if (rc != MW_OK) return rc;
+    if (cudaMemcpyAsync(rank_offsets_host, ctx->d.rank_offsets, sizeof(int32_t) * (size_t)(ctx->cfg.R + 1), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MW_ERR_CUDA;
+    rc = mw_get_totals(ctx, totals_host, stream);       // synchronises: the row count is needed for the copy back
+    if (rc != MW_OK) return rc;
+    if (totals_host->total_dest > recv_capacity_rows) return MW_ERR_CAPACITY;
+    if (totals_host->total_dest > 0) {
+        if (cudaMemcpyAsync(recv_host, ctx->st_recv, (size_t)totals_host->total_dest * B, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return MW_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return MW_ERR_CUDA;
+    }
+    return MW_OK;
+}
+
+int mw_read_device(mw_ctx *ctx, void *host_dst, const void *device_src, int64_t bytes, void *stream)
+{
+    if (!ctx || bytes < 0 || (bytes > 0 && (!host_dst || !device_src))) return MW_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return MW_ERR_CUDA;
+    if (bytes == 0) return MW_OK;
+    return cudaMemcpy(host_dst, device_src, (size_t)bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}
+
+int64_t mw_kernel_launches(const mw_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *mw_strerror(int code)
+{
+    switch (code) {
+    case MW_OK: return "ok";
+    case MW_ERR_INVALID_ARG: return "invalid argument";
+    case MW_ERR_ALIGNMENT: return "pointer, stride or row size is not a multiple of 16 bytes";
+    case MW_ERR_CAPACITY: return "a buffer is too small for the rows assigned to it";
+    case MW_ERR_CUDA: return "a CUDA runtime call failed";
+    case MW_ERR_BAD_INDEX: return "expert id or expert-to-rank entry out of range";
+    case MW_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case MW_ERR_NO_PLAN: return "no plan has been made on this context";
+    default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,101 @@
+// Internal declarations shared by the translation units of libmw.so.  Not part of the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mw.h"
+
+#define MW_TILE 256          // tokens per plan tile = threads per plan block
+#define MW_SMALL_T_MAX 1024  // largest T the single-block plan handles
+
+// Per-plan accumulators filled by atomics; double buffered by plan parity so that the
+// buffer of the next plan is cleared by the current one and no separate memset is needed.
+struct mw_acc {
+    unsigned long long valid_slots;  // expert slots that named a valid expert on a valid rank
+    unsigned int self_only;          // tokens whose only destination is the source rank itself
+    int status;                      // first data-dependent error seen while planning
+};
+
+// Device workspace (all pointers into one slab owned by the context).
+struct mw_dev {
+    // public plan arrays (exposed through mw_plan_view)
+    uint64_t *token_mask;
+    int32_t *token_ndest, *token_group, *token_mw_row, *mw_row_token, *group_offsets;
+    uint64_t *group_mask;
+    int32_t *rank_offsets, *rank_tokens, *dest_rank, *dest_pos;
+    mw_totals *totals;
+    // internal plan arrays
+    int32_t *token_slot;     // [Tm]      hash slot of the token's bitmap
+    int32_t *token_leader;   // [Tm]      smallest token index with the same bitmap, -1 if empty
+    int32_t *token_gcount;   // [Tm]      size of the token's group
+    int32_t *gid_at;         // [Tm]      group id, stored at the leader's index
+    int32_t *goff_at;        // [Tm]      group offset, stored at the leader's index
+    int32_t *row_ndest;      // [Tm]      |D| of the token in MultiWrite send row j
+    int32_t *row_dest_rank;  // [Tm, Kd]  destination ranks of send row j
+    int32_t *row_dest_pos;   // [Tm, Kd]  slots of send row j
+    int32_t *uc_row_rank;    // [Tm * Kd] rank of every unicast send row
+    // scratch
+    int32_t *slot_rep, *slot_leader, *slot_count;  // [HS] open-addressed table keyed by bitmap
+    unsigned long long *tile_state;                // [max_tiles, NC] look-back records
+    unsigned int *ticket;                          // tile ticket counter
+    mw_acc *acc;                                   // [2]
+};
+
+struct mw_ctx {
+    mw_config cfg;
+    int W, Kd, HS, NC, max_tiles;
+    int sm_count;
+    int max_smem_optin;
+    mw_dev d;
+    void *slab;
+    uint32_t epoch;         // plans issued so far (tile records carry it, so they need no clearing)
+    uint32_t tickets_used;  // tile tickets handed out by all previous plans
+    int32_t planned_T;      // T of the latest plan, -1 before the first
+    int64_t launches;
+    // host staging (MW_FLAG_HOST_STAGING)
+    int32_t *st_ids, *st_e2r;
+    uint8_t *st_x, *st_send, *st_recv;
+    int64_t st_recv_rows;
+};
+
+// ---- plan (mw_plan.cu) ----
+int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t st);
+int mw_plan_smem_setup(mw_ctx *ctx);
+
+// ---- row copies (mw_copy.cu) ----
+enum mw_copy_mode {
+    MW_CP_PACK_MW = 0,      // send[j] = x[mw_row_token[j]]
+    MW_CP_SCATTER = 1,      // dst(region, slot) = src[row] for every destination of the row
+    MW_CP_DELIVER_UC = 2,   // region(r)[i] = send[rank_offsets[r] + i]
+    MW_CP_AG_PACK_MW = 3,   // send[i] = shard[i]
+    MW_CP_AG_DELIVER_MW = 4,// region(d)[i] = send[i] for every d of the window
+    MW_CP_AG_PACK_UC = 5,   // send[i][d] = shard[i] for every d of the window except rank i itself
+    MW_CP_AG_DELIVER_UC = 6 // region(d)[i] = send[i][d] (own shard: taken from shards)
+};
+
+struct mw_copy_args {
+    int mode;
+    const uint8_t *src;        // source rows (x, send buffer or shards)
+    const uint8_t *src2;       // AllGather unicast deliver: the shards (own copy is local)
+    uint8_t *dst;              // destination base
+    int64_t row_bytes;         // bytes per row (B, or the shard size)
+    int64_t dst_stride;        // bytes between receive regions; 0 = compact
+    int64_t capacity_rows;     // rows the destination may hold (per region when strided)
+    int64_t host_rows;         // row count known on the host (-1: read from totals)
+    int rows_from;             // 0: host_rows, 1: totals->T_nonempty, 2: totals->total_dest
+    int32_t chunk_bytes;       // bytes moved per work item (multiple of 16)
+    int32_t chunks_per_row;
+    int stages;                // bulk-copy pipeline depth per warp
+    int Kd, R, dst_begin, dst_count;
+    const int32_t *src_index;  // PACK_MW: mw_row_token
+    const int32_t *ndst;       // SCATTER: destinations per row
+    const int32_t *d_rank;     // SCATTER: [rows, Kd]
+    const int32_t *d_pos;      // SCATTER: [rows, Kd]
+    const int32_t *rank_offsets;
+    const int32_t *uc_row_rank;
+    mw_totals *totals;         // device accounting (row counts, status)
+};
+
+int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st);
+int mw_copy_smem_setup(mw_ctx *ctx);

@@ -1,0 +1,344 @@
+// Source-side planning kernels: destination bitmaps with per-rank dedup, grouping of tokens by
+// identical bitmap, per-group and per-rank counts with exclusive prefix sums, and every token's
+// send row and receive slots.  (Paper: Section 4.1, metadata encoding at the source; Section 5.1,
+// task decomposition in cs_send.  The slot layout rules are stated in mw.h.)
+//
+// Three kernels, chained on one stream:
+//   k_plan_mask   one thread per token: bitmap words, |D_t|, insertion of the bitmap into an
+//                 open-addressed table whose slot value is the smallest token index seen
+//                 (atomicMin), which makes the group "leader" independent of thread order;
+//   k_plan_tile   one block per 256-token tile, tiles taken in ticket order: a rank x token
+//                 bit matrix in shared memory gives every (token, rank) its position inside
+//                 the tile, the per-tile histogram of R rank counts (+ leader count, + group
+//                 size sum) is combined across tiles by a decoupled look-back scan, and the
+//                 last tile turns the grand totals into rank_offsets and the byte accounting;
+//   k_plan_final  one thread per token: group id / offset looked up at the leader, rank inside
+//                 the group, send row, inverse maps, per-row delivery descriptors; also restores
+//                 the table to its empty state for the next plan.
+#include "mw_internal.cuh"
+
+namespace {
+
+constexpr int kEmpty = -1;
+constexpr int kNoLeader = 0x7fffffff;
+constexpr unsigned kFlagAgg = 1u, kFlagPrefix = 2u;
+constexpr int kSpinLimit = 1 << 20;  // look-back polls before a tile gives up (about a second)
+
+struct PlanArgs {
+    const int32_t *ids, *e2r;
+    int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask;
+    int64_t row_bytes;
+    uint32_t epoch, ticket_base;
+    mw_dev d;
+};
+
+__device__ __forceinline__ void set_status(int *status, int err) { atomicCAS(status, 0, err); }
+
+__device__ __forceinline__ uint64_t mix64(uint64_t h, uint64_t v)
+{
+    h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
+    h ^= h >> 33; h *= 0xff51afd7ed558ccdull; h ^= h >> 29;
+    return h;
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel 1: bitmaps (Section 4.1: bit r set <=> rank r is a target) and the bitmap table.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(MW_TILE) k_plan_mask(PlanArgs a)
+{
+    const int t = blockIdx.x * MW_TILE + threadIdx.x;
+    mw_acc *acc = a.d.acc + (a.epoch & 1u);
+    int valid = 0, self_only = 0, bad = 0;
+    if (t < a.T) {
+        const int32_t *my = a.ids + (int64_t)t * a.K;
+        uint64_t *m = a.d.token_mask + (int64_t)t * a.W;
+        int nd = 0;
+        uint64_t h = 0x2545f4914f6cdd1dull, self_word = 0;
+        for (int w = 0; w < a.W; ++w) {
+            uint64_t word = 0;
+            for (int k = 0; k < a.K; ++k) {
+                const int id = my[k];
+                if (id == -1) continue;                               // padding slot
+                if (id < 0 || id >= a.E) { bad |= (w == 0); continue; }
+                const int r = a.e2r[id];
+                if (r < 0 || r >= a.R) { bad |= (w == 0); continue; }
+                valid += (w == 0);
+                if ((r >> 6) == w) word |= 1ull << (r & 63);          // OR = per-rank dedup
+            }
+            m[w] = word;
+            nd += __popcll(word);
+            h = mix64(h, word);
+            if (a.src_rank >= 0 && (a.src_rank >> 6) == w) self_word = word & (1ull << (a.src_rank & 63));
+        }
+        a.d.token_ndest[t] = nd;
+        self_only = (nd == 1 && self_word != 0);
+        int slot = kEmpty;
+        if (nd > 0) {
+            __threadfence();                                          // bitmap visible before the slot is claimed
+            slot = (int)(h & (uint64_t)a.hs_mask);
+            int probes = 0;
+            for (; probes <= a.hs_mask; ++probes) {
+                const int cur = atomicCAS(a.d.slot_rep + slot, kEmpty, t);
+                if (cur == kEmpty) break;                             // claimed an empty slot
+                __threadfence();
+                const uint64_t *o = a.d.token_mask + (int64_t)cur * a.W;
+                bool same = true;
+                for (int w = 0; w < a.W; ++w) same &= (__ldcg(o + w) == m[w]);
+                if (same) break;                                      // slot already holds this bitmap
+                slot = (slot + 1) & a.hs_mask;
+            }
+            if (probes > a.hs_mask) { set_status(&acc->status, MW_ERR_CAPACITY); slot = kEmpty; a.d.token_ndest[t] = 0; }
+            else { atomicMin(a.d.slot_leader + slot, t); atomicAdd(a.d.slot_count + slot, 1); }
+        }
+        a.d.token_slot[t] = slot;
+    }
+    valid = __reduce_add_sync(0xffffffffu, valid);
+    self_only = __reduce_add_sync(0xffffffffu, self_only);
+    bad = __reduce_or_sync(0xffffffffu, (unsigned)bad);
+    if ((threadIdx.x & 31) == 0) {
+        if (valid) atomicAdd(&acc->valid_slots, (unsigned long long)valid);
+        if (self_only) atomicAdd(&acc->self_only, (unsigned)self_only);
+        if (bad) set_status(&acc->status, MW_ERR_BAD_INDEX);
+    }
+}
+
+// Exclusive prefix sum over the 256 threads of a block; `total` is returned to every thread.
+__device__ __forceinline__ int block_excl_scan(int v, int *warp_sums /* [8] shared */, int &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { int n = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += n; }
+    __syncthreads();                       // protects warp_sums from a previous use
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = 0, sum = 0;
+#pragma unroll
+    for (int w = 0; w < MW_TILE / 32; ++w) { int s = warp_sums[w]; if (w < warp) before += s; sum += s; }
+    total = sum;
+    return before + incl - v;
+}
+
+__device__ __forceinline__ unsigned long long pack_state(uint32_t epoch, unsigned flag, uint32_t value)
+{
+    return ((unsigned long long)((epoch << 2) | flag) << 32) | value;
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel 2: per-tile histogram + decoupled look-back scan over tiles; positions inside regions.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
+{
+    extern __shared__ uint32_t sm[];
+    uint32_t *bits = sm;                          // [R, 8]  bit i of word w: token 32 w + i of the tile targets rank r
+    uint32_t *pre = bits + (size_t)a.R * 8;       // [R, 8]  tokens of the tile before word w that target rank r
+    int *cnt = (int *)(pre + (size_t)a.R * 8);    // [NC]    this tile's counters
+    int *base = cnt + a.NC;                       // [NC]    sum of the counters of all earlier tiles
+    __shared__ int warp_sums[MW_TILE / 32];
+    __shared__ int s_tile;
+
+    const int tid = threadIdx.x;
+    mw_acc *acc = a.d.acc + (a.epoch & 1u);
+    // Tiles are numbered in the order blocks start, so a tile only ever waits for tiles that are already running.
+    if (tid == 0) s_tile = (int)(atomicAdd(a.d.ticket, 1u) - a.ticket_base);
+    for (int i = tid; i < a.R * 8; i += MW_TILE) bits[i] = 0;
+    __syncthreads();
+    const int tile = s_tile;
+    const int t = tile * MW_TILE + tid;
+    const bool active = t < a.T;
+    const int nd = active ? a.d.token_ndest[t] : 0;
+    int leader = -1, gcount = 0;
+    if (nd > 0) {
+        const int slot = a.d.token_slot[t];
+        leader = a.d.slot_leader[slot];
+        gcount = a.d.slot_count[slot];
+    }
+    const bool is_leader = nd > 0 && leader == t;
+    if (active) { a.d.token_leader[t] = leader; a.d.token_gcount[t] = gcount; }
+
+    const uint64_t *m = a.d.token_mask + (int64_t)t * a.W;
+    const int wi = tid >> 5;
+    const uint32_t bit = 1u << (tid & 31);
+    if (nd > 0)
+        for (int w = 0; w < a.W; ++w)
+            for (uint64_t word = m[w]; word; word &= word - 1)
+                atomicOr(bits + (size_t)(w * 64 + __ffsll((long long)word) - 1) * 8 + wi, bit);
+    __syncthreads();
+    for (int r = tid; r < a.R; r += MW_TILE) {
+        int run = 0;
+#pragma unroll
+        for (int w8 = 0; w8 < 8; ++w8) { pre[r * 8 + w8] = run; run += __popc(bits[r * 8 + w8]); }
+        cnt[r] = run;
+    }
+    int lead_total, gc_total;
+    const int lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
+    const int gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
+    if (tid == 0) { cnt[a.R] = lead_total; cnt[a.R + 1] = gc_total; }
+    __syncthreads();
+
+    // Decoupled look-back, one thread per counter.  A record is one 64-bit word (epoch, flag, value),
+    // so flag and value are always read together; the epoch makes records of earlier plans invisible.
+    for (int c = tid; c < a.NC; c += MW_TILE) {
+        const uint32_t mine = (uint32_t)cnt[c];
+        volatile unsigned long long *rec = a.d.tile_state + (size_t)tile * a.NC + c;
+        uint32_t excl = 0;
+        if (tile == 0) {
+            *rec = pack_state(a.epoch, kFlagPrefix, mine);
+        } else {
+            *rec = pack_state(a.epoch, kFlagAgg, mine);
+            for (int j = tile - 1; j >= 0; --j) {
+                volatile unsigned long long *prev = a.d.tile_state + (size_t)j * a.NC + c;
+                unsigned long long s = 0;
+                int spins = 0;
+                for (; spins < kSpinLimit; ++spins) {
+                    s = *prev;
+                    const uint32_t hi = (uint32_t)(s >> 32);
+                    if ((hi >> 2) == (a.epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
+                    __nanosleep(64);
+                }
+                if (spins == kSpinLimit) { set_status(&acc->status, MW_ERR_TIMEOUT); break; }
+                excl += (uint32_t)s;
+                if (((uint32_t)(s >> 32) & 3u) == kFlagPrefix) break;
+            }
+            *rec = pack_state(a.epoch, kFlagPrefix, excl + mine);
+        }
+        base[c] = (int)excl;
+    }
+    __syncthreads();
+
+    if (active) {
+        if (is_leader) { a.d.gid_at[t] = base[a.R] + lead_excl; a.d.goff_at[t] = base[a.R + 1] + gc_excl; }
+        int i = 0;
+        int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
+        if (nd > 0)
+            for (int w = 0; w < a.W; ++w)
+                for (uint64_t word = m[w]; word; word &= word - 1) {
+                    const int r = w * 64 + __ffsll((long long)word) - 1;
+                    dr[i] = r;
+                    dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
+                    ++i;
+                }
+        for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
+    }
+
+    if (tile == a.ntiles - 1) {
+        // This tile's inclusive prefix is the grand total of every counter.
+        int carry = 0;
+        for (int r0 = 0; r0 < a.R; r0 += MW_TILE) {
+            const int r = r0 + tid;
+            const int v = r < a.R ? base[r] + cnt[r] : 0;
+            int total;
+            const int excl = block_excl_scan(v, warp_sums, total);
+            if (r < a.R) a.d.rank_offsets[r] = carry + excl;
+            carry += total;
+        }
+        if (tid == 0) {
+            const int64_t G = base[a.R] + cnt[a.R], Tn = base[a.R + 1] + cnt[a.R + 1], SD = carry;
+            const int64_t self_copies = a.src_rank >= 0 ? base[a.src_rank] + cnt[a.src_rank] : 0;
+            const int64_t sent_rows = Tn - (int64_t)acc->self_only;
+            a.d.rank_offsets[a.R] = (int32_t)SD;
+            a.d.group_offsets[G] = (int32_t)Tn;
+            mw_totals tt;
+            tt.T_nonempty = Tn;
+            tt.G = G;
+            tt.total_dest = SD;
+            tt.mw_bytes = sent_rows * a.row_bytes;
+            tt.unicast_bytes = (SD - self_copies) * a.row_bytes;
+            tt.unicast_per_expert_bytes = (int64_t)acc->valid_slots * a.row_bytes;
+            // Section 6.4: beyond 64 ranks the bitmap travels in the payload, once per 4096-byte packet
+            tt.meta_bytes = a.R <= 64 ? 0 : sent_rows * ((a.row_bytes + 4095) / 4096) * (int64_t)(8 * a.W);
+            tt.status = acc->status;
+            tt.reserved = 0;
+            *a.d.totals = tt;
+            mw_acc *next = a.d.acc + ((a.epoch + 1u) & 1u);
+            next->valid_slots = 0; next->self_only = 0; next->status = 0;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel 3: group ids and send rows, inverse maps, delivery descriptors, table clean-up.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
+{
+    const int t = blockIdx.x * MW_TILE + threadIdx.x;
+    const mw_totals *tot = a.d.totals;
+    const int Tn = (int)tot->T_nonempty, G = (int)tot->G, SD = (int)tot->total_dest;
+    if (t <= a.T && t > G) a.d.group_offsets[t] = -1;
+    if (t >= a.T) return;
+    if (t >= Tn) a.d.mw_row_token[t] = -1;
+    for (int i = 0; i < a.Kd; ++i)
+        if ((int64_t)t * a.Kd + i >= SD) a.d.rank_tokens[(int64_t)t * a.Kd + i] = -1;
+    for (int w = 0; w < a.W; ++w)
+        if (t >= G) a.d.group_mask[(int64_t)t * a.W + w] = 0;
+
+    const int leader = a.d.token_leader[t];
+    if (leader < 0) { a.d.token_group[t] = -1; a.d.token_mw_row[t] = -1; return; }
+    const int g = a.d.gid_at[leader], goff = a.d.goff_at[leader];
+    int within = 0;                                   // members of the group with a smaller token index
+    if (a.d.token_gcount[t] > 1)
+        for (int u = leader; u < t; ++u) within += (a.d.token_leader[u] == leader);
+    const int row = goff + within;
+    a.d.token_group[t] = g;
+    a.d.token_mw_row[t] = row;
+    a.d.mw_row_token[row] = t;
+    const int nd = a.d.token_ndest[t];
+    a.d.row_ndest[row] = nd;
+    if (leader == t) {
+        a.d.group_offsets[g] = goff;
+        for (int w = 0; w < a.W; ++w) a.d.group_mask[(int64_t)g * a.W + w] = a.d.token_mask[(int64_t)t * a.W + w];
+    }
+    for (int i = 0; i < a.Kd; ++i) {
+        const int r = a.d.dest_rank[(int64_t)t * a.Kd + i], p = a.d.dest_pos[(int64_t)t * a.Kd + i];
+        a.d.row_dest_rank[(int64_t)row * a.Kd + i] = r;
+        a.d.row_dest_pos[(int64_t)row * a.Kd + i] = p;
+        if (r >= 0) {
+            const int at = a.d.rank_offsets[r] + p;
+            a.d.rank_tokens[at] = t;
+            a.d.uc_row_rank[at] = r;
+        }
+    }
+    // leave the bitmap table empty for the next plan
+    const int slot = a.d.token_slot[t];
+    a.d.slot_rep[slot] = kEmpty;
+    a.d.slot_leader[slot] = kNoLeader;
+    a.d.slot_count[slot] = 0;
+}
+
+size_t tile_smem_bytes(const mw_ctx *ctx) { return ((size_t)ctx->cfg.R * 16 + 2 * (size_t)ctx->NC) * sizeof(uint32_t); }
+
+}  // namespace
+
+int mw_plan_smem_setup(mw_ctx *ctx)
+{
+    const size_t need = tile_smem_bytes(ctx);
+    if (need > (size_t)ctx->max_smem_optin) return MW_ERR_INVALID_ARG;
+    if (need > 48 * 1024 &&
+        cudaFuncSetAttribute(k_plan_tile, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)
+        return MW_ERR_CUDA;
+    return MW_OK;
+}
+
+int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t st)
+{
+    PlanArgs a;
+    a.ids = topk_ids; a.e2r = expert_to_rank;
+    a.T = T; a.K = ctx->cfg.K; a.E = ctx->cfg.E; a.R = ctx->cfg.R; a.W = ctx->W; a.Kd = ctx->Kd;
+    a.src_rank = ctx->cfg.src_rank;
+    a.ntiles = T > 0 ? (T + MW_TILE - 1) / MW_TILE : 1;
+    a.NC = ctx->NC; a.hs_mask = ctx->HS - 1;
+    a.row_bytes = ctx->cfg.row_bytes;
+    ctx->epoch += 1;
+    a.epoch = ctx->epoch & 0x3fffffffu;
+    a.ticket_base = ctx->tickets_used;
+    a.d = ctx->d;
+    const int blocks = a.ntiles;
+    k_plan_mask<<<blocks, MW_TILE, 0, st>>>(a);
+    k_plan_tile<<<blocks, MW_TILE, tile_smem_bytes(ctx), st>>>(a);
+    ctx->tickets_used += (uint32_t)blocks;
+    // one extra thread beyond T so that group_offsets[T] is covered
+    k_plan_final<<<(T + 1 + MW_TILE - 1) / MW_TILE, MW_TILE, 0, st>>>(a);
+    ctx->launches += 3;
+    ctx->planned_T = T;
+    return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}

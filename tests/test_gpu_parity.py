@@ -1,0 +1,296 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, bit for bit.
+
+Metadata arrays are compared whole (including their -1 / 0 tails), payload buffers byte by byte,
+with sentinel guard bands around every output buffer.  Integer and data-movement work only, so the
+tolerance is zero everywhere.
+"""
+import numpy as np
+import pytest
+
+from oracle import mwo
+from paper_2605_22428_b200 import binding as mw
+from paper_2605_22428_b200 import workloads as wl
+
+from gpu_util import Guarded, SENTINEL, assert_plan_equal, run_dispatch, torch_mod
+
+pytestmark = pytest.mark.gpu
+
+
+# ---- the four dispatch configurations ----------------------------------------------------------
+@pytest.mark.parametrize("cfg", [0, 1, 2, 3])
+@pytest.mark.parametrize("seed", [None, 100, 101])
+def test_plan_parity_full_configurations(cfg, seed):
+    inp = wl.make_dispatch(cfg, seed, payload=False)
+    run_dispatch(inp, check_payload=False, repeats=2)
+
+
+@pytest.mark.parametrize("cfg", [0, 3])
+def test_dispatch_parity_small_configurations_full_size(cfg):
+    run_dispatch(wl.make_dispatch(cfg))
+
+
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_dispatch_parity_large_configurations_full_size(cfg):
+    # full T and full hidden size, the shapes the benchmark times; compact MultiWrite + strided unicast
+    inp = wl.make_dispatch(cfg)
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",))
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_UNICAST,), strides=("strided",))
+
+
+@pytest.mark.parametrize("cfg", [1, 2])
+@pytest.mark.parametrize("seed", [100, 101])
+def test_dispatch_parity_large_configurations_reduced_hidden(cfg, seed):
+    run_dispatch(wl.make_dispatch(cfg, seed, H=264))          # 528-byte rows: ragged against every tile size
+
+
+@pytest.mark.parametrize("cfg", [0, 1])
+def test_register_copy_variant_matches(cfg):
+    inp = wl.make_dispatch(cfg, H=None if cfg == 0 else 520)
+    run_dispatch(inp, flags=mw.MW_FLAG_COPY_LDST)
+
+
+# ---- edge cases ------------------------------------------------------------------------------------
+@pytest.mark.parametrize("R", [1, 2, 63, 64, 65, 128, 129, 256, 1000, 1024])
+def test_rank_word_boundaries(R):
+    E = R if R > 8 else 8 * R
+    inp = wl.make_random_dispatch(R, T=300, K=min(6, R), E=E, R=R, H=24, pad_fraction=0.1)
+    ids = inp.topk_ids.copy()
+    e2r = inp.expert_to_rank.copy()
+    e2r[0], e2r[1] = 0, R - 1
+    ids[0, 0], ids[0, -1] = 0, 1                                   # first and last rank in one token
+    inp.topk_ids, inp.expert_to_rank = ids, e2r
+    run_dispatch(inp)
+
+
+@pytest.mark.parametrize("T", [0, 1, 31, 255, 256, 257, 1000, 1025])
+def test_token_counts_around_tile_edges(T):
+    inp = wl.make_random_dispatch(T + 3, T=T, K=3, E=40, R=10, H=40)
+    run_dispatch(inp, max_tokens=1100)
+
+
+def test_top1_and_few_large_groups():
+    # every token in a large group: exercises member ranking inside groups across tiles
+    inp = wl.make_random_dispatch(5, T=3000, K=1, E=12, R=6, H=16)
+    p, tot = run_dispatch(inp)
+    assert tot["G"] <= 6 and tot["mw_bytes"] == tot["unicast_bytes"]
+    inp = wl.make_random_dispatch(6, T=2500, K=2, E=8, R=4, H=16)
+    p, tot = run_dispatch(inp)
+    assert tot["G"] <= 10
+
+
+def test_all_tokens_identical_and_all_distinct():
+    T, R = 700, 70
+    e2r = np.arange(R, dtype=np.int32)
+    same = wl.make_random_dispatch(1, T=T, K=3, E=R, R=R, H=16)
+    same.expert_to_rank = e2r
+    same.topk_ids = np.tile(np.array([[3, 66, 9]], np.int32), (T, 1))
+    p, tot = run_dispatch(same)
+    assert tot["G"] == 1
+    dist = wl.make_random_dispatch(2, T=R, K=2, E=R, R=R, H=16)
+    dist.expert_to_rank = e2r
+    dist.topk_ids = np.stack([np.arange(R), (np.arange(R) + 1) % R], 1).astype(np.int32)
+    p, tot = run_dispatch(dist)
+    assert tot["G"] == R
+
+
+def test_padding_empty_tokens_duplicates_and_invalid_ids():
+    inp = wl.make_random_dispatch(7, T=600, K=4, E=24, R=7, H=16, pad_fraction=0.35, distinct=False)
+    ids = inp.topk_ids.copy()
+    ids[3, :] = -1
+    ids[299, :] = -1
+    ids[6, :] = ids[6, 0]
+    inp.topk_ids = ids
+    p, tot = run_dispatch(inp)
+    assert tot["status"] == 0 and tot["T_nonempty"] < 600
+    ids[4, 0] = 24                 # == E
+    ids[5, 1] = -2                 # negative, not the padding value
+    ids[500, 2] = 1 << 30
+    inp.topk_ids = ids
+    p, tot = run_dispatch(inp)
+    assert tot["status"] == mw.MW_ERR_BAD_INDEX
+    e2r = inp.expert_to_rank.copy()
+    e2r[2] = 7                     # == R
+    e2r[3] = -1
+    inp.expert_to_rank = e2r
+    p, tot = run_dispatch(inp)
+    assert tot["status"] == mw.MW_ERR_BAD_INDEX
+
+
+def test_all_padding_batch():
+    inp = wl.make_random_dispatch(9, T=300, K=4, E=16, R=4, H=16)
+    inp.topk_ids = np.full_like(inp.topk_ids, -1)
+    p, tot = run_dispatch(inp)
+    assert tot["G"] == 0 and tot["total_dest"] == 0 and tot["mw_bytes"] == 0
+
+
+def test_source_rank_inside_domain():
+    inp = wl.make_random_dispatch(11, T=500, K=3, E=16, R=6, H=16)
+    p, tot = run_dispatch(inp, src_rank=2)
+    q = mwo.plan(inp.topk_ids, inp.expert_to_rank, 6, 32, -1)
+    assert tot["unicast_bytes"] < q.totals["unicast_bytes"]
+
+
+def test_context_reuse_with_changing_batches_is_stateless():
+    """One context, many plans of different sizes: each result depends only on its own inputs."""
+    torch = torch_mod()
+    R, E, K, H = 16, 64, 4, 16
+    with mw.Context(R, E, K, 2048, 2 * H) as ctx:
+        for seed, T in [(1, 2048), (2, 5), (3, 777), (4, 0), (5, 2047), (1, 2048)]:
+            inp = wl.make_random_dispatch(seed, T=T, K=K, E=E, R=R, H=H, contiguous_map=True)
+            p = mwo.plan(inp.topk_ids, inp.expert_to_rank, R, 2 * H)
+            ids_d = torch.from_numpy(inp.topk_ids).cuda()
+            e2r_d = torch.from_numpy(inp.expert_to_rank).cuda()
+            ctx.mw_plan(ids_d, e2r_d, T)
+            assert_plan_equal(ctx.plan_arrays(T), p, ctx.mw_get_totals())
+
+
+def test_two_runs_give_identical_bytes():
+    torch = torch_mod()
+    inp = wl.make_dispatch("tiny")
+    s = inp.shape
+    outs = []
+    for _ in range(2):
+        with mw.Context(s.R, s.E, s.K, s.T, s.row_bytes) as ctx:
+            ids_d, e2r_d = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+            x_d = torch.from_numpy(inp.x.view(np.int16)).cuda()
+            ctx.mw_plan(ids_d, e2r_d, s.T)
+            tot = ctx.mw_get_totals()
+            send = torch.zeros(tot["T_nonempty"] * s.row_bytes, dtype=torch.uint8, device="cuda")
+            recv = torch.zeros(tot["total_dest"] * s.row_bytes, dtype=torch.uint8, device="cuda")
+            ctx.mw_dispatch(x_d, mw.MW_LAYOUT_MULTIWRITE, send, tot["T_nonempty"], recv, 0, tot["total_dest"])
+            torch.cuda.synchronize()
+            outs.append((send.cpu().numpy(), recv.cpu().numpy(), ctx.plan_arrays(s.T)))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    for k in outs[0][2]:
+        assert np.array_equal(outs[0][2][k], outs[1][2][k])
+
+
+def test_nan_and_negative_zero_payload_round_trips():
+    inp = wl.make_random_dispatch(3, T=64, K=2, E=8, R=4, H=16)
+    x = inp.x.copy()
+    x[0, :] = 0x7FC1      # NaN with payload
+    x[1, :] = 0x8000      # -0
+    x[2, :] = 0xFFFF
+    inp.x = x
+    run_dispatch(inp)
+
+
+# ---- capacity and argument errors ----------------------------------------------------------------
+def test_capacity_overflow_is_reported_and_contained():
+    torch = torch_mod()
+    inp = wl.make_random_dispatch(21, T=400, K=3, E=32, R=8, H=16, contiguous_map=True)
+    s = inp.shape
+    B = s.row_bytes
+    p = mwo.plan(inp.topk_ids, inp.expert_to_rank, s.R, B)
+    Tn, SD = p.totals["T_nonempty"], p.totals["total_dest"]
+    ids_d, e2r_d = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    x_d = torch.from_numpy(inp.x.view(np.int16)).cuda()
+    with mw.Context(s.R, s.E, s.K, s.T, B) as ctx:
+        # send buffer one row short
+        ctx.mw_plan(ids_d, e2r_d, s.T)
+        send, recv = Guarded((Tn - 1) * B), Guarded(SD * B)
+        ctx.mw_pack(x_d, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn - 1)
+        assert ctx.mw_get_totals()["status"] == mw.MW_ERR_CAPACITY
+        assert send.guards_intact()
+        assert np.array_equal(send.host().reshape(-1, B), mwo.pack_mw(p, inp.x)[:Tn - 1])
+        # compact receive area ten rows short: the rows that fit are right, nothing is written past the end
+        ctx.mw_plan(ids_d, e2r_d, s.T)
+        send = Guarded(Tn * B)
+        recv = Guarded((SD - 10) * B)
+        ctx.mw_dispatch(x_d, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn, recv.ptr(), 0, SD - 10)
+        assert ctx.mw_get_totals()["status"] == mw.MW_ERR_CAPACITY
+        assert recv.guards_intact()
+        want = mwo.deliver_mw(p, mwo.pack_mw(p, inp.x))
+        assert np.array_equal(recv.host(), want[:(SD - 10) * B])
+        # strided regions smaller than the fullest region
+        ctx.mw_plan(ids_d, e2r_d, s.T)
+        cap = int(np.diff(p.rank_offsets).max()) - 1
+        recv = Guarded(s.R * cap * B)
+        send_uc = Guarded(SD * B)
+        ctx.mw_dispatch(x_d, mw.MW_LAYOUT_UNICAST, send_uc.ptr(), SD, recv.ptr(), cap * B, cap)
+        assert ctx.mw_get_totals()["status"] == mw.MW_ERR_CAPACITY
+        assert recv.guards_intact()
+        # a fresh plan clears the status
+        ctx.mw_plan(ids_d, e2r_d, s.T)
+        assert ctx.mw_get_totals()["status"] == 0
+
+
+def test_host_side_argument_errors():
+    torch = torch_mod()
+    with pytest.raises(mw.MwError):
+        mw.Context(0, 8, 2, 16, 32)
+    with pytest.raises(mw.MwError):
+        mw.Context(2000, 8, 2, 16, 32)
+    with pytest.raises(mw.MwError) as e:
+        mw.Context(8, 8, 2, 16, 24)                       # row size not a multiple of 16
+    assert e.value.code == mw.MW_ERR_ALIGNMENT
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    ids = torch.zeros((16, 2), dtype=torch.int32, device="cuda")
+    e2r = torch.zeros(8, dtype=torch.int32, device="cuda")
+    with mw.Context(8, 8, 2, 16, 32) as ctx:
+        assert ctx.mw_pack(buf, 0, buf, 16, check=False) == mw.MW_ERR_NO_PLAN
+        assert ctx.mw_plan(ids, e2r, 17, check=False) == mw.MW_ERR_INVALID_ARG
+        assert ctx.mw_plan(None, e2r, 4, check=False) == mw.MW_ERR_INVALID_ARG
+        ctx.mw_plan(ids, e2r, 16)
+        assert ctx.mw_pack(buf.data_ptr() + 8, 0, buf, 16, check=False) == mw.MW_ERR_ALIGNMENT
+        assert ctx.mw_pack(buf, 5, buf, 16, check=False) == mw.MW_ERR_INVALID_ARG
+        assert ctx.mw_deliver(0, buf, buf.data_ptr() + 4, 0, 16, check=False) == mw.MW_ERR_ALIGNMENT
+        assert ctx.mw_deliver(0, buf, buf, 40, 1, check=False) == mw.MW_ERR_ALIGNMENT
+        assert ctx.mw_deliver(0, buf, buf, 64, 3, check=False) == mw.MW_ERR_CAPACITY
+        assert ctx.mw_deliver(0, None, buf, 0, 16, check=False) == mw.MW_ERR_INVALID_ARG
+        rc, _ = ctx.mw_allgather_pack(buf, 24, 0, buf, buf, check=False)
+        assert rc == mw.MW_ERR_ALIGNMENT
+        rc, _ = ctx.mw_allgather_pack(buf, 32, 0, buf, buf, 0, 6, 4, check=False)
+        assert rc == mw.MW_ERR_INVALID_ARG
+        rc, _ = ctx.mw_dispatch_host(ids, e2r, buf, 4, 0, buf, 16, e2r, check=False)
+        assert rc == mw.MW_ERR_INVALID_ARG               # context was created without host staging
+    assert mw.strerror(mw.MW_ERR_TIMEOUT) and mw.strerror(12345) == "unknown error code"
+
+
+# ---- AllGather ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
+@pytest.mark.parametrize("R,S,begin,count,strided", [
+    (8, 48, 0, 8, False), (5, 4112, 1, 3, True), (64, 4096, 0, 64, False), (64, 16384, 0, 64, False),
+    (64, 65536, 0, 64, True), (64, 1 << 18, 0, 64, False), (64, 1 << 20, 16, 16, False),
+    (64, 4 << 20, 60, 4, False), (64, 16 << 20, 63, 1, False), (1, 64, 0, 1, False), (3, 16, 2, 0, False)])
+def test_allgather_parity(layout, R, S, begin, count, strided):
+    torch = torch_mod()
+    sh = wl.make_allgather_shards(R, S, seed=4)
+    stride = R * S + 4096 if strided else 0
+    want_send, want_recv, want_tot, ret = mwo.allgather(sh, layout, begin, count, stride, SENTINEL)
+    assert ret == 0
+    sh_d = torch.from_numpy(sh).cuda()
+    send, recv = Guarded(len(want_send)), Guarded(max(len(want_recv), 16))
+    with mw.Context(R, 8, 2, 16, 32) as ctx:
+        rc, tot = ctx.mw_allgather_pack(sh_d, S, layout, send.ptr(), recv.ptr(), stride, begin, count)
+        torch.cuda.synchronize()
+    assert tot == want_tot
+    assert np.array_equal(send.host(), want_send)
+    assert np.array_equal(recv.host()[:len(want_recv)], want_recv)
+    assert send.guards_intact() and recv.guards_intact()
+
+
+# ---- the host-buffer entry point ---------------------------------------------------------------------
+@pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
+def test_dispatch_from_host_buffers(layout):
+    torch = torch_mod()
+    inp = wl.make_dispatch("dsv3_prefill", 100, T=1500, H=520)
+    s = inp.shape
+    B = s.row_bytes
+    p = mwo.plan(inp.topk_ids, inp.expert_to_rank, s.R, B)
+    want = mwo.deliver_definition(p, inp.x, inp.topk_ids, inp.expert_to_rank)
+    SD = p.totals["total_dest"]
+    recv_h = torch.full((SD * B + 64,), SENTINEL, dtype=torch.uint8).pin_memory()
+    ro_h = torch.zeros(s.R + 1, dtype=torch.int32).pin_memory()
+    x_h = torch.from_numpy(inp.x.view(np.int16)).pin_memory()
+    ids_h = torch.from_numpy(inp.topk_ids).pin_memory()
+    e2r_h = torch.from_numpy(inp.expert_to_rank)
+    with mw.Context(s.R, s.E, s.K, 2000, B, flags=mw.MW_FLAG_HOST_STAGING) as ctx:
+        for _ in range(2):
+            rc, tot = ctx.mw_dispatch_host(ids_h, e2r_h, x_h, s.T, layout, recv_h, SD, ro_h)
+            assert tot == p.totals
+            assert np.array_equal(ro_h.numpy(), p.rank_offsets)
+            assert np.array_equal(recv_h.numpy()[:SD * B], want)
+            assert (recv_h.numpy()[SD * B:] == SENTINEL).all()
+        rc, _ = ctx.mw_dispatch_host(ids_h, e2r_h, x_h, s.T, layout, recv_h, SD - 1, ro_h, check=False)
+        assert rc == mw.MW_ERR_CAPACITY
