@@ -76,6 +76,7 @@ extern "C" {
 
 #define MW_MAX_RANKS   1024
 #define MW_MAX_TOPK    64
+#define MW_STATIC_MAX_TOKENS 16384   /* largest T of mw_group_tokens_static */
 
 typedef struct mw_ctx mw_ctx;   /* opaque: configuration, device workspace, plan metadata */
 
@@ -217,6 +218,44 @@ MW_API int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_byte
 MW_API int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int32_t *expert_to_rank_host,
                      const void *x_host, int32_t T, int layout, void *recv_host, int64_t recv_capacity_rows,
                      int32_t *rank_offsets_host, mw_totals *totals_host, void *stream);
+
+/*
+ * Bitmaps and token grouping without any allocation.  (The paper has no counterpart for this
+ * entry point; it exists for a class of callers, not for a step of the method.)
+ *
+ * Some hosts of this library may not allocate device memory themselves: a serving process that
+ * hands the whole GPU to its framework's memory pool at start-up leaves nothing for a later
+ * cudaMalloc, and a caller on a latency-critical path cannot afford the device-wide
+ * synchronisation an allocation or free may imply.  Such callers cannot use mw_create.  This call
+ * allocates nothing, neither through CUDA nor through any library: its scratch (the table keyed by
+ * bitmap and one slot index per token, 448 KB) is a fixed array inside the library image, present
+ * on every GPU that loads the library until the process exits.  The caller passes all inputs and
+ * all outputs.
+ *
+ * It computes, for the current device and on `stream`, the first part of the plan:
+ *   token_mask        device, uint64 [T, W], W = ceil(R / 64): destination bitmap (same rules as mw_plan)
+ *   token_ndest       device, int32 [T]: |D_t|
+ *   token_leader      device, int32 [T]: smallest token index whose bitmap equals this token's
+ *                     (the first member of its group), -1 if the bitmap is empty
+ *   token_group_size  device, int32 [T]: number of tokens with that bitmap, 0 if empty
+ *   status            device, int32 [1]: MW_OK, or MW_ERR_BAD_INDEX if an id or table entry was
+ *                     out of range (such slots are ignored)
+ * Inputs as for mw_plan: topk_ids device int32 [T, K], expert_to_rank device int32 [E].
+ *
+ * Limits and rules
+ *   - T <= MW_STATIC_MAX_TOKENS; a larger T returns MW_ERR_CAPACITY and launches nothing.
+ *   - The first call on each device looks up the device address of the array (one CUDA runtime
+ *     query, no allocation); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous call's contents;
+ *     every call therefore begins by emptying the table on `stream`.  Two calls whose GPU work
+ *     overlaps (different streams, or different host threads without ordering) race on the array
+ *     and give undefined results: order them on one stream or with events.
+ *   - Returns MW_ERR_INVALID_ARG for null pointers or sizes out of range, MW_ERR_CUDA if the
+ *     runtime fails; asynchronous otherwise.
+ */
+MW_API int mw_group_tokens_static(const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, int32_t K,
+                                  int32_t E, int32_t R, uint64_t *token_mask, int32_t *token_ndest,
+                                  int32_t *token_leader, int32_t *token_group_size, int32_t *status, void *stream);
 
 /*
  * Convenience for reading plan metadata: waits for `stream`, then copies `bytes` from a device

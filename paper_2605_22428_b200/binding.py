@@ -28,7 +28,8 @@ MW_FLAG_PLAN_MULTIPASS = 0x2
 MW_FLAG_COPY_LDST = 0x4
 
 EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch",
-           "mw_allgather_pack", "mw_dispatch_host", "mw_read_device", "mw_kernel_launches", "mw_strerror")
+           "mw_allgather_pack", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
+           "mw_strerror")
 
 
 class mw_config(C.Structure):
@@ -87,12 +88,13 @@ def lib():
         L.mw_dispatch.argtypes = [vp, vp, C.c_int, vp, i64, vp, i64, i64, vp]
         L.mw_allgather_pack.argtypes = [vp, vp, i64, C.c_int, vp, vp, i64, i32, i32, C.POINTER(mw_totals), vp]
         L.mw_dispatch_host.argtypes = [vp, vp, vp, vp, i32, C.c_int, vp, i64, vp, C.POINTER(mw_totals), vp]
+        L.mw_group_tokens_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.mw_read_device.argtypes = [vp, vp, vp, i64, vp]
         L.mw_kernel_launches.argtypes = [vp]
         L.mw_kernel_launches.restype = C.c_int64
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:10]:
+        for name in EXPORTS[:11]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -120,6 +122,20 @@ def _stream(stream) -> C.c_void_p:
     if isinstance(stream, int):
         return C.c_void_p(stream)
     return C.c_void_p(stream.cuda_stream)
+
+
+MW_STATIC_MAX_TOKENS = 16384
+
+
+def mw_group_tokens_static(topk_ids, expert_to_rank, T: int, K: int, E: int, R: int, token_mask, token_ndest,
+                           token_leader, token_group_size, status, stream=None) -> int:
+    """Bitmaps and token grouping for callers that may not allocate device memory (for example a
+    server whose framework pool owns the whole GPU): the library's own fixed scratch array is used,
+    every buffer is the caller's.  Returns the C return code; see include/mw.h for the rules
+    (T <= MW_STATIC_MAX_TOKENS, calls that overlap on the GPU race on the shared scratch)."""
+    return lib().mw_group_tokens_static(_ptr(topk_ids), _ptr(expert_to_rank), T, K, E, R, _ptr(token_mask),
+                                        _ptr(token_ndest), _ptr(token_leader), _ptr(token_group_size),
+                                        _ptr(status), _stream(stream))
 
 
 class Context:
