@@ -49,11 +49,12 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.row_dest_rank = k.take<int32_t>(Tm * Kd);
     d.row_dest_pos = k.take<int32_t>(Tm * Kd);
     d.uc_row_rank = k.take<int32_t>(Tm * Kd);
-    d.slot_rep = k.take<int32_t>((size_t)c->HS);
+    d.slot_key = k.take<unsigned long long>((size_t)c->HS);
     d.slot_leader = k.take<int32_t>((size_t)c->HS);
     d.slot_count = k.take<int32_t>((size_t)c->HS);
     d.tile_state = k.take<unsigned long long>((size_t)c->max_tiles * (size_t)c->NC);
     d.ticket = k.take<unsigned int>(1);
+    d.gbar = k.take<unsigned int>(1);
     d.acc = k.take<mw_acc>(2);
     if (c->cfg.flags & MW_FLAG_HOST_STAGING) {
         const size_t B = (size_t)c->cfg.row_bytes;
@@ -116,12 +117,13 @@ int mw_create(mw_ctx **out, const mw_config *cfg)
     c->Kd = cfg->K < cfg->R ? cfg->K : cfg->R;
     c->NC = cfg->R + 2;
     c->max_tiles = (cfg->max_tokens + MW_TILE - 1) / MW_TILE;
-    int hs = 256;
-    while (hs < 2 * cfg->max_tokens) hs <<= 1;
+    int hs = 1024;                                    // load factor <= 1/8 keeps probe chains short
+    while (hs < 8 * cfg->max_tokens) hs <<= 1;
     c->HS = hs;
     c->planned_T = -1;
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
+    cudaDeviceGetAttribute(&c->coop_ok, cudaDevAttrCooperativeLaunch, cfg->device);
 
     const size_t bytes = carve(c, nullptr);
     if (cudaMalloc(&c->slab, bytes) != cudaSuccess) { cudaGetLastError(); delete c; return MW_ERR_CUDA; }
@@ -130,7 +132,7 @@ int mw_create(mw_ctx **out, const mw_config *cfg)
     if (cudaMemset(c->slab, 0, bytes) != cudaSuccess) rc = MW_ERR_CUDA;
     // empty table: no representative, no leader
     if (rc == MW_OK) {
-        k_fill_i32<<<64, 256>>>(c->d.slot_rep, c->HS, -1);
+        k_fill_i32<<<64, 256>>>((int32_t *)c->d.slot_key, 2 * (int64_t)c->HS, -1);   // all ones = empty slot
         k_fill_i32<<<64, 256>>>(c->d.slot_leader, c->HS, 0x7fffffff);
         if (cudaDeviceSynchronize() != cudaSuccess) rc = MW_ERR_CUDA;
     }

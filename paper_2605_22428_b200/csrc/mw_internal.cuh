@@ -36,9 +36,11 @@ struct mw_dev {
     int32_t *row_dest_pos;   // [Tm, Kd]  slots of send row j
     int32_t *uc_row_rank;    // [Tm * Kd] rank of every unicast send row
     // scratch
-    int32_t *slot_rep, *slot_leader, *slot_count;  // [HS] open-addressed table keyed by bitmap
+    unsigned long long *slot_key;                  // [HS] open-addressed table keyed by bitmap: (hash tag, first token)
+    int32_t *slot_leader, *slot_count;             // [HS] smallest token index / number of tokens with that bitmap
     unsigned long long *tile_state;                // [max_tiles, NC] look-back records
     unsigned int *ticket;                          // tile ticket counter
+    unsigned int *gbar;                            // arrival counter of the fused plan's grid barriers
     mw_acc *acc;                                   // [2]
 };
 
@@ -51,6 +53,8 @@ struct mw_ctx {
     void *slab;
     uint32_t epoch;         // plans issued so far (tile records carry it, so they need no clearing)
     uint32_t tickets_used;  // tile tickets handed out by all previous plans
+    uint32_t gbar_arrivals; // grid-barrier arrivals made by all previous fused plans
+    int coop_ok;            // device supports cooperative launch
     int32_t planned_T;      // T of the latest plan, -1 before the first
     int64_t launches;
     // host staging (MW_FLAG_HOST_STAGING)

@@ -3,7 +3,12 @@
 // send row and receive slots.  (Paper: Section 4.1, metadata encoding at the source; Section 5.1,
 // task decomposition in cs_send.  The slot layout rules are stated in mw.h.)
 //
-// Three kernels, chained on one stream:
+// Two ways to run the same three phases:
+//   k_plan_fused  one cooperative launch, one block per 256-token tile, all blocks resident, the
+//                 phases separated by two bounded grid barriers; a token's values stay in the
+//                 registers of "its" thread from phase to phase.  Taken whenever the tiles fit on
+//                 the SMs (T <= 256 x SM count).
+//   multi-pass    three kernels chained on one stream, for larger T (or MW_FLAG_PLAN_MULTIPASS):
 //   k_plan_mask   one thread per token: bitmap words, |D_t|, insertion of the bitmap into an
 //                 open-addressed table whose slot value is the smallest token index seen
 //                 (atomicMin), which makes the group "leader" independent of thread order;
@@ -20,6 +25,7 @@
 namespace {
 
 constexpr int kEmpty = -1;
+constexpr unsigned long long kEmptyKey = ~0ull;
 constexpr int kNoLeader = 0x7fffffff;
 constexpr unsigned kFlagAgg = 1u, kFlagPrefix = 2u;
 constexpr int kSpinLimit = 1 << 20;  // look-back polls before a tile gives up (about a second)
@@ -28,7 +34,7 @@ struct PlanArgs {
     const int32_t *ids, *e2r;
     int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask;
     int64_t row_bytes;
-    uint32_t epoch, ticket_base;
+    uint32_t epoch, ticket_base, bar_base;
     mw_dev d;
 };
 
@@ -39,6 +45,28 @@ __device__ __forceinline__ uint64_t mix64(uint64_t h, uint64_t v)
     h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
     h ^= h >> 33; h *= 0xff51afd7ed558ccdull; h ^= h >> 29;
     return h;
+}
+
+
+// Finds (or claims) the table slot of a bitmap.  A slot holds (32-bit hash tag, first token that
+// claimed it); a probe that meets another tag moves on after one CAS, and the full bitmap is only
+// compared when the tags agree.  Returns -1 if the table is full (cannot happen at load <= 1/8).
+template <class SameFn>
+__device__ __forceinline__ int table_insert(unsigned long long *slot_key, int hs_mask, uint64_t h, int t, SameFn same_as)
+{
+    const uint32_t tag = (uint32_t)(h >> 32);
+    const unsigned long long mine = ((unsigned long long)tag << 32) | (uint32_t)t;
+    int slot = (int)(h & (uint64_t)hs_mask);
+    for (int probes = 0; probes <= hs_mask; ++probes) {
+        const unsigned long long cur = atomicCAS(slot_key + slot, kEmptyKey, mine);
+        if (cur == kEmptyKey) return slot;                                // claimed an empty slot
+        if ((uint32_t)(cur >> 32) == tag) {
+            __threadfence();
+            if (same_as((int)(uint32_t)cur)) return slot;                 // slot already holds this bitmap
+        }
+        slot = (slot + 1) & hs_mask;
+    }
+    return -1;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -75,19 +103,14 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_mask(PlanArgs a)
         int slot = kEmpty;
         if (nd > 0) {
             __threadfence();                                          // bitmap visible before the slot is claimed
-            slot = (int)(h & (uint64_t)a.hs_mask);
-            int probes = 0;
-            for (; probes <= a.hs_mask; ++probes) {
-                const int cur = atomicCAS(a.d.slot_rep + slot, kEmpty, t);
-                if (cur == kEmpty) break;                             // claimed an empty slot
-                __threadfence();
-                const uint64_t *o = a.d.token_mask + (int64_t)cur * a.W;
+            const int W = a.W;
+            const uint64_t *masks = a.d.token_mask;
+            slot = table_insert(a.d.slot_key, a.hs_mask, h, t, [=](int other) {
                 bool same = true;
-                for (int w = 0; w < a.W; ++w) same &= (__ldcg(o + w) == m[w]);
-                if (same) break;                                      // slot already holds this bitmap
-                slot = (slot + 1) & a.hs_mask;
-            }
-            if (probes > a.hs_mask) { set_status(&acc->status, MW_ERR_CAPACITY); slot = kEmpty; a.d.token_ndest[t] = 0; }
+                for (int w = 0; w < W; ++w) same &= (__ldcg(masks + (int64_t)other * W + w) == m[w]);
+                return same;
+            });
+            if (slot < 0) { set_status(&acc->status, MW_ERR_CAPACITY); a.d.token_ndest[t] = 0; }
             else { atomicMin(a.d.slot_leader + slot, t); atomicAdd(a.d.slot_count + slot, 1); }
         }
         a.d.token_slot[t] = slot;
@@ -257,27 +280,107 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
 }
 
 // ------------------------------------------------------------------------------------------
+// Rank of every token inside its group (number of members with a smaller token index), for one
+// 256-token tile, computed by the whole block.  Only groups with more than one member need work:
+//   - the tile's distinct multi-member leaders go into a small shared-memory hash (key = leader);
+//     each entry has a 256-bit bitmap of the tile's members, whose popcount prefix gives the rank
+//     inside the tile, and a counter of members seen in earlier tiles;
+//   - every earlier tile, from the tile of the smallest such leader on, is read once (coalesced,
+//     eight independent loads per round) and each value is looked up in the hash.
+// A group's first member is its leader, so no member lives before the leader's tile.
+// ------------------------------------------------------------------------------------------
+constexpr int kRankSlots = 512;      // shared hash slots: at most 256 distinct leaders per tile
+struct RankScratch {
+    int key[kRankSlots];             // leader token index, -1 = empty
+    int earlier[kRankSlots];         // members in earlier tiles
+    uint32_t members[kRankSlots][8]; // bit i of word w: token 32 w + i of this tile is a member
+    int first_tile;                  // smallest tile that holds one of the tile's multi-member leaders
+};
+
+__device__ __forceinline__ int rank_slot_find(const int *key, int leader)
+{
+    int e = (int)(((uint32_t)leader * 2654435761u) >> 23) & (kRankSlots - 1);
+    while (true) {
+        const int k = key[e];
+        if (k == leader) return e;
+        if (k == -1) return -1;
+        e = (e + 1) & (kRankSlots - 1);
+    }
+}
+
+// `leader` is -1 for a token without destinations; `gcount` its group size; `token_leader` is the
+// global array holding the leader of every token (complete before this is called).  All threads of
+// the block must call it.
+__device__ int group_rank_in_tile(RankScratch *rs, const int32_t *token_leader, int tile, int leader, int gcount)
+{
+    const int tid = threadIdx.x;
+    const bool multi = leader >= 0 && gcount > 1;
+    if (!__syncthreads_or(multi)) return 0;                       // every group of this tile is a singleton
+    for (int i = tid; i < kRankSlots; i += MW_TILE) {
+        rs->key[i] = -1; rs->earlier[i] = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) rs->members[i][w] = 0;
+    }
+    if (tid == 0) rs->first_tile = tile;
+    __syncthreads();
+    int e = -1;
+    if (multi) {
+        e = (int)(((uint32_t)leader * 2654435761u) >> 23) & (kRankSlots - 1);
+        while (true) {
+            const int k = atomicCAS(rs->key + e, -1, leader);
+            if (k == -1 || k == leader) break;
+            e = (e + 1) & (kRankSlots - 1);
+        }
+        atomicOr(&rs->members[e][tid >> 5], 1u << (tid & 31));
+        atomicMin(&rs->first_tile, leader / MW_TILE);
+    }
+    __syncthreads();
+    const int first_tile = rs->first_tile;
+    for (int j0 = first_tile; j0 < tile; j0 += 8) {
+        int v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = (j0 + i < tile) ? __ldcg(token_leader + (int64_t)(j0 + i) * MW_TILE + tid) : -1;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (v[i] < 0) continue;
+            const int f = rank_slot_find(rs->key, v[i]);
+            if (f >= 0) atomicAdd(rs->earlier + f, 1);
+        }
+    }
+    __syncthreads();
+    int within = 0;
+    if (multi) {
+        within = rs->earlier[e];
+        const int wi = tid >> 5;
+        for (int w = 0; w < wi; ++w) within += __popc(rs->members[e][w]);
+        within += __popc(rs->members[e][wi] & ((1u << (tid & 31)) - 1u));
+    }
+    return within;
+}
+
+// ------------------------------------------------------------------------------------------
 // Kernel 3: group ids and send rows, inverse maps, delivery descriptors, table clean-up.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
 {
+    __shared__ RankScratch rank_scratch;
     const int t = blockIdx.x * MW_TILE + threadIdx.x;
     const mw_totals *tot = a.d.totals;
     const int Tn = (int)tot->T_nonempty, G = (int)tot->G, SD = (int)tot->total_dest;
     if (t <= a.T && t > G) a.d.group_offsets[t] = -1;
+    if (t < a.T) {
+        if (t >= Tn) a.d.mw_row_token[t] = -1;
+        for (int i = 0; i < a.Kd; ++i)
+            if ((int64_t)t * a.Kd + i >= SD) a.d.rank_tokens[(int64_t)t * a.Kd + i] = -1;
+        for (int w = 0; w < a.W; ++w)
+            if (t >= G) a.d.group_mask[(int64_t)t * a.W + w] = 0;
+    }
+    const int leader = t < a.T ? a.d.token_leader[t] : -1;
+    const int gcount = leader >= 0 ? a.d.token_gcount[t] : 0;
+    const int within = group_rank_in_tile(&rank_scratch, a.d.token_leader, blockIdx.x, leader, gcount);
     if (t >= a.T) return;
-    if (t >= Tn) a.d.mw_row_token[t] = -1;
-    for (int i = 0; i < a.Kd; ++i)
-        if ((int64_t)t * a.Kd + i >= SD) a.d.rank_tokens[(int64_t)t * a.Kd + i] = -1;
-    for (int w = 0; w < a.W; ++w)
-        if (t >= G) a.d.group_mask[(int64_t)t * a.W + w] = 0;
-
-    const int leader = a.d.token_leader[t];
     if (leader < 0) { a.d.token_group[t] = -1; a.d.token_mw_row[t] = -1; return; }
     const int g = a.d.gid_at[leader], goff = a.d.goff_at[leader];
-    int within = 0;                                   // members of the group with a smaller token index
-    if (a.d.token_gcount[t] > 1)
-        for (int u = leader; u < t; ++u) within += (a.d.token_leader[u] == leader);
     const int row = goff + within;
     a.d.token_group[t] = g;
     a.d.token_mw_row[t] = row;
@@ -300,7 +403,295 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
     }
     // leave the bitmap table empty for the next plan
     const int slot = a.d.token_slot[t];
-    a.d.slot_rep[slot] = kEmpty;
+    a.d.slot_key[slot] = kEmptyKey;
+    a.d.slot_leader[slot] = kNoLeader;
+    a.d.slot_count[slot] = 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused plan: the three phases in one cooperative launch.
+// ------------------------------------------------------------------------------------------
+constexpr int kBarrierSpinLimit = 1 << 21;   // polls of the arrival counter before a block gives up (about a second)
+
+__device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.volatile.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// All blocks of the (co-resident) grid arrive; a block that is still `alive` then waits until the
+// counter reaches `target`.  Every block always arrives, so the host's running count of arrivals
+// stays exact even after a block has given up.  Returns false for a block that gave up (now or before).
+__device__ bool grid_barrier(unsigned int *counter, unsigned int target, bool alive, int *status)
+{
+    __shared__ int s_alive;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        int ok = alive ? 1 : 0;
+        if (ok) {
+            int spins = 0;
+            while ((int)(ld_volatile_u32(counter) - target) < 0) {
+                if (++spins > kBarrierSpinLimit) { ok = 0; set_status(status, MW_ERR_TIMEOUT); break; }
+                __nanosleep(32);
+            }
+        }
+        __threadfence();
+        s_alive = ok;
+    }
+    __syncthreads();
+    return s_alive != 0;
+}
+
+template <int WT>
+__global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
+{
+    extern __shared__ uint32_t sm[];
+    uint32_t *bits = sm;
+    uint32_t *pre = bits + (size_t)a.R * 8;
+    int *cnt = (int *)(pre + (size_t)a.R * 8);
+    int *base = cnt + a.NC;
+    __shared__ int warp_sums[MW_TILE / 32];
+    __shared__ RankScratch rank_scratch;
+
+    const int tid = threadIdx.x, tile = blockIdx.x;
+    const int t = tile * MW_TILE + tid;
+    const bool active = t < a.T;
+    mw_acc *acc = a.d.acc + (a.epoch & 1u);
+
+    // ---- phase A: bitmap (Section 4.1: bit r set <=> rank r is a target) and the bitmap table ----
+    uint64_t m[WT];
+#pragma unroll
+    for (int w = 0; w < WT; ++w) m[w] = 0;
+    int nd = 0, slot = kEmpty;
+    {
+        int valid = 0, bad = 0, self_only = 0;
+        if (active) {
+            const int32_t *my = a.ids + (int64_t)t * a.K;
+            for (int k0 = 0; k0 < a.K; k0 += 8) {
+                int id[8], r[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) id[j] = (k0 + j < a.K) ? my[k0 + j] : -1;      // 8 independent loads
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const bool ok = id[j] >= 0 && id[j] < a.E;
+                    bad |= (id[j] != -1 && !ok);
+                    r[j] = ok ? a.e2r[id[j]] : -1;                                          // 8 independent loads
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const bool ok = r[j] >= 0 && r[j] < a.R;
+                    bad |= (id[j] >= 0 && id[j] < a.E && !ok);
+                    valid += ok;
+                    if (ok) {
+#pragma unroll
+                        for (int w = 0; w < WT; ++w)
+                            if ((r[j] >> 6) == w) m[w] |= 1ull << (r[j] & 63);              // OR = per-rank dedup
+                    }
+                }
+            }
+            uint64_t h = 0x2545f4914f6cdd1dull;
+            uint64_t *mg = a.d.token_mask + (int64_t)t * a.W;
+#pragma unroll
+            for (int w = 0; w < WT; ++w)
+                if (w < a.W) { mg[w] = m[w]; nd += __popcll(m[w]); h = mix64(h, m[w]); }
+            a.d.token_ndest[t] = nd;
+            if (a.src_rank >= 0 && nd == 1) {
+#pragma unroll
+                for (int w = 0; w < WT; ++w)
+                    if ((a.src_rank >> 6) == w) self_only = (m[w] >> (a.src_rank & 63)) & 1;
+            }
+            if (nd > 0) {
+                __threadfence();                                      // bitmap visible before the slot is claimed
+                const int W = a.W;
+                const uint64_t *masks = a.d.token_mask;
+                slot = table_insert(a.d.slot_key, a.hs_mask, h, t, [&](int other) {
+                    bool same = true;
+#pragma unroll
+                    for (int w = 0; w < WT; ++w)
+                        if (w < W) same &= (__ldcg(masks + (int64_t)other * W + w) == m[w]);
+                    return same;
+                });
+                if (slot < 0) { set_status(&acc->status, MW_ERR_CAPACITY); nd = 0; a.d.token_ndest[t] = 0; }
+                else { atomicMin(a.d.slot_leader + slot, t); atomicAdd(a.d.slot_count + slot, 1); }
+            }
+        }
+        valid = __reduce_add_sync(0xffffffffu, valid);
+        self_only = __reduce_add_sync(0xffffffffu, self_only);
+        bad = __reduce_or_sync(0xffffffffu, (unsigned)bad);
+        if ((tid & 31) == 0) {
+            if (valid) atomicAdd(&acc->valid_slots, (unsigned long long)valid);
+            if (self_only) atomicAdd(&acc->self_only, (unsigned)self_only);
+            if (bad) set_status(&acc->status, MW_ERR_BAD_INDEX);
+        }
+    }
+    for (int i = tid; i < a.R * 8; i += MW_TILE) bits[i] = 0;
+    bool alive = grid_barrier(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
+
+    // ---- phase B: positions inside the tile, tile histogram, look-back over tiles ----
+    int leader = -1, gcount = 0;
+    const int wi = tid >> 5;
+    const uint32_t bit = 1u << (tid & 31);
+    if (alive) {
+        if (nd > 0) { leader = __ldcg(a.d.slot_leader + slot); gcount = __ldcg(a.d.slot_count + slot); }
+        const bool is_leader = nd > 0 && leader == t;
+        if (active) a.d.token_leader[t] = leader;
+        if (nd > 0) {
+#pragma unroll
+            for (int w = 0; w < WT; ++w)
+                for (uint64_t word = m[w]; word; word &= word - 1)
+                    atomicOr(bits + (size_t)(w * 64 + __ffsll((long long)word) - 1) * 8 + wi, bit);
+        }
+        __syncthreads();
+        for (int r = tid; r < a.R; r += MW_TILE) {
+            int run = 0;
+#pragma unroll
+            for (int w8 = 0; w8 < 8; ++w8) { pre[r * 8 + w8] = run; run += __popc(bits[r * 8 + w8]); }
+            cnt[r] = run;
+        }
+        int lead_total, gc_total;
+        const int lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
+        const int gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
+        if (tid == 0) { cnt[a.R] = lead_total; cnt[a.R + 1] = gc_total; }
+        __syncthreads();
+
+        // Decoupled look-back, one thread per counter, eight predecessors fetched per round trip.
+        for (int c = tid; c < a.NC; c += MW_TILE) {
+            const uint32_t mine = (uint32_t)cnt[c];
+            volatile unsigned long long *rec = a.d.tile_state + (size_t)tile * a.NC + c;
+            uint32_t excl = 0;
+            if (tile == 0) {
+                *rec = pack_state(a.epoch, kFlagPrefix, mine);
+            } else {
+                *rec = pack_state(a.epoch, kFlagAgg, mine);
+                bool done = false;
+                for (int j = tile - 1; j >= 0 && !done; j -= 8) {
+                    unsigned long long s[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        s[i] = (j - i >= 0) ? *(volatile unsigned long long *)(a.d.tile_state + (size_t)(j - i) * a.NC + c) : 0ull;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (done || j - i < 0) continue;
+                        int spins = 0;
+                        while (true) {
+                            const uint32_t hi = (uint32_t)(s[i] >> 32);
+                            if ((hi >> 2) == (a.epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
+                            if (++spins > kSpinLimit) { set_status(&acc->status, MW_ERR_TIMEOUT); done = true; break; }
+                            __nanosleep(64);
+                            s[i] = *(volatile unsigned long long *)(a.d.tile_state + (size_t)(j - i) * a.NC + c);
+                        }
+                        if (done) break;
+                        excl += (uint32_t)s[i];
+                        if (((uint32_t)(s[i] >> 32) & 3u) == kFlagPrefix) done = true;
+                    }
+                }
+                *rec = pack_state(a.epoch, kFlagPrefix, excl + mine);
+            }
+            base[c] = (int)excl;
+        }
+        __syncthreads();
+
+        if (active) {
+            if (is_leader) { a.d.gid_at[t] = base[a.R] + lead_excl; a.d.goff_at[t] = base[a.R + 1] + gc_excl; }
+            int i = 0;
+            int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
+            if (nd > 0) {
+#pragma unroll
+                for (int w = 0; w < WT; ++w)
+                    for (uint64_t word = m[w]; word; word &= word - 1) {
+                        const int r = w * 64 + __ffsll((long long)word) - 1;
+                        dr[i] = r;
+                        dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
+                        ++i;
+                    }
+            }
+            for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
+        }
+        if (tile == a.ntiles - 1) {
+            int carry = 0;
+            for (int r0 = 0; r0 < a.R; r0 += MW_TILE) {
+                const int r = r0 + tid;
+                const int v = r < a.R ? base[r] + cnt[r] : 0;
+                int total;
+                const int excl = block_excl_scan(v, warp_sums, total);
+                if (r < a.R) a.d.rank_offsets[r] = carry + excl;
+                carry += total;
+            }
+            if (tid == 0) {
+                const int64_t G = base[a.R] + cnt[a.R], Tn = base[a.R + 1] + cnt[a.R + 1], SD = carry;
+                const int64_t self_copies = a.src_rank >= 0 ? base[a.src_rank] + cnt[a.src_rank] : 0;
+                const int64_t sent_rows = Tn - (int64_t)acc->self_only;
+                a.d.rank_offsets[a.R] = (int32_t)SD;
+                a.d.group_offsets[G] = (int32_t)Tn;
+                mw_totals tt;
+                tt.T_nonempty = Tn; tt.G = G; tt.total_dest = SD;
+                tt.mw_bytes = sent_rows * a.row_bytes;
+                tt.unicast_bytes = (SD - self_copies) * a.row_bytes;
+                tt.unicast_per_expert_bytes = (int64_t)acc->valid_slots * a.row_bytes;
+                tt.meta_bytes = a.R <= 64 ? 0 : sent_rows * ((a.row_bytes + 4095) / 4096) * (int64_t)(8 * a.W);
+                tt.status = acc->status;
+                tt.reserved = 0;
+                *a.d.totals = tt;
+                mw_acc *next = a.d.acc + ((a.epoch + 1u) & 1u);
+                next->valid_slots = 0; next->self_only = 0; next->status = 0;
+            }
+        }
+    }
+    alive = grid_barrier(a.d.gbar, a.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
+    if (!alive) {
+        if (tid == 0) set_status(&a.d.totals->status, MW_ERR_TIMEOUT);
+        return;
+    }
+
+    // ---- phase C: group ids, send rows, inverse maps, delivery descriptors, table clean-up ----
+    const int Tn = (int)__ldcg(&a.d.totals->T_nonempty), G = (int)__ldcg(&a.d.totals->G);
+    const int SD = (int)__ldcg(&a.d.totals->total_dest);
+    // tails: every index up to T (inclusive for group_offsets) is covered by some thread of the grid
+    for (int u = t; u <= a.T; u += a.ntiles * MW_TILE) {
+        if (u > G) a.d.group_offsets[u] = -1;
+        if (u < a.T) {
+            if (u >= Tn) a.d.mw_row_token[u] = -1;
+            for (int i = 0; i < a.Kd; ++i)
+                if ((int64_t)u * a.Kd + i >= SD) a.d.rank_tokens[(int64_t)u * a.Kd + i] = -1;
+            if (u >= G)
+                for (int w = 0; w < a.W; ++w) a.d.group_mask[(int64_t)u * a.W + w] = 0;
+        }
+    }
+    const int within = group_rank_in_tile(&rank_scratch, a.d.token_leader, tile, nd > 0 ? leader : -1, gcount);
+    if (!active) return;
+    if (nd == 0) { a.d.token_group[t] = -1; a.d.token_mw_row[t] = -1; return; }
+    const int g = __ldcg(a.d.gid_at + leader), goff = __ldcg(a.d.goff_at + leader);
+    const int row = goff + within;
+    a.d.token_group[t] = g;
+    a.d.token_mw_row[t] = row;
+    a.d.mw_row_token[row] = t;
+    a.d.row_ndest[row] = nd;
+    if (leader == t) {
+        a.d.group_offsets[g] = goff;
+#pragma unroll
+        for (int w = 0; w < WT; ++w)
+            if (w < a.W) a.d.group_mask[(int64_t)g * a.W + w] = m[w];
+    }
+    {
+        int i = 0;
+#pragma unroll
+        for (int w = 0; w < WT; ++w)
+            for (uint64_t word = m[w]; word; word &= word - 1) {
+                const int r = w * 64 + __ffsll((long long)word) - 1;
+                const int p = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
+                a.d.row_dest_rank[(int64_t)row * a.Kd + i] = r;
+                a.d.row_dest_pos[(int64_t)row * a.Kd + i] = p;
+                const int at = __ldcg(a.d.rank_offsets + r) + p;
+                a.d.rank_tokens[at] = t;
+                a.d.uc_row_rank[at] = r;
+                ++i;
+            }
+        for (; i < a.Kd; ++i) { a.d.row_dest_rank[(int64_t)row * a.Kd + i] = -1; a.d.row_dest_pos[(int64_t)row * a.Kd + i] = -1; }
+    }
+    a.d.slot_key[slot] = kEmptyKey;
     a.d.slot_leader[slot] = kNoLeader;
     a.d.slot_count[slot] = 0;
 }
@@ -313,9 +704,15 @@ int mw_plan_smem_setup(mw_ctx *ctx)
 {
     const size_t need = tile_smem_bytes(ctx);
     if (need > (size_t)ctx->max_smem_optin) return MW_ERR_INVALID_ARG;
-    if (need > 48 * 1024 &&
-        cudaFuncSetAttribute(k_plan_tile, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)
-        return MW_ERR_CUDA;
+    if (need > 48 * 1024) {
+        const int n = (int)need;
+        if (cudaFuncSetAttribute(k_plan_tile, cudaFuncAttributeMaxDynamicSharedMemorySize, n) != cudaSuccess ||
+            cudaFuncSetAttribute(k_plan_fused<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n) != cudaSuccess ||
+            cudaFuncSetAttribute(k_plan_fused<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n) != cudaSuccess ||
+            cudaFuncSetAttribute(k_plan_fused<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, n) != cudaSuccess ||
+            cudaFuncSetAttribute(k_plan_fused<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, n) != cudaSuccess)
+            return MW_ERR_CUDA;
+    }
     return MW_OK;
 }
 
@@ -332,13 +729,28 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.epoch = ctx->epoch & 0x3fffffffu;
     a.ticket_base = ctx->tickets_used;
     a.d = ctx->d;
+    a.bar_base = ctx->gbar_arrivals;
     const int blocks = a.ntiles;
+    ctx->planned_T = T;
+    if (ctx->coop_ok && blocks <= ctx->sm_count && !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS)) {
+        // one cooperative launch: all tiles resident, phases separated by grid barriers
+        void *params[] = {&a};
+        const void *fn = ctx->W <= 1 ? (const void *)k_plan_fused<1>
+                       : ctx->W <= 2 ? (const void *)k_plan_fused<2>
+                       : ctx->W <= 4 ? (const void *)k_plan_fused<4> : (const void *)k_plan_fused<16>;
+        const cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(blocks), dim3(MW_TILE), params, tile_smem_bytes(ctx), st);
+        if (e == cudaSuccess) {
+            ctx->gbar_arrivals += 2u * (uint32_t)blocks;
+            ctx->launches += 1;
+            return MW_OK;
+        }
+        cudaGetLastError();   // could not be placed (e.g. SMs partly occupied): take the multi-pass route
+    }
     k_plan_mask<<<blocks, MW_TILE, 0, st>>>(a);
     k_plan_tile<<<blocks, MW_TILE, tile_smem_bytes(ctx), st>>>(a);
     ctx->tickets_used += (uint32_t)blocks;
     // one extra thread beyond T so that group_offsets[T] is covered
     k_plan_final<<<(T + 1 + MW_TILE - 1) / MW_TILE, MW_TILE, 0, st>>>(a);
     ctx->launches += 3;
-    ctx->planned_T = T;
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
 }
