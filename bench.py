@@ -308,7 +308,7 @@ def run_cuda(args):
     B, T = s.row_bytes, s.T
     ids = torch.from_numpy(inp.topk_ids).cuda()
     e2r = torch.from_numpy(inp.expert_to_rank).cuda()
-    ctx = mw.Context(s.R, s.E, s.K, T, B, device=local)
+    ctx = mw.Context(s.R, s.E, s.K, T, B, device=local, flags=args.flags)
     ctx.mw_plan(ids, e2r, T)
     tot = ctx.mw_get_totals()
     assert tot["status"] == 0, tot
@@ -446,6 +446,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the decode-latency and bytes-saved extras")
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="MW_FLAG_* bits for the timed context")
     ap.add_argument("--kernels-only", action="store_true",
                     help="only the device-timed steps (for profiler runs): no end-to-end leg, extras or CPU baseline")
     args = ap.parse_args()

@@ -73,6 +73,11 @@ extern "C" {
 #define MW_FLAG_HOST_STAGING   0x1u  /* allocate device staging so mw_dispatch_host can be used */
 #define MW_FLAG_PLAN_MULTIPASS 0x2u  /* always take the tiled multi-kernel plan, even for small T */
 #define MW_FLAG_COPY_LDST      0x4u  /* row copies by 16-byte register loads/stores, not bulk copies */
+#define MW_FLAG_PLAN_COOPERATIVE 0x8u /* launch the fused plan through the cooperative-launch API (the   */
+                                      /* driver then guarantees that all its blocks are resident; costs   */
+                                      /* about 20 us of host time per plan); default is an ordinary launch */
+#define MW_FLAG_NO_OVERLAP     0x10u /* do not let a kernel's start-up overlap the previous kernel's tail */
+#define MW_FLAG_COPY_REG_STORE 0x20u /* fan rows out with 16-byte register stores instead of shared->global bulk copies */
 
 #define MW_MAX_RANKS   1024
 #define MW_MAX_TOPK    64

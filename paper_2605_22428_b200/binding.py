@@ -26,6 +26,9 @@ MW_LAYOUT_UNICAST = 1
 MW_FLAG_HOST_STAGING = 0x1
 MW_FLAG_PLAN_MULTIPASS = 0x2
 MW_FLAG_COPY_LDST = 0x4
+MW_FLAG_PLAN_COOPERATIVE = 0x8
+MW_FLAG_NO_OVERLAP = 0x10
+MW_FLAG_COPY_REG_STORE = 0x20
 
 EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch",
            "mw_allgather_pack", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",

@@ -48,13 +48,16 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.row_ndest = k.take<int32_t>(Tm);
     d.row_dest_rank = k.take<int32_t>(Tm * Kd);
     d.row_dest_pos = k.take<int32_t>(Tm * Kd);
+    d.row_dest_flat = k.take<int32_t>(Tm * Kd);
     d.uc_row_rank = k.take<int32_t>(Tm * Kd);
+    d.uc_row_pos = k.take<int32_t>(Tm * Kd);
     d.slot_key = k.take<unsigned long long>((size_t)c->HS);
     d.slot_leader = k.take<int32_t>((size_t)c->HS);
     d.slot_count = k.take<int32_t>((size_t)c->HS);
     d.tile_state = k.take<unsigned long long>((size_t)c->max_tiles * (size_t)c->NC);
     d.ticket = k.take<unsigned int>(1);
     d.gbar = k.take<unsigned int>(1);
+    d.copy_ctr = k.take<unsigned int>(2);
     d.acc = k.take<mw_acc>(2);
     if (c->cfg.flags & MW_FLAG_HOST_STAGING) {
         const size_t B = (size_t)c->cfg.row_bytes;
@@ -87,6 +90,7 @@ mw_copy_args base_args(mw_ctx *ctx)
     a.R = ctx->cfg.R;
     a.rank_offsets = ctx->d.rank_offsets;
     a.uc_row_rank = ctx->d.uc_row_rank;
+    a.uc_row_pos = ctx->d.uc_row_pos;
     a.totals = ctx->d.totals;
     return a;
 }
@@ -191,13 +195,15 @@ int mw_pack(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send
         a.src_index = ctx->d.mw_row_token;
         a.host_rows = ctx->planned_T;          // estimate for the chunking heuristic
     } else {
-        // one pass over the tokens: each hidden row is read once and written to its |D_t| unicast slots
+        // one pass over the non-empty tokens: each hidden row is read once and written to its |D_t| unicast slots
         a.mode = MW_CP_SCATTER;
-        a.rows_from = 0;
-        a.host_rows = ctx->planned_T;
-        a.ndst = ctx->d.token_ndest;
-        a.d_rank = ctx->d.dest_rank;
-        a.d_pos = ctx->d.dest_pos;
+        a.rows_from = 1;
+        a.host_rows = ctx->planned_T;          // estimate for the chunking heuristic
+        a.src_index = ctx->d.mw_row_token;
+        a.ndst = ctx->d.row_ndest;
+        a.d_rank = ctx->d.row_dest_rank;
+        a.d_pos = ctx->d.row_dest_pos;
+        a.d_flat = ctx->d.row_dest_flat;
         a.dst_stride = 0;
     }
     return mw_copy_launch(ctx, a, as_stream(stream));
@@ -222,6 +228,7 @@ int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_base, i
         a.ndst = ctx->d.row_ndest;
         a.d_rank = ctx->d.row_dest_rank;
         a.d_pos = ctx->d.row_dest_pos;
+        a.d_flat = ctx->d.row_dest_flat;
         a.host_rows = ctx->planned_T;          // estimate for the chunking heuristic
     } else {
         a.mode = MW_CP_DELIVER_UC;

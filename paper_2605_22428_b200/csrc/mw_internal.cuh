@@ -34,13 +34,16 @@ struct mw_dev {
     int32_t *row_ndest;      // [Tm]      |D| of the token in MultiWrite send row j
     int32_t *row_dest_rank;  // [Tm, Kd]  destination ranks of send row j
     int32_t *row_dest_pos;   // [Tm, Kd]  slots of send row j
+    int32_t *row_dest_flat;  // [Tm, Kd]  row of the compact receive area for each destination of send row j, -1 pad
     int32_t *uc_row_rank;    // [Tm * Kd] rank of every unicast send row
+    int32_t *uc_row_pos;     // [Tm * Kd] slot of every unicast send row inside its rank's region
     // scratch
     unsigned long long *slot_key;                  // [HS] open-addressed table keyed by bitmap: (hash tag, first token)
     int32_t *slot_leader, *slot_count;             // [HS] smallest token index / number of tokens with that bitmap
     unsigned long long *tile_state;                // [max_tiles, NC] look-back records
     unsigned int *ticket;                          // tile ticket counter
     unsigned int *gbar;                            // arrival counter of the fused plan's grid barriers
+    unsigned int *copy_ctr;                        // [2] work-ticket and finished-warp counters of the copy kernels
     mw_acc *acc;                                   // [2]
 };
 
@@ -62,6 +65,30 @@ struct mw_ctx {
     uint8_t *st_x, *st_send, *st_recv;
     int64_t st_recv_rows;
 };
+
+// Ordinary launch; with `overlap` the kernel's blocks may be scheduled while the previous kernel of
+// the stream drains (programmatic dependent launch).  Such a kernel must execute
+// grid_dependency_wait() before it touches global memory that an earlier kernel reads or writes.
+template <class... KArgs, class... Args>
+inline cudaError_t mw_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool overlap,
+                             Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+#ifdef __CUDACC__
+// Blocks until every kernel this launch depends on has completed and its writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Allows the next kernel of the stream to start being scheduled.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
 
 // ---- plan (mw_plan.cu) ----
 int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t st);
@@ -91,13 +118,18 @@ struct mw_copy_args {
     int32_t chunk_bytes;       // bytes moved per work item (multiple of 16)
     int32_t chunks_per_row;
     int stages;                // bulk-copy pipeline depth per warp
+    int batch;                 // consecutive items claimed per work ticket
+    int keep_in_l2;            // destination rows are read again soon: do not mark them evict-first
+    unsigned int *work_ctr;    // [2] ticket counter, finished-warp counter (both zero between launches)
     int Kd, R, dst_begin, dst_count;
     const int32_t *src_index;  // PACK_MW: mw_row_token
     const int32_t *ndst;       // SCATTER: destinations per row
     const int32_t *d_rank;     // SCATTER: [rows, Kd]
     const int32_t *d_pos;      // SCATTER: [rows, Kd]
+    const int32_t *d_flat;     // SCATTER, compact destination: [rows, Kd] destination row, -1 pad
     const int32_t *rank_offsets;
     const int32_t *uc_row_rank;
+    const int32_t *uc_row_pos;
     mw_totals *totals;         // device accounting (row counts, status)
 };
 

@@ -395,11 +395,14 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
         const int r = a.d.dest_rank[(int64_t)t * a.Kd + i], p = a.d.dest_pos[(int64_t)t * a.Kd + i];
         a.d.row_dest_rank[(int64_t)row * a.Kd + i] = r;
         a.d.row_dest_pos[(int64_t)row * a.Kd + i] = p;
+        int at = -1;
         if (r >= 0) {
-            const int at = a.d.rank_offsets[r] + p;
+            at = a.d.rank_offsets[r] + p;
             a.d.rank_tokens[at] = t;
             a.d.uc_row_rank[at] = r;
+            a.d.uc_row_pos[at] = p;
         }
+        a.d.row_dest_flat[(int64_t)row * a.Kd + i] = at;
     }
     // leave the bitmap table empty for the next plan
     const int slot = a.d.token_slot[t];
@@ -426,6 +429,11 @@ __device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p)
 __device__ bool grid_barrier(unsigned int *counter, unsigned int target, bool alive, int *status)
 {
     __shared__ int s_alive;
+    if (gridDim.x == 1) {          // a single tile: block-level ordering is all that is needed
+        if (threadIdx.x == 0) atomicAdd(counter, 1u);
+        __syncthreads();
+        return alive;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -460,6 +468,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     const int t = tile * MW_TILE + tid;
     const bool active = t < a.T;
     mw_acc *acc = a.d.acc + (a.epoch & 1u);
+    grid_launch_dependents();      // the pack kernel may set itself up while the plan runs
 
     // ---- phase A: bitmap (Section 4.1: bit r set <=> rank r is a target) and the bitmap table ----
     uint64_t m[WT];
@@ -685,11 +694,17 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                 a.d.row_dest_rank[(int64_t)row * a.Kd + i] = r;
                 a.d.row_dest_pos[(int64_t)row * a.Kd + i] = p;
                 const int at = __ldcg(a.d.rank_offsets + r) + p;
+                a.d.row_dest_flat[(int64_t)row * a.Kd + i] = at;
                 a.d.rank_tokens[at] = t;
                 a.d.uc_row_rank[at] = r;
+                a.d.uc_row_pos[at] = p;
                 ++i;
             }
-        for (; i < a.Kd; ++i) { a.d.row_dest_rank[(int64_t)row * a.Kd + i] = -1; a.d.row_dest_pos[(int64_t)row * a.Kd + i] = -1; }
+        for (; i < a.Kd; ++i) {
+            a.d.row_dest_rank[(int64_t)row * a.Kd + i] = -1;
+            a.d.row_dest_pos[(int64_t)row * a.Kd + i] = -1;
+            a.d.row_dest_flat[(int64_t)row * a.Kd + i] = -1;
+        }
     }
     a.d.slot_key[slot] = kEmptyKey;
     a.d.slot_leader[slot] = kNoLeader;
@@ -732,19 +747,31 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.bar_base = ctx->gbar_arrivals;
     const int blocks = a.ntiles;
     ctx->planned_T = T;
-    if (ctx->coop_ok && blocks <= ctx->sm_count && !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS)) {
-        // one cooperative launch: all tiles resident, phases separated by grid barriers
-        void *params[] = {&a};
-        const void *fn = ctx->W <= 1 ? (const void *)k_plan_fused<1>
-                       : ctx->W <= 2 ? (const void *)k_plan_fused<2>
-                       : ctx->W <= 4 ? (const void *)k_plan_fused<4> : (const void *)k_plan_fused<16>;
-        const cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(blocks), dim3(MW_TILE), params, tile_smem_bytes(ctx), st);
+    if (blocks <= ctx->sm_count && !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS)) {
+        // One launch, at most one block per SM, phases separated by grid barriers.  The blocks wait for
+        // one another, so all of them must become resident: an ordinary launch achieves that as soon
+        // as earlier kernels of the stream have drained (the grid never exceeds the SM count and needs
+        // a fraction of an SM each); should other work keep SMs occupied for about a second, the
+        // barrier gives up with MW_ERR_TIMEOUT instead of hanging.  MW_FLAG_PLAN_COOPERATIVE asks the
+        // driver for the residency guarantee instead, at the price of a much slower launch call.
+        // The plan is not launched as a programmatic dependent of the previous kernel: measured on
+        // B200 that costs about 30 us per step, while the pack kernel that follows does overlap its
+        // start-up with the plan.
+        cudaError_t e;
+        void (*fn)(PlanArgs) = ctx->W <= 1 ? k_plan_fused<1> : ctx->W <= 2 ? k_plan_fused<2>
+                             : ctx->W <= 4 ? k_plan_fused<4> : k_plan_fused<16>;
+        if ((ctx->cfg.flags & MW_FLAG_PLAN_COOPERATIVE) && ctx->coop_ok) {
+            void *params[] = {&a};
+            e = cudaLaunchCooperativeKernel((const void *)fn, dim3(blocks), dim3(MW_TILE), params, tile_smem_bytes(ctx), st);
+        } else {
+            e = mw_launch(fn, dim3(blocks), dim3(MW_TILE), tile_smem_bytes(ctx), st, false, a);
+        }
         if (e == cudaSuccess) {
             ctx->gbar_arrivals += 2u * (uint32_t)blocks;
             ctx->launches += 1;
             return MW_OK;
         }
-        cudaGetLastError();   // could not be placed (e.g. SMs partly occupied): take the multi-pass route
+        cudaGetLastError();   // the launch was refused: take the multi-pass route
     }
     k_plan_mask<<<blocks, MW_TILE, 0, st>>>(a);
     k_plan_tile<<<blocks, MW_TILE, tile_smem_bytes(ctx), st>>>(a);

@@ -49,6 +49,17 @@ def test_register_copy_variant_matches(cfg):
     run_dispatch(inp, flags=mw.MW_FLAG_COPY_LDST)
 
 
+@pytest.mark.parametrize("flags", [mw.MW_FLAG_PLAN_MULTIPASS, mw.MW_FLAG_PLAN_COOPERATIVE, mw.MW_FLAG_NO_OVERLAP,
+                                   mw.MW_FLAG_COPY_REG_STORE,
+                                   mw.MW_FLAG_PLAN_MULTIPASS | mw.MW_FLAG_COPY_LDST | mw.MW_FLAG_NO_OVERLAP])
+def test_launch_and_plan_variants_match(flags):
+    """The multi-pass plan, the cooperative-launch plan, the non-overlapped launches and the other copy
+    kernels give the same bits."""
+    run_dispatch(wl.make_dispatch("large_ep", 100, H=264), flags=flags, repeats=2)
+    run_dispatch(wl.make_random_dispatch(31, T=1025, K=2, E=12, R=6, H=24, pad_fraction=0.1), flags=flags)
+    run_dispatch(wl.make_dispatch("decode", H=64), flags=flags)
+
+
 # ---- edge cases ------------------------------------------------------------------------------------
 @pytest.mark.parametrize("R", [1, 2, 63, 64, 65, 128, 129, 256, 1000, 1024])
 def test_rank_word_boundaries(R):
