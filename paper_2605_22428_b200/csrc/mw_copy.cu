@@ -261,7 +261,9 @@ struct TicketSource {
     __device__ __forceinline__ void start(unsigned int *t, int64_t n, int b, int64_t first_item)
     {
         ticket = t; items = n; batch = b; base = first_item; cur = cur_end = 0;
-        pending = atomicAdd(ticket, 1u);
+        pending = 0;
+        if (n > first_item) pending = atomicAdd(ticket, 1u);   // small launches are fully covered by the static part
+        else items = 0;
     }
     // Next item of this warp, or -1 when the work list is exhausted (stays -1 afterwards).
     __device__ __forceinline__ int64_t next()
@@ -277,9 +279,9 @@ struct TicketSource {
     }
 };
 
-__device__ __forceinline__ void tickets_finish(const mw_copy_args &a, int lane, unsigned total_warps)
+__device__ __forceinline__ void tickets_finish(const mw_copy_args &a, int lane, unsigned total_warps, bool used)
 {
-    if (lane == 0) {
+    if (lane == 0 && used) {
         __threadfence();
         if (atomicAdd(a.work_ctr + 1, 1u) == total_warps - 1u) {
             a.work_ctr[0] = 0;
@@ -331,11 +333,12 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_stage(const __gr
         bulk_load(stages + (size_t)s * stage_stride, src_row_with(a, g.row, index) + g.off, g.bytes, bar + s);
     };
 
-    // first loads: item (global warp index * npro + lane) goes to stage `lane`, issued by that lane
+    // first loads: item (lane * warps of the grid + this warp) goes to stage `lane`, issued by that lane, so a
+    // small launch spreads over all warps and a large one starts with every pipeline full
     const int npro = nst;
-    const int64_t gw = (int64_t)blockIdx.x * nwarps + warp;
+    const int64_t gw = (int64_t)warp * gridDim.x + blockIdx.x;
     if (lane < nst) {
-        const int64_t it = lane < npro ? gw * npro + lane : -1;
+        const int64_t it = lane < npro ? (int64_t)lane * gridDim.x * nwarps + gw : -1;
         const bool has = it >= 0 && it < items;
         held[lane] = has ? it : -1;
         if (has) issue_load(it, src_is_indexed(a) ? a.src_index[it / a.chunks_per_row] : 0, lane);
@@ -411,7 +414,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_stage(const __gr
         for (int m = n + 1; m < n + nst; ++m)
             if (held[m % nst] >= 0) mbar_wait(bar + (m % nst), (uint32_t)(m / nst) & 1u);
     }
-    tickets_finish(a, lane, (unsigned)(gridDim.x * nwarps));
+    tickets_finish(a, lane, (unsigned)(gridDim.x * nwarps), items > (int64_t)gridDim.x * nwarps * npro);
 }
 
 // ---- bulk-copy loads, bulk-copy stores ------------------------------------------------------
@@ -444,11 +447,12 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_bulk(const __gri
         bulk_load(stages + (size_t)s * stage_stride, src_row_with(a, g.row, index) + g.off, g.bytes, bar + s);
     };
 
-    // first loads: item (global warp index * npro + lane) goes to stage `lane`, issued by that lane
+    // first loads: item (lane * warps of the grid + this warp) goes to stage `lane`, issued by that lane, so a
+    // small launch spreads over all warps and a large one starts with every pipeline full
     const int npro = nst - 1;
-    const int64_t gw = (int64_t)blockIdx.x * nwarps + warp;
+    const int64_t gw = (int64_t)warp * gridDim.x + blockIdx.x;
     if (lane < nst) {
-        const int64_t it = lane < npro ? gw * npro + lane : -1;
+        const int64_t it = lane < npro ? (int64_t)lane * gridDim.x * nwarps + gw : -1;
         const bool has = it >= 0 && it < items;
         held[lane] = has ? it : -1;
         if (has) issue_load(it, src_is_indexed(a) ? a.src_index[it / a.chunks_per_row] : 0, lane);
@@ -507,7 +511,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_bulk(const __gri
             if (held[m % nst] >= 0) mbar_wait(bar + (m % nst), (uint32_t)(m / nst) & 1u);
     }
     bulk_wait_all();
-    tickets_finish(a, lane, (unsigned)(gridDim.x * nwarps));
+    tickets_finish(a, lane, (unsigned)(gridDim.x * nwarps), items > (int64_t)gridDim.x * nwarps * npro);
 }
 
 // ---- register copies, no staging ---------------------------------------------------------------

@@ -1,0 +1,76 @@
+"""The pins must bite: plausible mistakes planted in a *copy* of the oracle's C source (on the CPU;
+nothing here touches the GPU path) have to make at least one pin fail."""
+import ctypes
+import os
+import subprocess
+
+import pytest
+
+import test_oracle_pins as pins
+from oracle import mwo
+from paper_2605_22428_b200 import workloads as wl
+
+SRC = os.path.join(os.path.dirname(mwo.__file__), "mwo.c")
+
+MUTATIONS = {
+    "bit index taken modulo 32": ("(uint64_t)1 << (r % 64)", "(uint64_t)1 << (r % 32)"),
+    "always word 0": ("m[r / 64] |=", "m[0] |="),
+    "padding treated as an error": ("if (id == -1) continue;                         /* padding slot            */", ""),
+    "slot of the previous row": ("dest_pos[(int64_t)t * Kd + i] = rank_seen[r];",
+                                 "dest_pos[(int64_t)t * Kd + i] = rank_seen[r] > 0 ? rank_seen[r] - 1 : 0;"),
+    "rank offsets shifted": ("rank_offsets[r + 1] = rank_offsets[r] + rank_seen[r];",
+                             "rank_offsets[r + 1] = rank_offsets[r] + rank_seen[r] - (r == 0 && rank_seen[r] > 0);"),
+    "groups compared on the first word only": ("if (memcmp(group_mask + g * W, m, (size_t)W * sizeof(uint64_t)) == 0) break;",
+                                               "if (memcmp(group_mask + g * W, m, sizeof(uint64_t)) == 0) break;"),
+    "member order reversed in a group": ("int32_t row = group_offsets[g] + group_count[g]++;",
+                                         "int32_t row = group_offsets[g + 1] - 1 - group_count[g]++;"),
+    "deliver reads the wrong send row": ("send_mw + j * row_bytes, (size_t)row_bytes);\n        }\n    }\n}",
+                                         "send_mw + (T_nonempty - 1 - j) * row_bytes, (size_t)row_bytes);\n        }\n    }\n}"),
+    "unicast bytes count rows, not copies": ("totals->unicast_bytes = sent_copies * row_bytes;", "totals->unicast_bytes = sent_rows * row_bytes;"),
+    "per-expert bytes deduplicated": ("++valid_slots;", "if (!(m[r / 64] >> (r % 64) & 1)) ++valid_slots;"),
+    "metadata: one word instead of W": ("(int64_t)(8 * W);", "(int64_t)(8);"),
+    "self copy counted as transmitted": ("if (src_rank >= 0 && (token_mask[(int64_t)t * W + src_rank / 64] >> (src_rank % 64) & 1)) --nd;", ""),
+    "allgather transmits the self copy": ("if (dst_begin + d == i) continue;\n                memcpy(send_buf", "memcpy(send_buf"),
+    "allgather unicast counts R copies": ("totals->unicast_bytes = (int64_t)R * (R - 1) * shard_bytes;", "totals->unicast_bytes = (int64_t)R * R * shard_bytes;"),
+    "allgather shards concatenated in reverse": ("memcpy(recv_base + d * stride + (int64_t)i * shard_bytes,\n                       send_buf + (int64_t)i * shard_bytes",
+                                                 "memcpy(recv_base + d * stride + (int64_t)(R - 1 - i) * shard_bytes,\n                       send_buf + (int64_t)i * shard_bytes"),
+}
+
+
+def run_pins():
+    """A fast subset of the pins; raises AssertionError when the oracle is wrong."""
+    for seed, (R, E, K) in enumerate([(3, 6, 2), (8, 32, 4), (9, 9, 3), (65, 130, 4), (2, 8, 5)]):
+        inp = wl.make_random_dispatch(seed, T=29, K=K, E=E, R=R, H=8, pad_fraction=0.15 if seed % 2 else 0.0)
+        pins.check_against_brute_force(inp, R)
+    pins.test_brute_force_with_padding_duplicates_and_invalid_ids()
+    pins.test_brute_force_source_inside_domain()
+    pins.test_groups_differing_only_in_a_high_word()
+    pins.test_paper_constants()
+    pins.test_identical_and_all_distinct_tokens()
+    for layout in (0, 1):
+        pins.test_allgather_is_concatenate(layout, 5, 48, 1, 3)
+        pins.test_allgather_is_concatenate(layout, 8, 64, 0, 8)
+    pins.test_allgather_saved_closed_form_and_paper_example()
+
+
+def test_unmutated_oracle_passes_the_subset():
+    run_pins()
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_planted_mistake_is_caught(name, tmp_path, monkeypatch):
+    old, new = MUTATIONS[name]
+    text = open(SRC).read()
+    assert text.count(old) >= 1, f"mutation anchor not found: {name}"
+    mutated = tmp_path / "mwo_mut.c"
+    mutated.write_text(text.replace(old, new, 1))
+    lib_path = tmp_path / "libmwo_mut.so"
+    subprocess.check_call(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-w", "-o", str(lib_path), str(mutated)])
+    lib = ctypes.CDLL(str(lib_path))
+    lib.mwo_plan.restype = ctypes.c_int
+    lib.mwo_allgather.restype = ctypes.c_int
+    for fn in ("mwo_pack_mw", "mwo_pack_uc", "mwo_deliver_mw", "mwo_deliver_uc", "mwo_deliver_definition"):
+        getattr(lib, fn).restype = None
+    monkeypatch.setattr(mwo, "_lib", lib)
+    with pytest.raises(AssertionError):
+        run_pins()

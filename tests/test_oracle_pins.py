@@ -157,6 +157,17 @@ def test_brute_force_with_padding_duplicates_and_invalid_ids():
     check_against_brute_force(inp, 5)
 
 
+def test_groups_differing_only_in_a_high_word():
+    """Tokens that share the first 64 ranks' bits but differ above rank 63 are different groups."""
+    R = 130
+    inp = wl.make_random_dispatch(1, T=12, K=2, E=R, R=R, H=8)
+    inp.expert_to_rank = np.arange(R, dtype=np.int32)
+    inp.topk_ids = np.array([[0, 64], [0, 65], [0, 64], [0, 129], [0, 128], [0, 0], [0, 129], [5, 64], [0, 65],
+                             [64, 0], [128, 0], [0, -1]], np.int32)
+    p, bf = check_against_brute_force(inp, R)
+    assert bf["G"] == 6 and list(p.token_group) == [0, 1, 0, 2, 3, 4, 2, 5, 1, 0, 3, 4]
+
+
 def test_brute_force_source_inside_domain():
     inp = wl.make_random_dispatch(11, T=40, K=3, E=16, R=6, H=8)
     p, _ = check_against_brute_force(inp, 6, src_rank=2)
