@@ -49,8 +49,6 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.row_dest_rank = k.take<int32_t>(Tm * Kd);
     d.row_dest_pos = k.take<int32_t>(Tm * Kd);
     d.row_dest_flat = k.take<int32_t>(Tm * Kd);
-    d.uc_row_rank = k.take<int32_t>(Tm * Kd);
-    d.uc_row_pos = k.take<int32_t>(Tm * Kd);
     d.slot_key = k.take<unsigned long long>((size_t)c->HS);
     d.slot_leader = k.take<int32_t>((size_t)c->HS);
     d.slot_count = k.take<int32_t>((size_t)c->HS);
@@ -89,8 +87,7 @@ mw_copy_args base_args(mw_ctx *ctx)
     a.Kd = ctx->Kd;
     a.R = ctx->cfg.R;
     a.rank_offsets = ctx->d.rank_offsets;
-    a.uc_row_rank = ctx->d.uc_row_rank;
-    a.uc_row_pos = ctx->d.uc_row_pos;
+    a.d_stride = ctx->cfg.max_tokens;
     a.totals = ctx->d.totals;
     return a;
 }

@@ -155,12 +155,12 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
         return a.dst + row * a.row_bytes;
     case MW_CP_SCATTER: {
         if (a.dst_stride) {
-            const int r = a.d_rank[row * a.Kd + q], p = a.d_pos[row * a.Kd + q];
+            const int r = a.d_rank[q * a.d_stride + row], p = a.d_pos[q * a.d_stride + row];
             if (r < 0) return nullptr;
             if (p >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
             return a.dst + (int64_t)r * a.dst_stride + (int64_t)p * a.row_bytes;
         }
-        const int64_t at = a.d_flat[row * a.Kd + q];
+        const int64_t at = a.d_flat[q * a.d_stride + row];
         if (at < 0) return nullptr;
         if (at >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
         return a.dst + at * a.row_bytes;
@@ -170,10 +170,15 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
             if (row >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
             return a.dst + row * a.row_bytes;
         }
-        const int r = a.uc_row_rank[row];
-        const int64_t p = a.uc_row_pos[row];
+        // rank of unicast row `row`: the last r with rank_offsets[r] <= row (binary search, R + 1 entries)
+        int lo = 0, hi = a.R;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (a.rank_offsets[mid] <= row) lo = mid; else hi = mid;
+        }
+        const int64_t p = row - a.rank_offsets[lo];
         if (p >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
-        return a.dst + (int64_t)r * a.dst_stride + p * a.row_bytes;
+        return a.dst + (int64_t)lo * a.dst_stride + p * a.row_bytes;
     }
     case MW_CP_AG_DELIVER_MW: return a.dst + (int64_t)q * a.dst_stride + row * a.row_bytes;
     case MW_CP_AG_PACK_UC:
@@ -208,11 +213,9 @@ __device__ __forceinline__ RawDesc fetch_raw(const mw_copy_args &a, int64_t row,
     if (a.mode == MW_CP_SCATTER) {
         d.n = a.ndst[row];
         if (lane < a.Kd) {
-            if (a.dst_stride) { d.x = a.d_rank[row * a.Kd + lane]; d.y = a.d_pos[row * a.Kd + lane]; }
-            else d.x = a.d_flat[row * a.Kd + lane];
+            if (a.dst_stride) { d.x = a.d_rank[lane * a.d_stride + row]; d.y = a.d_pos[lane * a.d_stride + row]; }
+            else d.x = a.d_flat[lane * a.d_stride + row];
         }
-    } else if (a.mode == MW_CP_DELIVER_UC && a.dst_stride) {
-        d.x = a.uc_row_rank[row]; d.y = a.uc_row_pos[row];
     }
     return d;
 }
@@ -233,10 +236,7 @@ __device__ __forceinline__ uint8_t *resolve_dst(const mw_copy_args &a, int64_t r
     }
     case MW_CP_DELIVER_UC:
         *nd = 1;
-        if (lane != 0) return nullptr;
-        if (!a.dst_stride) return dst_row(a, row, 0);
-        if (d.y >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
-        return a.dst + (int64_t)d.x * a.dst_stride + (int64_t)d.y * a.row_bytes;
+        return lane == 0 ? dst_row(a, row, 0) : nullptr;
     default:
         *nd = n_dst(a, row);          // no load involved in the remaining modes
         return lane < *nd ? dst_row(a, row, lane) : nullptr;

@@ -32,11 +32,9 @@ struct mw_dev {
     int32_t *gid_at;         // [Tm]      group id, stored at the leader's index
     int32_t *goff_at;        // [Tm]      group offset, stored at the leader's index
     int32_t *row_ndest;      // [Tm]      |D| of the token in MultiWrite send row j
-    int32_t *row_dest_rank;  // [Tm, Kd]  destination ranks of send row j
-    int32_t *row_dest_pos;   // [Tm, Kd]  slots of send row j
-    int32_t *row_dest_flat;  // [Tm, Kd]  row of the compact receive area for each destination of send row j, -1 pad
-    int32_t *uc_row_rank;    // [Tm * Kd] rank of every unicast send row
-    int32_t *uc_row_pos;     // [Tm * Kd] slot of every unicast send row inside its rank's region
+    int32_t *row_dest_rank;  // [Kd, Tm]  destination ranks of send row j (entry i of row j at i * Tm + j)
+    int32_t *row_dest_pos;   // [Kd, Tm]  slots of send row j
+    int32_t *row_dest_flat;  // [Kd, Tm]  row of the compact receive area for each destination of send row j, -1 pad
     // scratch
     unsigned long long *slot_key;                  // [HS] open-addressed table keyed by bitmap: (hash tag, first token)
     int32_t *slot_leader, *slot_count;             // [HS] smallest token index / number of tokens with that bitmap
@@ -124,12 +122,11 @@ struct mw_copy_args {
     int Kd, R, dst_begin, dst_count;
     const int32_t *src_index;  // PACK_MW: mw_row_token
     const int32_t *ndst;       // SCATTER: destinations per row
-    const int32_t *d_rank;     // SCATTER: [rows, Kd]
-    const int32_t *d_pos;      // SCATTER: [rows, Kd]
-    const int32_t *d_flat;     // SCATTER, compact destination: [rows, Kd] destination row, -1 pad
+    const int32_t *d_rank;     // SCATTER: [Kd, d_stride] destination ranks, entry i of row j at i * d_stride + j
+    const int32_t *d_pos;      // SCATTER: [Kd, d_stride] slots
+    const int32_t *d_flat;     // SCATTER, compact destination: [Kd, d_stride] destination row, -1 pad
+    int64_t d_stride;          // rows per descriptor plane (max_tokens)
     const int32_t *rank_offsets;
-    const int32_t *uc_row_rank;
-    const int32_t *uc_row_pos;
     mw_totals *totals;         // device accounting (row counts, status)
 };
 

@@ -32,7 +32,7 @@ constexpr int kSpinLimit = 1 << 20;  // look-back polls before a tile gives up (
 
 struct PlanArgs {
     const int32_t *ids, *e2r;
-    int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask;
+    int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask, Tm;
     int64_t row_bytes;
     uint32_t epoch, ticket_base, bar_base;
     mw_dev d;
@@ -393,16 +393,14 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
     }
     for (int i = 0; i < a.Kd; ++i) {
         const int r = a.d.dest_rank[(int64_t)t * a.Kd + i], p = a.d.dest_pos[(int64_t)t * a.Kd + i];
-        a.d.row_dest_rank[(int64_t)row * a.Kd + i] = r;
-        a.d.row_dest_pos[(int64_t)row * a.Kd + i] = p;
+        a.d.row_dest_rank[(int64_t)i * a.Tm + row] = r;
+        a.d.row_dest_pos[(int64_t)i * a.Tm + row] = p;
         int at = -1;
         if (r >= 0) {
             at = a.d.rank_offsets[r] + p;
             a.d.rank_tokens[at] = t;
-            a.d.uc_row_rank[at] = r;
-            a.d.uc_row_pos[at] = p;
         }
-        a.d.row_dest_flat[(int64_t)row * a.Kd + i] = at;
+        a.d.row_dest_flat[(int64_t)i * a.Tm + row] = at;
     }
     // leave the bitmap table empty for the next plan
     const int slot = a.d.token_slot[t];
@@ -423,21 +421,28 @@ __device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p)
     return v;
 }
 
-// All blocks of the (co-resident) grid arrive; a block that is still `alive` then waits until the
-// counter reaches `target`.  Every block always arrives, so the host's running count of arrivals
-// stays exact even after a block has given up.  Returns false for a block that gave up (now or before).
-__device__ bool grid_barrier(unsigned int *counter, unsigned int target, bool alive, int *status)
+// Grid barrier in two halves, so that work which does not depend on the other blocks can run between
+// them.  Every block always arrives, so the host's running count of arrivals stays exact even after a
+// block has given up waiting.
+__device__ __forceinline__ void grid_barrier_arrive(unsigned int *counter)
 {
-    __shared__ int s_alive;
-    if (gridDim.x == 1) {          // a single tile: block-level ordering is all that is needed
-        if (threadIdx.x == 0) atomicAdd(counter, 1u);
-        __syncthreads();
-        return alive;
-    }
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         atomicAdd(counter, 1u);
+    }
+}
+
+// A block that is still `alive` waits until the counter reaches `target`; returns false for a block
+// that gave up (now or before).  With a single block, block-level ordering is all that is needed.
+__device__ bool grid_barrier_wait(unsigned int *counter, unsigned int target, bool alive, int *status)
+{
+    __shared__ int s_alive;
+    if (gridDim.x == 1) {
+        __syncthreads();
+        return alive;
+    }
+    if (threadIdx.x == 0) {
         int ok = alive ? 1 : 0;
         if (ok) {
             int spins = 0;
@@ -451,6 +456,12 @@ __device__ bool grid_barrier(unsigned int *counter, unsigned int target, bool al
     }
     __syncthreads();
     return s_alive != 0;
+}
+
+__device__ __forceinline__ bool grid_barrier(unsigned int *counter, unsigned int target, bool alive, int *status)
+{
+    grid_barrier_arrive(counter);
+    return grid_barrier_wait(counter, target, alive, status);
 }
 
 template <int WT>
@@ -469,6 +480,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     const bool active = t < a.T;
     mw_acc *acc = a.d.acc + (a.epoch & 1u);
     grid_launch_dependents();      // the pack kernel may set itself up while the plan runs
+    for (int i = tid; i < a.R * 8; i += MW_TILE) bits[i] = 0;
 
     // ---- phase A: bitmap (Section 4.1: bit r set <=> rank r is a target) and the bitmap table ----
     uint64_t m[WT];
@@ -536,38 +548,11 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             if (bad) set_status(&acc->status, MW_ERR_BAD_INDEX);
         }
     }
-    for (int i = tid; i < a.R * 8; i += MW_TILE) bits[i] = 0;
-    bool alive = grid_barrier(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
-
-    // ---- phase B: positions inside the tile, tile histogram, look-back over tiles ----
-    int leader = -1, gcount = 0;
-    const int wi = tid >> 5;
-    const uint32_t bit = 1u << (tid & 31);
-    if (alive) {
-        if (nd > 0) { leader = __ldcg(a.d.slot_leader + slot); gcount = __ldcg(a.d.slot_count + slot); }
-        const bool is_leader = nd > 0 && leader == t;
-        if (active) a.d.token_leader[t] = leader;
-        if (nd > 0) {
-#pragma unroll
-            for (int w = 0; w < WT; ++w)
-                for (uint64_t word = m[w]; word; word &= word - 1)
-                    atomicOr(bits + (size_t)(w * 64 + __ffsll((long long)word) - 1) * 8 + wi, bit);
-        }
-        __syncthreads();
-        for (int r = tid; r < a.R; r += MW_TILE) {
-            int run = 0;
-#pragma unroll
-            for (int w8 = 0; w8 < 8; ++w8) { pre[r * 8 + w8] = run; run += __popc(bits[r * 8 + w8]); }
-            cnt[r] = run;
-        }
-        int lead_total, gc_total;
-        const int lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
-        const int gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
-        if (tid == 0) { cnt[a.R] = lead_total; cnt[a.R + 1] = gc_total; }
-        __syncthreads();
-
-        // Decoupled look-back, one thread per counter, eight predecessors fetched per round trip.
-        for (int c = tid; c < a.NC; c += MW_TILE) {
+    // Decoupled look-back over tiles for counters [c0, c1): one thread per counter, eight predecessors
+    // fetched per round trip.  A record is one 64-bit word (epoch, flag, value), so flag and value are
+    // always read together; the epoch makes records of earlier plans invisible.
+    auto look_back = [&](int c0, int c1) {
+        for (int c = c0 + tid; c < c1; c += MW_TILE) {
             const uint32_t mine = (uint32_t)cnt[c];
             volatile unsigned long long *rec = a.d.tile_state + (size_t)tile * a.NC + c;
             uint32_t excl = 0;
@@ -601,25 +586,62 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             }
             base[c] = (int)excl;
         }
-        __syncthreads();
+    };
 
-        if (active) {
-            if (is_leader) { a.d.gid_at[t] = base[a.R] + lead_excl; a.d.goff_at[t] = base[a.R + 1] + gc_excl; }
-            int i = 0;
-            int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
-            if (nd > 0) {
+    // ---- phase B1 (needs only this tile's bitmaps, so it runs between the two halves of the first grid
+    //      barrier and overlaps the barrier's latency): positions inside the tile, rank histogram, look-back ----
+    const int wi = tid >> 5;
+    const uint32_t bit = 1u << (tid & 31);
+    grid_barrier_arrive(a.d.gbar);  // this tile's bitmaps are in the table (also orders the clearing of the bit matrix)
+    if (nd > 0) {
 #pragma unroll
-                for (int w = 0; w < WT; ++w)
-                    for (uint64_t word = m[w]; word; word &= word - 1) {
-                        const int r = w * 64 + __ffsll((long long)word) - 1;
-                        dr[i] = r;
-                        dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
-                        ++i;
-                    }
-            }
-            for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
+        for (int w = 0; w < WT; ++w)
+            for (uint64_t word = m[w]; word; word &= word - 1)
+                atomicOr(bits + (size_t)(w * 64 + __ffsll((long long)word) - 1) * 8 + wi, bit);
+    }
+    __syncthreads();
+    for (int r = tid; r < a.R; r += MW_TILE) {
+        int run = 0;
+#pragma unroll
+        for (int w8 = 0; w8 < 8; ++w8) { pre[r * 8 + w8] = run; run += __popc(bits[r * 8 + w8]); }
+        cnt[r] = run;
+    }
+    __syncthreads();
+    look_back(0, a.R);
+    __syncthreads();
+    if (active) {
+        int i = 0;
+        int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
+        if (nd > 0) {
+#pragma unroll
+            for (int w = 0; w < WT; ++w)
+                for (uint64_t word = m[w]; word; word &= word - 1) {
+                    const int r = w * 64 + __ffsll((long long)word) - 1;
+                    dr[i] = r;
+                    dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
+                    ++i;
+                }
         }
+        for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
+    }
+    bool alive = grid_barrier_wait(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
+
+    // ---- phase B2: leaders and group sizes are final; group ids and offsets ----
+    int leader = -1, gcount = 0;
+    if (alive) {
+        if (nd > 0) { leader = __ldcg(a.d.slot_leader + slot); gcount = __ldcg(a.d.slot_count + slot); }
+        const bool is_leader = nd > 0 && leader == t;
+        if (active) a.d.token_leader[t] = leader;
+        int lead_total, gc_total;
+        const int lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
+        const int gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
+        if (tid == 0) { cnt[a.R] = lead_total; cnt[a.R + 1] = gc_total; }
+        __syncthreads();
+        look_back(a.R, a.R + 2);
+        __syncthreads();
+        if (is_leader) { a.d.gid_at[t] = base[a.R] + lead_excl; a.d.goff_at[t] = base[a.R + 1] + gc_excl; }
         if (tile == a.ntiles - 1) {
+            // this tile's inclusive prefix is the grand total of every counter
             int carry = 0;
             for (int r0 = 0; r0 < a.R; r0 += MW_TILE) {
                 const int r = r0 + tid;
@@ -640,6 +662,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                 tt.mw_bytes = sent_rows * a.row_bytes;
                 tt.unicast_bytes = (SD - self_copies) * a.row_bytes;
                 tt.unicast_per_expert_bytes = (int64_t)acc->valid_slots * a.row_bytes;
+                // Section 6.4: beyond 64 ranks the bitmap travels in the payload, once per 4096-byte packet
                 tt.meta_bytes = a.R <= 64 ? 0 : sent_rows * ((a.row_bytes + 4095) / 4096) * (int64_t)(8 * a.W);
                 tt.status = acc->status;
                 tt.reserved = 0;
@@ -658,6 +681,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     // ---- phase C: group ids, send rows, inverse maps, delivery descriptors, table clean-up ----
     const int Tn = (int)__ldcg(&a.d.totals->T_nonempty), G = (int)__ldcg(&a.d.totals->G);
     const int SD = (int)__ldcg(&a.d.totals->total_dest);
+    if (__ldcg(&a.d.totals->status) == MW_ERR_TIMEOUT) return;      // a look-back gave up somewhere: nothing below can be trusted
     // tails: every index up to T (inclusive for group_offsets) is covered by some thread of the grid
     for (int u = t; u <= a.T; u += a.ntiles * MW_TILE) {
         if (u > G) a.d.group_offsets[u] = -1;
@@ -691,19 +715,17 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             for (uint64_t word = m[w]; word; word &= word - 1) {
                 const int r = w * 64 + __ffsll((long long)word) - 1;
                 const int p = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
-                a.d.row_dest_rank[(int64_t)row * a.Kd + i] = r;
-                a.d.row_dest_pos[(int64_t)row * a.Kd + i] = p;
+                a.d.row_dest_rank[(int64_t)i * a.Tm + row] = r;
+                a.d.row_dest_pos[(int64_t)i * a.Tm + row] = p;
                 const int at = __ldcg(a.d.rank_offsets + r) + p;
-                a.d.row_dest_flat[(int64_t)row * a.Kd + i] = at;
+                a.d.row_dest_flat[(int64_t)i * a.Tm + row] = at;
                 a.d.rank_tokens[at] = t;
-                a.d.uc_row_rank[at] = r;
-                a.d.uc_row_pos[at] = p;
                 ++i;
             }
         for (; i < a.Kd; ++i) {
-            a.d.row_dest_rank[(int64_t)row * a.Kd + i] = -1;
-            a.d.row_dest_pos[(int64_t)row * a.Kd + i] = -1;
-            a.d.row_dest_flat[(int64_t)row * a.Kd + i] = -1;
+            a.d.row_dest_rank[(int64_t)i * a.Tm + row] = -1;
+            a.d.row_dest_pos[(int64_t)i * a.Tm + row] = -1;
+            a.d.row_dest_flat[(int64_t)i * a.Tm + row] = -1;
         }
     }
     a.d.slot_key[slot] = kEmptyKey;
@@ -738,7 +760,7 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.T = T; a.K = ctx->cfg.K; a.E = ctx->cfg.E; a.R = ctx->cfg.R; a.W = ctx->W; a.Kd = ctx->Kd;
     a.src_rank = ctx->cfg.src_rank;
     a.ntiles = T > 0 ? (T + MW_TILE - 1) / MW_TILE : 1;
-    a.NC = ctx->NC; a.hs_mask = ctx->HS - 1;
+    a.NC = ctx->NC; a.hs_mask = ctx->HS - 1; a.Tm = ctx->cfg.max_tokens;
     a.row_bytes = ctx->cfg.row_bytes;
     ctx->epoch += 1;
     a.epoch = ctx->epoch & 0x3fffffffu;

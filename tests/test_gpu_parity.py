@@ -53,8 +53,9 @@ def test_register_copy_variant_matches(cfg):
                                    mw.MW_FLAG_COPY_REG_STORE,
                                    mw.MW_FLAG_PLAN_MULTIPASS | mw.MW_FLAG_COPY_LDST | mw.MW_FLAG_NO_OVERLAP])
 def test_launch_and_plan_variants_match(flags):
-    """The multi-pass plan, the cooperative-launch plan, the non-overlapped launches and the other copy
-    kernels give the same bits."""
+    """The multi-pass plan, the grid plan (ordinary and cooperative launch), the non-overlapped launches
+    and the other copy kernels give the same bits as the defaults."""
+    run_dispatch(wl.make_random_dispatch(41, T=3000, K=1, E=12, R=6, H=16), flags=flags)       # large groups
     run_dispatch(wl.make_dispatch("large_ep", 100, H=264), flags=flags, repeats=2)
     run_dispatch(wl.make_random_dispatch(31, T=1025, K=2, E=12, R=6, H=24, pad_fraction=0.1), flags=flags)
     run_dispatch(wl.make_dispatch("decode", H=64), flags=flags)
