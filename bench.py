@@ -259,6 +259,43 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
     return out
 
 
+def allgather_sweep(mw, wl, torch) -> list:
+    """AllGather pack + deliver over shard sizes 4 KB .. 64 MB at R = 64 (MultiWrite layout).  The full
+    R x R result does not fit in memory for large shards: a window of destination ranks is materialised
+    (the largest power of two whose receive area stays under 8 GB); GB/s counts the bytes actually moved."""
+    R = wl.ALLGATHER_R
+    out = []
+    with mw.Context(R, 8, 2, 16, 32) as ctx:
+        for S in wl.ALLGATHER_SHARD_BYTES:
+            window = R
+            while window > 1 and window * R * S > (8 << 30):
+                window //= 2
+            shards = torch.empty(R * S, dtype=torch.uint8, device="cuda").random_(0, 256)
+            send = torch.empty(R * S, dtype=torch.uint8, device="cuda")
+            recv = torch.empty(window * R * S, dtype=torch.uint8, device="cuda")
+            reps = 20 if S <= (1 << 20) else 5
+
+            def run():
+                ctx.mw_allgather_pack(shards, S, mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, 0, window)
+
+            for _ in range(3):
+                run()
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            torch.cuda.synchronize()
+            for a, b in evs:
+                a.record()
+                run()
+                b.record()
+            torch.cuda.synchronize()
+            us = statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3
+            moved = 2 * R * S + R * S + window * R * S        # pack read+write, deliver read + window copies
+            out.append({"shard_bytes": S, "window_ranks": window, "p50_us": round(us, 1),
+                        "gbs": round(moved / us / 1e3, 1), "l2_resident": bool(moved < (100 << 20))})
+            del shards, send, recv
+            torch.cuda.empty_cache()
+    return out
+
+
 def bytes_saved(wl) -> dict:
     """Transmitted-byte savings of the MultiWrite layout, exact integers from the plan (device side)."""
     import torch
@@ -436,6 +473,7 @@ def run_cuda(args):
         if not args.no_extras:
             line["decode"] = decode_latency(mw, wl, torch)
             line["bytes_saved_pct"] = bytes_saved(wl)
+            line["allgather_r64"] = allgather_sweep(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:
