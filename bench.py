@@ -68,7 +68,7 @@ def recorded_traffic():
 
 def kernel_source_hash() -> str:
     h = hashlib.sha256()
-    for name in ("mw_copy.cu", "mw_internal.cuh"):
+    for name in ("mw_copy.cu",):
         with open(os.path.join(ROOT, "paper_2605_22428_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
@@ -242,7 +242,10 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
             plan()
             dispatch()
 
-        for name, fn in (("plan", plan), ("pack_deliver", dispatch), ("chain", chain)):
+        def one_call():
+            ctx.mw_plan_dispatch(ids, e2r, s.T, x, mw.MW_LAYOUT_MULTIWRITE, send, Tn, recv, 0, SD)
+
+        for name, fn in (("plan", plan), ("pack_deliver", dispatch), ("chain", chain), ("one_call", one_call)):
             for _ in range(50):
                 fn()
             evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
@@ -255,7 +258,9 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
             us = [a.elapsed_time(b) * 1e3 for a, b in evs]
             out[name] = {"p50_us": round(percentile(us, 0.5), 2), "p99_us": round(percentile(us, 0.99), 2)}
     out["launches"] = launches
-    out["note"] = "L2-resident working set (0.9 MB in, 7.3 MB out): judged on latency, not on HBM fraction"
+    out["note"] = ("L2-resident working set (0.9 MB in, 7.3 MB out): judged on latency, not on HBM fraction; chain = "
+                   "mw_plan + mw_dispatch (3 launches), one_call = mw_plan_dispatch (1 launch); each figure includes "
+                   "the host's launch cost through the Python binding")
     return out
 
 

@@ -194,6 +194,19 @@ MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, i
                 void *recv_base, int64_t recv_stride_bytes, int64_t recv_capacity_rows, void *stream);
 
 /*
+ * mw_plan followed by mw_dispatch in one call (same arguments, same results, the context is left
+ * in the same state).  For small batches in the MultiWrite layout (T <= 256, R <= 256, min(K, R)
+ * <= 16: the decode-sized batches of Section 6.3, where the paper finds the replication overhead
+ * to outweigh the savings) the three kernels are replaced by a single launch in which every
+ * block recomputes the plan in shared memory and then moves its share of the rows; larger
+ * batches, the unicast layout and contexts created with a plan or copy variant flag take the
+ * ordinary three-kernel route.
+ */
+MW_API int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
+                            const void *x, int layout, void *send_buf, int64_t send_capacity_rows, void *recv_base,
+                            int64_t recv_stride_bytes, int64_t recv_capacity_rows, mw_plan_view *view, void *stream);
+
+/*
  * AllGather pack + deliver (Section 5.2): R ranks each contribute one shard of shard_bytes;
  * every destination rank ends with shard_0 | shard_1 | ... | shard_{R-1}.  Uses cfg.R only.
  *   shards       device, [R, shard_bytes] contiguous, 16-byte aligned; shard_bytes multiple of 16

@@ -30,7 +30,7 @@ MW_FLAG_PLAN_COOPERATIVE = 0x8
 MW_FLAG_NO_OVERLAP = 0x10
 MW_FLAG_COPY_REG_STORE = 0x20
 
-EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch",
+EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
            "mw_allgather_pack", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
            "mw_strerror")
 
@@ -89,6 +89,7 @@ def lib():
         L.mw_pack.argtypes = [vp, vp, C.c_int, vp, i64, vp]
         L.mw_deliver.argtypes = [vp, C.c_int, vp, vp, i64, i64, vp]
         L.mw_dispatch.argtypes = [vp, vp, C.c_int, vp, i64, vp, i64, i64, vp]
+        L.mw_plan_dispatch.argtypes = [vp, vp, vp, i32, vp, C.c_int, vp, i64, vp, i64, i64, C.POINTER(mw_plan_view), vp]
         L.mw_allgather_pack.argtypes = [vp, vp, i64, C.c_int, vp, vp, i64, i32, i32, C.POINTER(mw_totals), vp]
         L.mw_dispatch_host.argtypes = [vp, vp, vp, vp, i32, C.c_int, vp, i64, vp, C.POINTER(mw_totals), vp]
         L.mw_group_tokens_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -97,7 +98,7 @@ def lib():
         L.mw_kernel_launches.restype = C.c_int64
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:11]:
+        for name in EXPORTS[:12]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -207,6 +208,17 @@ class Context:
                                recv_stride_bytes, recv_capacity_rows, _stream(stream))
         if check and rc != MW_OK:
             raise MwError(rc, "mw_dispatch")
+        return rc
+
+    def mw_plan_dispatch(self, topk_ids, expert_to_rank, T: int, x, layout: int, send_buf, send_capacity_rows: int,
+                         recv, recv_stride_bytes: int, recv_capacity_rows: int, stream=None, check: bool = True) -> int:
+        view = mw_plan_view()
+        rc = lib().mw_plan_dispatch(self._h, _ptr(topk_ids), _ptr(expert_to_rank), T, _ptr(x), layout, _ptr(send_buf),
+                                    send_capacity_rows, _ptr(recv), recv_stride_bytes, recv_capacity_rows,
+                                    C.byref(view), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_plan_dispatch")
+        self.view = view
         return rc
 
     def mw_allgather_pack(self, shards, shard_bytes: int, layout: int, send_buf, recv, recv_stride_bytes: int = 0,

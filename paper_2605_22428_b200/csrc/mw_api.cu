@@ -139,6 +139,7 @@ int mw_create(mw_ctx **out, const mw_config *cfg)
     }
     if (rc == MW_OK) rc = mw_plan_smem_setup(c);
     if (rc == MW_OK) rc = mw_copy_smem_setup(c);
+    if (rc == MW_OK) rc = mw_small_setup(c);
     if (rc != MW_OK) { cudaFree(c->slab); cudaGetLastError(); delete c; return rc; }
     *out = c;
     return MW_OK;
@@ -243,6 +244,32 @@ int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t 
     int rc = mw_pack(ctx, x, layout, send_buf, send_capacity_rows, stream);
     if (rc != MW_OK) return rc;
     return mw_deliver(ctx, layout, send_buf, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
+}
+
+int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x,
+                     int layout, void *send_buf, int64_t send_capacity_rows, void *recv_base, int64_t recv_stride_bytes,
+                     int64_t recv_capacity_rows, mw_plan_view *view, void *stream)
+{
+    if (!ctx || !expert_to_rank || T < 0 || T > ctx->cfg.max_tokens || (T > 0 && !topk_ids) || !x || !send_buf || !recv_base ||
+        send_capacity_rows < 0 || recv_stride_bytes < 0 || recv_capacity_rows < 0 || check_layout(layout))
+        return MW_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
+    if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
+    if (!mw_small_applies(ctx, T, layout)) {
+        const int rc = mw_plan(ctx, topk_ids, expert_to_rank, T, view, stream);
+        if (rc != MW_OK) return rc;
+        return mw_dispatch(ctx, x, layout, send_buf, send_capacity_rows, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
+    }
+    if (view) {
+        const mw_dev &d = ctx->d;
+        view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
+        view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
+        view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
+        view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
+        view->T = T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
+    }
+    return mw_small_launch(ctx, topk_ids, expert_to_rank, T, x, send_buf, send_capacity_rows, recv_base, recv_stride_bytes,
+                           recv_capacity_rows, as_stream(stream));
 }
 
 int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int layout, void *send_buf,

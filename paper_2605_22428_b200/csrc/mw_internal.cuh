@@ -92,6 +92,13 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t st);
 int mw_plan_smem_setup(mw_ctx *ctx);
 
+// ---- single-launch small-batch path (mw_small.cu) ----
+bool mw_small_applies(const mw_ctx *ctx, int32_t T, int layout);
+int mw_small_setup(mw_ctx *ctx);
+int mw_small_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x,
+                    void *send_buf, int64_t send_capacity_rows, void *recv_base, int64_t recv_stride_bytes,
+                    int64_t recv_capacity_rows, cudaStream_t st);
+
 // ---- row copies (mw_copy.cu) ----
 enum mw_copy_mode {
     MW_CP_PACK_MW = 0,      // send[j] = x[mw_row_token[j]]

@@ -57,7 +57,7 @@ def assert_plan_equal(got: dict, p: mwo.Plan, totals: dict):
 
 def run_dispatch(inp, *, layouts=(mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST), strides=("compact", "strided"),
                  flags: int = 0, src_rank: int = -1, max_tokens: int | None = None, check_payload: bool = True,
-                 repeats: int = 1):
+                 repeats: int = 1, one_call: bool = False):
     """Plans and dispatches `inp` on the GPU, checks everything against the oracle, returns (plan, totals)."""
     torch = torch_mod()
     s = inp.shape
@@ -87,8 +87,14 @@ def run_dispatch(inp, *, layouts=(mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST)
                              else mwo.deliver_uc(p, want_send[layout], stride, SENTINEL))
                 send = Guarded(nsend * B)
                 recv = Guarded(len(want_recv))
-                ctx.mw_dispatch(x_d.data_ptr(), layout, send.ptr(), nsend, recv.ptr(), stride, cap)
-                tot2 = ctx.mw_get_totals()
+                if one_call:
+                    # plan + dispatch through the single entry point; the plan it leaves behind must be the same
+                    ctx.mw_plan_dispatch(ids_d, e2r_d, T, x_d.data_ptr(), layout, send.ptr(), nsend, recv.ptr(), stride, cap)
+                    tot2 = ctx.mw_get_totals()
+                    assert_plan_equal(ctx.plan_arrays(T), p, tot2)
+                else:
+                    ctx.mw_dispatch(x_d.data_ptr(), layout, send.ptr(), nsend, recv.ptr(), stride, cap)
+                    tot2 = ctx.mw_get_totals()
                 assert tot2["status"] == p.totals["status"], tot2
                 assert np.array_equal(send.host().reshape(-1, B), want_send[layout]), ("send", layout, mode)
                 assert np.array_equal(recv.host(), want_recv), ("recv", layout, mode)

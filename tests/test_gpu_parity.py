@@ -187,6 +187,68 @@ def test_nan_and_negative_zero_payload_round_trips():
     run_dispatch(inp)
 
 
+# ---- plan + dispatch in one call (single-launch path for small batches) ----------------------------
+@pytest.mark.parametrize("cfg,H", [("decode", None), ("tiny", None), ("decode", 72)])
+def test_one_call_small_batches_match(cfg, H):
+    run_dispatch(wl.make_dispatch(cfg, H=H), one_call=True, repeats=1)
+    run_dispatch(wl.make_dispatch(cfg, 100, H=H), one_call=True)
+
+
+@pytest.mark.parametrize("T", [0, 1, 31, 255, 256, 257, 600])
+def test_one_call_token_counts(T):
+    # up to 256 tokens the single launch is taken, beyond that the three-kernel route: same results
+    inp = wl.make_random_dispatch(T + 11, T=T, K=3, E=40, R=10, H=40, pad_fraction=0.1)
+    run_dispatch(inp, one_call=True, max_tokens=700)
+
+
+def test_one_call_groups_padding_invalid_ids_and_source_rank():
+    same = wl.make_random_dispatch(1, T=200, K=2, E=8, R=4, H=16)            # few, large groups
+    run_dispatch(same, one_call=True)
+    inp = wl.make_random_dispatch(7, T=250, K=4, E=24, R=7, H=16, pad_fraction=0.35, distinct=False)
+    ids = inp.topk_ids.copy()
+    ids[3, :] = -1
+    ids[4, 0] = 24
+    ids[5, 1] = -2
+    inp.topk_ids = ids
+    p, tot = run_dispatch(inp, one_call=True)
+    assert tot["status"] == mw.MW_ERR_BAD_INDEX
+    run_dispatch(wl.make_random_dispatch(11, T=180, K=3, E=16, R=6, H=16), one_call=True, src_rank=2)
+    wide = wl.make_random_dispatch(12, T=256, K=8, E=512, R=256, H=24)       # four bitmap words
+    run_dispatch(wide, one_call=True)
+    big_k = wl.make_random_dispatch(13, T=100, K=20, E=64, R=64, H=16)       # more than 16 destinations: falls back
+    run_dispatch(big_k, one_call=True)
+
+
+def test_one_call_capacity_overflow_is_reported_and_contained():
+    torch = torch_mod()
+    inp = wl.make_random_dispatch(21, T=200, K=3, E=32, R=8, H=16, contiguous_map=True)
+    s = inp.shape
+    B = s.row_bytes
+    p = mwo.plan(inp.topk_ids, inp.expert_to_rank, s.R, B)
+    Tn, SD = p.totals["T_nonempty"], p.totals["total_dest"]
+    ids_d, e2r_d = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    x_d = torch.from_numpy(inp.x.view(np.int16)).cuda()
+    want_send = mwo.pack_mw(p, inp.x)
+    want_recv = mwo.deliver_mw(p, want_send)
+    with mw.Context(s.R, s.E, s.K, s.T, B) as ctx:
+        send, recv = Guarded((Tn - 1) * B), Guarded((SD - 10) * B)
+        ctx.mw_plan_dispatch(ids_d, e2r_d, s.T, x_d, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn - 1, recv.ptr(), 0, SD - 10)
+        assert ctx.mw_get_totals()["status"] == mw.MW_ERR_CAPACITY
+        assert send.guards_intact() and recv.guards_intact()
+        assert np.array_equal(send.host().reshape(-1, B), want_send[:Tn - 1])
+        assert np.array_equal(recv.host(), want_recv[:(SD - 10) * B])
+        send, recv = Guarded(Tn * B), Guarded(SD * B)
+        ctx.mw_plan_dispatch(ids_d, e2r_d, s.T, x_d, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn, recv.ptr(), 0, SD)
+        assert ctx.mw_get_totals()["status"] == 0
+        assert np.array_equal(recv.host(), want_recv)
+        # the plan left behind serves a later separate dispatch
+        recv2 = Guarded(SD * B)
+        ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send.ptr(), recv2.ptr(), 0, SD)
+        assert np.array_equal(recv2.host(), want_recv)
+        assert ctx.mw_plan_dispatch(ids_d, e2r_d, s.T, x_d.data_ptr() + 8, 0, send.ptr(), Tn, recv.ptr(), 0, SD,
+                                    check=False) == mw.MW_ERR_ALIGNMENT
+
+
 # ---- capacity and argument errors ----------------------------------------------------------------
 def test_capacity_overflow_is_reported_and_contained():
     torch = torch_mod()
