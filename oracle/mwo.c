@@ -325,3 +325,86 @@ int mwo_allgather(const uint8_t *shards, int32_t R, int64_t shard_bytes, int lay
     }
     return MWO_OK;
 }
+
+/*
+ * Two-level (relayed) MultiWrite for dispatch: Section 3.2 and Section 4.3.3.
+ *
+ * Ranks are grouped into servers of ranks_per_server consecutive ranks.  The source (src_rank, a
+ * member of the domain) writes directly to destinations inside its own server; for every other
+ * server that holds at least one destination of a token it sends ONE copy to the rank with its own
+ * index inside that server (the "same-index NPU"), which then replicates the row to the destinations
+ * inside its server (Section 3.2; Section 4.1 "Local forwarding table": one copy per distinct next hop;
+ * Section 4.3.3: M is partitioned by next hop).
+ */
+int mwo_next_hop(int32_t r, int32_t src_rank, int32_t ranks_per_server)
+{
+    if (r / ranks_per_server == src_rank / ranks_per_server) return r;          /* same server: direct   */
+    return (r / ranks_per_server) * ranks_per_server + src_rank % ranks_per_server;   /* same-index relay */
+}
+
+typedef struct {
+    int64_t hop_rows;               /* rows written by the source: one per (token, distinct next hop)       */
+    int64_t delivered_rows;         /* rows in the final receive regions (= flat total_dest)                */
+    int64_t direct_bytes;           /* source -> destinations in its own server (own rank excluded)         */
+    int64_t inter_multiwrite_bytes; /* source -> other servers, one copy per server that has a destination  */
+    int64_t inter_unicast_bytes;    /* source -> other servers, one copy per remote destination (baseline)  */
+    int64_t forward_bytes;          /* relays -> destinations in their server (the relay itself excluded)   */
+    int32_t status;
+    int32_t reserved;
+} mwo_relay_totals;
+
+/*
+ * hop_of_expert [E]: next hop of every expert's rank (the table handed to the first-level plan);
+ * entries whose rank is out of range are passed through unchanged so that the plan reports them.
+ */
+void mwo_relay_table(const int32_t *expert_to_rank, int32_t E, int32_t R, int32_t src_rank, int32_t ranks_per_server,
+                     int32_t *hop_of_expert)
+{
+    for (int32_t e = 0; e < E; ++e) {
+        int32_t r = expert_to_rank[e];
+        hop_of_expert[e] = (r < 0 || r >= R) ? r : mwo_next_hop(r, src_rank, ranks_per_server);
+    }
+}
+
+/*
+ * Second level: every row that arrived in hop region h (rows of the first-level plan, token order) is
+ * written to each final destination r of its token whose next hop is h, at the slot the flat plan gives
+ * that (token, rank) pair.  Also the byte accounting per link class.
+ *   hop_*   : first-level plan (computed by mwo_plan on hop_of_expert)
+ *   flat_*  : flat plan (computed by mwo_plan on expert_to_rank)
+ *   hop_buf : compact first-level receive area [hop_rows, row_bytes]
+ */
+void mwo_relay_expand(const uint8_t *hop_buf, int64_t row_bytes, int32_t T, int32_t R, int32_t K,
+                      int32_t src_rank, int32_t ranks_per_server,
+                      const int32_t *hop_rank_offsets, const int32_t *hop_rank_tokens,
+                      const int32_t *flat_dest_rank, const int32_t *flat_dest_pos, const int32_t *flat_rank_offsets,
+                      int32_t flat_status, uint8_t *recv_base, int64_t recv_stride_bytes, mwo_relay_totals *totals)
+{
+    const int Kd = K < R ? K : R;
+    memset(totals, 0, sizeof(*totals));
+    for (int32_t h = 0; h < R; ++h) {
+        for (int32_t q = hop_rank_offsets[h]; q < hop_rank_offsets[h + 1]; ++q) {
+            const int32_t t = hop_rank_tokens[q];
+            const int remote = h / ranks_per_server != src_rank / ranks_per_server;
+            ++totals->hop_rows;
+            if (remote) totals->inter_multiwrite_bytes += row_bytes;
+            for (int i = 0; i < Kd; ++i) {
+                const int32_t r = flat_dest_rank[(int64_t)t * Kd + i];
+                if (r < 0 || mwo_next_hop(r, src_rank, ranks_per_server) != h) continue;
+                if (recv_base)
+                    memcpy(region(recv_base, recv_stride_bytes, flat_rank_offsets, r, row_bytes) +
+                               (int64_t)flat_dest_pos[(int64_t)t * Kd + i] * row_bytes,
+                           hop_buf + (int64_t)q * row_bytes, (size_t)row_bytes);
+                ++totals->delivered_rows;
+                if (remote) {
+                    totals->inter_unicast_bytes += row_bytes;
+                    if (r != h) totals->forward_bytes += row_bytes;
+                } else if (r != src_rank) {
+                    totals->direct_bytes += row_bytes;
+                }
+            }
+        }
+    }
+    totals->status = flat_status;
+    (void)T;
+}

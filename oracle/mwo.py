@@ -165,6 +165,47 @@ def deliver_definition(p: Plan, x: np.ndarray, topk_ids: np.ndarray, expert_to_r
     return recv
 
 
+class RelayTotals(C.Structure):
+    _fields_ = [("hop_rows", C.c_int64), ("delivered_rows", C.c_int64), ("direct_bytes", C.c_int64),
+                ("inter_multiwrite_bytes", C.c_int64), ("inter_unicast_bytes", C.c_int64),
+                ("forward_bytes", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
+
+
+def next_hop(r: int, src_rank: int, ranks_per_server: int) -> int:
+    lib().mwo_next_hop.restype = C.c_int
+    return int(lib().mwo_next_hop(C.c_int32(r), C.c_int32(src_rank), C.c_int32(ranks_per_server)))
+
+
+def relay(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: int, src_rank: int,
+          ranks_per_server: int, x: np.ndarray | None = None, recv_stride_bytes: int = 0, fill: int = 0):
+    """Two-level dispatch.  Returns (hop_plan, flat_plan, send_buf, hop_buf, recv, totals); the buffers are None
+    when no payload is given."""
+    e2r = np.ascontiguousarray(expert_to_rank, dtype=np.int32)
+    hop_tab = np.zeros_like(e2r)
+    lib().mwo_relay_table.restype = None
+    lib().mwo_relay_expand.restype = None
+    lib().mwo_relay_table(_p(e2r), C.c_int32(len(e2r)), C.c_int32(R), C.c_int32(src_rank), C.c_int32(ranks_per_server),
+                          _p(hop_tab))
+    hp = plan(topk_ids, hop_tab, R, row_bytes, src_rank)
+    fp = plan(topk_ids, e2r, R, row_bytes, src_rank)
+    send = hop_buf = recv = None
+    hop_ptr, recv_ptr = C.c_void_p(0), C.c_void_p(0)
+    if x is not None:
+        send = pack_mw(hp, x)                                # each row once per group of identical next-hop set
+        hop_buf = deliver_mw(hp, send)                       # first level: one copy per next hop
+        recv = np.full(recv_bytes_needed(fp, recv_stride_bytes), fill, np.uint8)
+        hop_ptr, recv_ptr = _p(hop_buf), _p(recv)
+    tot = RelayTotals()
+    lib().mwo_relay_expand(hop_ptr, C.c_int64(row_bytes), C.c_int32(fp.T), C.c_int32(R), C.c_int32(fp.K),
+                           C.c_int32(src_rank), C.c_int32(ranks_per_server), _p(hp.rank_offsets), _p(hp.rank_tokens),
+                           _p(fp.dest_rank), _p(fp.dest_pos), _p(fp.rank_offsets),
+                           C.c_int32(fp.totals["status"]), recv_ptr, C.c_int64(recv_stride_bytes), C.byref(tot))
+    return hp, fp, send, hop_buf, recv, tot.as_dict()
+
+
 def allgather(shards: np.ndarray, layout: int, dst_begin: int = 0, dst_count: int | None = None,
               recv_stride_bytes: int = 0, fill: int = 0):
     """Returns (send_buf, recv, totals, ret).  shards: uint8 [R, S]."""
