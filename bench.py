@@ -301,6 +301,48 @@ def allgather_sweep(mw, wl, torch) -> list:
     return out
 
 
+def relay_measure(mw, wl, torch) -> dict:
+    """Two-level dispatch (Section 3.2) on the dsv3_prefill routing: 8 servers of 8 ranks, source = rank 0."""
+    inp = wl.make_dispatch(WORKLOAD)
+    s = inp.shape
+    B, T, P, src = s.row_bytes, s.T, 8, 0
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    x = torch.from_numpy(inp.x.view(np.int16)).cuda()
+    with mw.Relay(s.R, s.E, s.K, T, B, src, P) as relay:
+        relay.mw_relay_plan(ids, e2r, T)
+        tot = relay.mw_relay_get_totals()
+        rows_send = relay.hop.mw_get_totals()["T_nonempty"]
+        H, SD = tot["hop_rows"], tot["delivered_rows"]
+        sets = [(torch.empty(rows_send * B, dtype=torch.uint8, device="cuda"), torch.empty(H * B, dtype=torch.uint8, device="cuda"),
+                 torch.empty(SD * B, dtype=torch.uint8, device="cuda")) for _ in range(2)]
+
+        def step(i):
+            send, hop, recv = sets[i % 2]
+            relay.mw_relay_plan(ids, e2r, T)
+            relay.mw_relay_dispatch(x, send, rows_send, hop, H, recv, 0, SD)
+
+        for i in range(5):
+            step(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 50
+        a.record()
+        for i in range(n):
+            step(i)
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) * 1e3 / n
+        assert relay.mw_relay_get_totals()["status"] == 0
+    moved = (2 * rows_send + (rows_send + H) + (H + SD)) * B           # pack, first level, second level
+    return {"servers": s.R // P, "ranks_per_server": P, "src_rank": src, "hop_rows": H, "delivered_rows": SD,
+            "inter_server_unicast_mb": round(tot["inter_unicast_bytes"] / 1e6, 1),
+            "inter_server_multiwrite_mb": round(tot["inter_multiwrite_bytes"] / 1e6, 1),
+            "inter_server_bytes_saved_pct": round(100 * (1 - tot["inter_multiwrite_bytes"] / tot["inter_unicast_bytes"]), 2),
+            "direct_mb": round(tot["direct_bytes"] / 1e6, 1), "relay_forward_mb": round(tot["forward_bytes"] / 1e6, 1),
+            "step_us": round(us, 1), "gbs": round(moved / us / 1e3, 1),
+            "note": "step = both plans + descriptors + pack + first-level deliver + second-level expansion"}
+
+
 def bytes_saved(wl) -> dict:
     """Transmitted-byte savings of the MultiWrite layout, exact integers from the plan (device side)."""
     import torch
@@ -479,6 +521,7 @@ def run_cuda(args):
             line["decode"] = decode_latency(mw, wl, torch)
             line["bytes_saved_pct"] = bytes_saved(wl)
             line["allgather_r64"] = allgather_sweep(mw, wl, torch)
+            line["relay_two_level"] = relay_measure(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:

@@ -158,6 +158,9 @@ MW_API int mw_destroy(mw_ctx *ctx);
 MW_API int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
             mw_plan_view *view, void *stream);
 
+/* Fills `view` with the workspace pointers of the context and the T of its latest plan (no device work). */
+MW_API int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view);
+
 /* Waits for `stream`, then copies the accounting of the latest plan to host memory. */
 MW_API int mw_get_totals(mw_ctx *ctx, mw_totals *host_out, void *stream);
 
@@ -236,6 +239,58 @@ MW_API int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_byte
 MW_API int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int32_t *expert_to_rank_host,
                      const void *x_host, int32_t T, int layout, void *recv_host, int64_t recv_capacity_rows,
                      int32_t *rank_offsets_host, mw_totals *totals_host, void *stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Two-level (relayed) MultiWrite dispatch: Section 3.2 (oversubscribed inter-server bandwidth),
+ * Section 4.1 "Local forwarding table" (one copy per distinct next hop) and Section 4.3.3 (M is
+ * partitioned by next hop; a relay re-issues the write for its part).
+ *
+ * The R ranks form servers of ranks_per_server consecutive ranks; the source is rank cfg.src_rank
+ * (it must be a member of the domain).  A destination in the source's own server is its own next
+ * hop; every other server's next hop is the rank with the source's index inside that server (the
+ * "same-index NPU"), which forwards the row to the destinations inside its server.  First level:
+ * an ordinary MultiWrite plan / pack / deliver over next-hop sets into a hop area (one region per
+ * next hop).  Second level: every row of the hop area is written to the final destinations whose
+ * next hop it is, at the slots of the flat plan, so the final receive regions are byte-identical
+ * to those of mw_dispatch.  Byte accounting is per link class.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct mw_relay mw_relay;   /* opaque: two plans (next hops, final destinations) and the second-level descriptors */
+
+typedef struct {
+    int64_t hop_rows;               /* rows the source writes: one per (token, distinct next hop)            */
+    int64_t delivered_rows;         /* rows in the final receive regions (= total_dest of the flat plan)     */
+    int64_t direct_bytes;           /* source -> destinations in its own server (its own rank excluded)      */
+    int64_t inter_multiwrite_bytes; /* source -> other servers: one copy per server holding a destination    */
+    int64_t inter_unicast_bytes;    /* the same traffic with one copy per remote destination (the baseline)  */
+    int64_t forward_bytes;          /* relays -> destinations in their server (the relay itself excluded)    */
+    int32_t status;                 /* MW_OK or the first device-side MW_ERR_* of either plan or the dispatch */
+    int32_t reserved;
+} mw_relay_totals;
+
+/* cfg as for mw_create, with 0 <= cfg->src_rank < R and R a multiple of ranks_per_server.  Synchronous. */
+MW_API int mw_relay_create(mw_relay **out, const mw_config *cfg, int32_t ranks_per_server);
+MW_API int mw_relay_destroy(mw_relay *relay);
+
+/* Plans both levels (inputs as for mw_plan).  Asynchronous on `stream`. */
+MW_API int mw_relay_plan(mw_relay *relay, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, void *stream);
+
+/* Waits for `stream`, then copies the per-link accounting of the latest mw_relay_plan / mw_relay_dispatch. */
+MW_API int mw_relay_get_totals(mw_relay *relay, mw_relay_totals *host_out, void *stream);
+
+/*
+ * Pack (each row once per group of identical next-hop set), first-level deliver into the hop area,
+ * second-level expansion into the final receive regions.
+ *   send_buf   device, send_capacity_rows rows
+ *   hop_buf    device, compact hop area of hop_capacity_rows rows (region of next hop h starts at the
+ *              first-level rank offset of h)
+ *   recv_base, recv_stride_bytes, recv_capacity_rows   as for mw_deliver
+ */
+MW_API int mw_relay_dispatch(mw_relay *relay, const void *x, void *send_buf, int64_t send_capacity_rows, void *hop_buf,
+                             int64_t hop_capacity_rows, void *recv_base, int64_t recv_stride_bytes,
+                             int64_t recv_capacity_rows, void *stream);
+
+/* The two inner contexts (first level: next hops; flat: final destinations), e.g. to read their plan views. */
+MW_API int mw_relay_contexts(mw_relay *relay, mw_ctx **hop_ctx, mw_ctx **flat_ctx);
 
 /*
  * Bitmaps and token grouping without any allocation.  (The paper has no counterpart for this

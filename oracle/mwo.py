@@ -113,7 +113,9 @@ def plan(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: in
 
 def _bytes2d(x: np.ndarray) -> np.ndarray:
     x = np.ascontiguousarray(x)
-    return x.view(np.uint8).reshape(x.shape[0], -1) if x.ndim == 2 else x.view(np.uint8)
+    if x.ndim == 2:
+        return x.view(np.uint8).reshape(x.shape[0], x.shape[1] * x.itemsize)
+    return x.view(np.uint8)
 
 
 def recv_bytes_needed(p: Plan, recv_stride_bytes: int) -> int:

@@ -30,9 +30,11 @@ MW_FLAG_PLAN_COOPERATIVE = 0x8
 MW_FLAG_NO_OVERLAP = 0x10
 MW_FLAG_COPY_REG_STORE = 0x20
 
-EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
+RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
+                 "mw_relay_contexts")
+EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
            "mw_allgather_pack", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
-           "mw_strerror")
+           "mw_strerror") + RELAY_EXPORTS
 
 
 class mw_config(C.Structure):
@@ -46,6 +48,15 @@ class mw_totals(C.Structure):
                 ("mw_bytes", C.c_int64), ("unicast_bytes", C.c_int64),
                 ("unicast_per_expert_bytes", C.c_int64), ("meta_bytes", C.c_int64),
                 ("status", C.c_int32), ("reserved", C.c_int32)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
+
+
+class mw_relay_totals(C.Structure):
+    _fields_ = [("hop_rows", C.c_int64), ("delivered_rows", C.c_int64), ("direct_bytes", C.c_int64),
+                ("inter_multiwrite_bytes", C.c_int64), ("inter_unicast_bytes", C.c_int64),
+                ("forward_bytes", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
@@ -85,6 +96,7 @@ def lib():
         L.mw_create.argtypes = [C.POINTER(vp), C.POINTER(mw_config)]
         L.mw_destroy.argtypes = [vp]
         L.mw_plan.argtypes = [vp, vp, vp, i32, C.POINTER(mw_plan_view), vp]
+        L.mw_get_plan_view.argtypes = [vp, C.POINTER(mw_plan_view)]
         L.mw_get_totals.argtypes = [vp, C.POINTER(mw_totals), vp]
         L.mw_pack.argtypes = [vp, vp, C.c_int, vp, i64, vp]
         L.mw_deliver.argtypes = [vp, C.c_int, vp, vp, i64, i64, vp]
@@ -96,9 +108,17 @@ def lib():
         L.mw_read_device.argtypes = [vp, vp, vp, i64, vp]
         L.mw_kernel_launches.argtypes = [vp]
         L.mw_kernel_launches.restype = C.c_int64
+        L.mw_relay_create.argtypes = [C.POINTER(vp), C.POINTER(mw_config), i32]
+        L.mw_relay_destroy.argtypes = [vp]
+        L.mw_relay_plan.argtypes = [vp, vp, vp, i32, vp]
+        L.mw_relay_get_totals.argtypes = [vp, C.POINTER(mw_relay_totals), vp]
+        L.mw_relay_dispatch.argtypes = [vp, vp, vp, i64, vp, i64, vp, i64, i64, vp]
+        L.mw_relay_contexts.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
+        for name in RELAY_EXPORTS:
+            getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:12]:
+        for name in EXPORTS[:13]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -142,8 +162,16 @@ def mw_group_tokens_static(topk_ids, expert_to_rank, T: int, K: int, E: int, R: 
                                         _ptr(status), _stream(stream))
 
 
+def _view_of(ctx) -> "mw_plan_view":
+    view = mw_plan_view()
+    rc = lib().mw_get_plan_view(ctx._h, C.byref(view))
+    if rc != MW_OK:
+        raise MwError(rc, "mw_get_plan_view")
+    return view
+
+
 class Context:
-    """Owns one mw_ctx.  Methods mirror the C entry points and return the C return code checked."""
+    """Owns one mw_ctx (or borrows one owned by a Relay).  Methods mirror the C entry points and return the C return code checked."""
 
     def __init__(self, R: int, E: int, K: int, max_tokens: int, row_bytes: int, src_rank: int = -1,
                  device: int = 0, flags: int = 0):
@@ -158,10 +186,20 @@ class Context:
         self.device = device
         self.view = None
 
+    @classmethod
+    def borrowed(cls, handle, R: int, E: int, K: int, row_bytes: int, device: int = 0):
+        """A view of a context owned elsewhere (not destroyed on close)."""
+        self = cls.__new__(cls)
+        self._h = C.c_void_p(handle)
+        self._owned = False
+        self.R, self.E, self.K, self.row_bytes = R, E, K, row_bytes
+        self.W, self.Kd, self.device, self.view = (R + 63) // 64, min(K, R), device, None
+        return self
+
     def close(self):
-        if self._h:
+        if self._h and getattr(self, "_owned", True):
             lib().mw_destroy(self._h)
-            self._h = C.c_void_p()
+        self._h = C.c_void_p()
 
     __del__ = close
 
@@ -263,3 +301,59 @@ class Context:
                 raise MwError(rc, "mw_read_device")
             out[name] = a
         return out
+
+
+class Relay:
+    """Owns one mw_relay: two-level dispatch through same-index relays (mirrors the mw_relay_* entry points)."""
+
+    def __init__(self, R: int, E: int, K: int, max_tokens: int, row_bytes: int, src_rank: int, ranks_per_server: int,
+                 device: int = 0, flags: int = 0):
+        self.cfg = mw_config(R, E, K, max_tokens, row_bytes, src_rank, device, flags, 0)
+        self._h = C.c_void_p()
+        rc = lib().mw_relay_create(C.byref(self._h), C.byref(self.cfg), ranks_per_server)
+        if rc != MW_OK:
+            raise MwError(rc, "mw_relay_create")
+        hop, flat = C.c_void_p(), C.c_void_p()
+        lib().mw_relay_contexts(self._h, C.byref(hop), C.byref(flat))
+        self.hop = Context.borrowed(hop.value, R, E, K, row_bytes, device)
+        self.flat = Context.borrowed(flat.value, R, E, K, row_bytes, device)
+        self.R, self.Kd, self.row_bytes = R, min(K, R), row_bytes
+
+    def close(self):
+        if self._h:
+            lib().mw_relay_destroy(self._h)
+            self._h = C.c_void_p()
+
+    __del__ = close
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def mw_relay_plan(self, topk_ids, expert_to_rank, T: int, stream=None, check: bool = True) -> int:
+        rc = lib().mw_relay_plan(self._h, _ptr(topk_ids), _ptr(expert_to_rank), T, _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_relay_plan")
+        # the inner contexts' views are fixed workspace pointers: fetch them once for plan_arrays()
+        for ctx in (self.hop, self.flat) if rc == MW_OK else ():
+            if ctx.view is None:
+                ctx.view = _view_of(ctx)
+        return rc
+
+    def mw_relay_get_totals(self, stream=None) -> dict:
+        tot = mw_relay_totals()
+        rc = lib().mw_relay_get_totals(self._h, C.byref(tot), _stream(stream))
+        if rc != MW_OK:
+            raise MwError(rc, "mw_relay_get_totals")
+        return tot.as_dict()
+
+    def mw_relay_dispatch(self, x, send_buf, send_capacity_rows: int, hop_buf, hop_capacity_rows: int, recv,
+                          recv_stride_bytes: int, recv_capacity_rows: int, stream=None, check: bool = True) -> int:
+        rc = lib().mw_relay_dispatch(self._h, _ptr(x), _ptr(send_buf), send_capacity_rows, _ptr(hop_buf),
+                                     hop_capacity_rows, _ptr(recv), recv_stride_bytes, recv_capacity_rows,
+                                     _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_relay_dispatch")
+        return rc

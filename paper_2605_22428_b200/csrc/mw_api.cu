@@ -169,6 +169,19 @@ int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank,
     return mw_plan_launch(ctx, topk_ids, expert_to_rank, T, as_stream(stream));
 }
 
+int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view)
+{
+    if (!ctx || !view) return MW_ERR_INVALID_ARG;
+    if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
+    const mw_dev &d = ctx->d;
+    view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
+    view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
+    view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
+    view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
+    view->T = ctx->planned_T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
+    return MW_OK;
+}
+
 int mw_get_totals(mw_ctx *ctx, mw_totals *host_out, void *stream)
 {
     if (!ctx || !host_out) return MW_ERR_INVALID_ARG;
