@@ -408,3 +408,80 @@ void mwo_relay_expand(const uint8_t *hop_buf, int64_t row_bytes, int32_t T, int3
     totals->status = flat_status;
     (void)T;
 }
+
+/*
+ * Paired-relay AllGather on a full mesh with two communication domains (Section 3.1, Section 5.2).
+ *
+ * R = 2n ranks; ranks [0, n) form one domain, [n, 2n) the other; rank r is paired with (r + n) mod 2n.
+ * Each domain runs its own AllGather: afterwards every rank holds the n shards of its own domain,
+ * in rank order.  A shard of shard_bytes is split in two segments: bytes [0, direct_bytes) travel on
+ * the direct links to the n - 1 other members of the domain; bytes [direct_bytes, shard_bytes) go to
+ * the paired rank of the other domain, which forwards them to those n - 1 members.
+ *   layout 0 (MultiWrite): the relayed segment crosses the pair link once;
+ *   layout 1 (unicast relay): it crosses the pair link n - 1 times, one copy per final destination.
+ * relay_buf [R, copies, relay_bytes] (copies = 1 or n - 1): region p holds what rank p received from its
+ * partner.  recv [R, n * shard_bytes].  Link loads are in bytes per directed link; every link has the
+ * same bandwidth in the paper's model, so the transfer time is max_link_bytes / w.
+ */
+typedef struct {
+    int64_t direct_link_bytes;    /* load of each used intra-domain link                       */
+    int64_t pair_link_bytes;      /* load of each pair link (source -> its partner)            */
+    int64_t forward_link_bytes;   /* load of each link partner -> member of the other domain   */
+    int64_t max_link_bytes;       /* the bottleneck                                            */
+    int64_t total_bytes;          /* all bytes put on links by all ranks                       */
+} mwo_pair_totals;
+
+int mwo_paired_allgather(const uint8_t *shards, int32_t R, int64_t shard_bytes, int64_t direct_bytes, int layout,
+                         uint8_t *relay_buf, uint8_t *recv, mwo_pair_totals *totals)
+{
+    if (R < 2 || R % 2 || shard_bytes <= 0 || direct_bytes < 0 || direct_bytes > shard_bytes || (layout != 0 && layout != 1))
+        return MWO_ERR_INVALID_ARG;
+    const int32_t n = R / 2;
+    const int64_t relay_bytes = shard_bytes - direct_bytes;
+    const int64_t copies = layout == 0 ? 1 : n - 1;
+    for (int32_t r = 0; r < R; ++r) {
+        const int32_t dom = r / n, partner = (r + n) % R;
+        const uint8_t *mine = shards + (int64_t)r * shard_bytes;
+        /* own copy: local, not on any link */
+        memcpy(recv + ((int64_t)r * n + r % n) * shard_bytes, mine, (size_t)shard_bytes);
+        /* direct segment to the other members of the domain */
+        for (int32_t q = 0; q < n; ++q) {
+            const int32_t d = dom * n + q;
+            if (d == r) continue;
+            memcpy(recv + ((int64_t)d * n + r % n) * shard_bytes, mine, (size_t)direct_bytes);
+        }
+        /* relayed segment: to the partner (once, or once per final destination) ... */
+        for (int64_t c = 0; c < copies; ++c)
+            memcpy(relay_buf + ((int64_t)partner * copies + c) * relay_bytes, mine + direct_bytes, (size_t)relay_bytes);
+        /* ... which forwards it to the other members of the source's domain */
+        int64_t k = 0;
+        for (int32_t q = 0; q < n; ++q) {
+            const int32_t d = dom * n + q;
+            if (d == r) continue;
+            const int64_t c = layout == 0 ? 0 : k;
+            memcpy(recv + ((int64_t)d * n + r % n) * shard_bytes + direct_bytes,
+                   relay_buf + ((int64_t)partner * copies + c) * relay_bytes, (size_t)relay_bytes);
+            ++k;
+        }
+    }
+    if (totals) {
+        totals->direct_link_bytes = n > 1 ? direct_bytes : 0;
+        totals->pair_link_bytes = n > 1 ? copies * relay_bytes : 0;
+        totals->forward_link_bytes = n > 1 ? relay_bytes : 0;
+        int64_t m = totals->direct_link_bytes;
+        if (totals->pair_link_bytes > m) m = totals->pair_link_bytes;
+        if (totals->forward_link_bytes > m) m = totals->forward_link_bytes;
+        totals->max_link_bytes = m;
+        totals->total_bytes = (int64_t)R * ((n - 1) * direct_bytes + totals->pair_link_bytes + (n - 1) * totals->forward_link_bytes);
+    }
+    return MWO_OK;
+}
+
+/* The split that makes the direct links and the pair link finish together (Section 5.2 step 1), rounded
+ * down to a multiple of 16 bytes: direct = shard * c / (1 + c) with c copies on the pair link. */
+int64_t mwo_balanced_direct_bytes(int64_t shard_bytes, int32_t n, int layout)
+{
+    const int64_t c = layout == 0 ? 1 : n - 1;
+    if (n <= 1) return shard_bytes;
+    return (shard_bytes * c / (1 + c)) / 16 * 16;
+}

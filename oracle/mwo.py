@@ -208,6 +208,34 @@ def relay(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: i
     return hp, fp, send, hop_buf, recv, tot.as_dict()
 
 
+class PairTotals(C.Structure):
+    _fields_ = [("direct_link_bytes", C.c_int64), ("pair_link_bytes", C.c_int64), ("forward_link_bytes", C.c_int64),
+                ("max_link_bytes", C.c_int64), ("total_bytes", C.c_int64)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+def balanced_direct_bytes(shard_bytes: int, n: int, layout: int) -> int:
+    lib().mwo_balanced_direct_bytes.restype = C.c_int64
+    return int(lib().mwo_balanced_direct_bytes(C.c_int64(shard_bytes), C.c_int32(n), C.c_int(layout)))
+
+
+def paired_allgather(shards: np.ndarray, direct_bytes: int, layout: int, fill: int = 0):
+    """Returns (relay_buf, recv, totals, ret).  shards: uint8 [R, S], R = 2n."""
+    sh = np.ascontiguousarray(shards).view(np.uint8)
+    R, S = sh.shape
+    n = R // 2
+    copies = 1 if layout == LAYOUT_MULTIWRITE else max(n - 1, 0)
+    relay_buf = np.full(max(R * copies * (S - direct_bytes), 0), fill, np.uint8)
+    recv = np.full(R * n * S, fill, np.uint8)
+    tot = PairTotals()
+    lib().mwo_paired_allgather.restype = C.c_int
+    ret = lib().mwo_paired_allgather(_p(sh), C.c_int32(R), C.c_int64(S), C.c_int64(direct_bytes), C.c_int(layout),
+                                     _p(relay_buf), _p(recv), C.byref(tot))
+    return relay_buf, recv, tot.as_dict(), ret
+
+
 def allgather(shards: np.ndarray, layout: int, dst_begin: int = 0, dst_count: int | None = None,
               recv_stride_bytes: int = 0, fill: int = 0):
     """Returns (send_buf, recv, totals, ret).  shards: uint8 [R, S]."""
