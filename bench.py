@@ -343,6 +343,39 @@ def relay_measure(mw, wl, torch) -> dict:
             "note": "step = both plans + descriptors + pack + first-level deliver + second-level expansion"}
 
 
+def paired_allgather_measure(mw, torch) -> list:
+    """Paired-relay AllGather (Sections 3.1, 5.2): 8 ranks, two TP=4 domains, 16 MB per rank (the paper's size)."""
+    R, S = 8, 16 << 20
+    n = R // 2
+    out = []
+    with mw.Context(R, 8, 2, 16, 32) as ctx:
+        shards = torch.empty(R * S, dtype=torch.uint8, device="cuda").random_(0, 256)
+        recv = torch.empty(R * n * S, dtype=torch.uint8, device="cuda")
+        relay = torch.empty(R * (n - 1) * S, dtype=torch.uint8, device="cuda")
+        cases = (("direct only", mw.MW_LAYOUT_MULTIWRITE, S),
+                 ("unicast relay", mw.MW_LAYOUT_UNICAST, mw.mw_pair_balanced_direct_bytes(S, n, mw.MW_LAYOUT_UNICAST)),
+                 ("multiwrite relay", mw.MW_LAYOUT_MULTIWRITE, mw.mw_pair_balanced_direct_bytes(S, n, mw.MW_LAYOUT_MULTIWRITE)))
+        for name, layout, direct in cases:
+            tot = None
+            for _ in range(3):
+                _, tot = ctx.mw_paired_allgather(shards, S, direct, layout, relay, recv)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(10)]
+            torch.cuda.synchronize()
+            for a, b in evs:
+                a.record()
+                ctx.mw_paired_allgather(shards, S, direct, layout, relay, recv)
+                b.record()
+            torch.cuda.synchronize()
+            us = statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3
+            copies = 1 if layout == mw.MW_LAYOUT_MULTIWRITE else n - 1
+            moved = R * ((1 + n) * direct + (S - direct) * (1 + copies + 1) + (n - 1) * 2 * (S - direct)) if direct < S \
+                else R * (1 + n) * S
+            out.append({"scheme": name, "direct_bytes": direct, "p50_us": round(us, 1), "gbs": round(moved / us / 1e3, 1),
+                        "max_link_mb": round(tot["max_link_bytes"] / 1e6, 2),
+                        "model_time_vs_direct_only": round(tot["max_link_bytes"] / S, 4)})
+    return out
+
+
 def bytes_saved(wl) -> dict:
     """Transmitted-byte savings of the MultiWrite layout, exact integers from the plan (device side)."""
     import torch
@@ -522,6 +555,7 @@ def run_cuda(args):
             line["bytes_saved_pct"] = bytes_saved(wl)
             line["allgather_r64"] = allgather_sweep(mw, wl, torch)
             line["relay_two_level"] = relay_measure(mw, wl, torch)
+            line["paired_allgather_8x16MB"] = paired_allgather_measure(mw, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:

@@ -228,6 +228,36 @@ MW_API int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_byte
                       mw_totals *host_totals, void *stream);
 
 /*
+ * Paired-relay AllGather with segment split (Section 3.1 "paired relaying", Section 5.2): cfg.R = 2n
+ * ranks on a full mesh form two domains, [0, n) and [n, 2n); rank r is paired with (r + n) mod 2n.
+ * Each domain gathers its own n shards: afterwards the receive region of every rank holds the shards
+ * of its domain in rank order.  Bytes [0, direct_bytes) of a shard go on the direct links to the other
+ * members of the domain; bytes [direct_bytes, shard_bytes) go to the paired rank, which forwards them
+ * to those members.  MW_LAYOUT_MULTIWRITE: the relayed segment crosses the pair link once;
+ * MW_LAYOUT_UNICAST: n - 1 times, one copy per final destination.
+ *   shards      device, [R, shard_bytes]; shard_bytes and direct_bytes multiples of 16
+ *   relay_buf   device, [R, copies, shard_bytes - direct_bytes], copies = 1 or n - 1: region p is what
+ *               rank p received from its partner
+ *   recv_base   device, [R, n * shard_bytes]
+ *   host_totals host, optional: bytes per directed link (every link has the same bandwidth in the
+ *               paper's model, so the transfer time is max_link_bytes / bandwidth)
+ */
+typedef struct {
+    int64_t direct_link_bytes;    /* load of each used intra-domain link                     */
+    int64_t pair_link_bytes;      /* load of each pair link (source -> its partner)          */
+    int64_t forward_link_bytes;   /* load of each link partner -> member of the other domain */
+    int64_t max_link_bytes;       /* the bottleneck                                          */
+    int64_t total_bytes;          /* all bytes put on links by all ranks                     */
+} mw_pair_totals;
+
+MW_API int mw_paired_allgather(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int64_t direct_bytes, int layout,
+                               void *relay_buf, void *recv_base, mw_pair_totals *host_totals, void *stream);
+
+/* The split that lets the direct links and the pair link finish together (Section 5.2 step 1, equal link
+ * bandwidths): shard_bytes * c / (1 + c) with c copies on the pair link, rounded down to a multiple of 16. */
+MW_API int64_t mw_pair_balanced_direct_bytes(int64_t shard_bytes, int32_t ranks_per_domain, int layout);
+
+/*
  * One whole dispatch from host memory (plan, pack, deliver) for callers whose data lives on
  * the host: copies topk_ids, expert_to_rank and x to the device, runs mw_plan and mw_dispatch
  * into context-owned staging, and copies the compact receive area (total_dest rows), the

@@ -33,8 +33,8 @@ MW_FLAG_COPY_REG_STORE = 0x20
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
 EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
-           "mw_allgather_pack", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
-           "mw_strerror") + RELAY_EXPORTS
+           "mw_allgather_pack", "mw_paired_allgather", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
+           "mw_strerror", "mw_pair_balanced_direct_bytes") + RELAY_EXPORTS
 
 
 class mw_config(C.Structure):
@@ -60,6 +60,14 @@ class mw_relay_totals(C.Structure):
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
+
+
+class mw_pair_totals(C.Structure):
+    _fields_ = [("direct_link_bytes", C.c_int64), ("pair_link_bytes", C.c_int64), ("forward_link_bytes", C.c_int64),
+                ("max_link_bytes", C.c_int64), ("total_bytes", C.c_int64)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
 
 
 class mw_plan_view(C.Structure):
@@ -103,6 +111,9 @@ def lib():
         L.mw_dispatch.argtypes = [vp, vp, C.c_int, vp, i64, vp, i64, i64, vp]
         L.mw_plan_dispatch.argtypes = [vp, vp, vp, i32, vp, C.c_int, vp, i64, vp, i64, i64, C.POINTER(mw_plan_view), vp]
         L.mw_allgather_pack.argtypes = [vp, vp, i64, C.c_int, vp, vp, i64, i32, i32, C.POINTER(mw_totals), vp]
+        L.mw_paired_allgather.argtypes = [vp, vp, i64, i64, C.c_int, vp, vp, C.POINTER(mw_pair_totals), vp]
+        L.mw_pair_balanced_direct_bytes.argtypes = [i64, i32, C.c_int]
+        L.mw_pair_balanced_direct_bytes.restype = i64
         L.mw_dispatch_host.argtypes = [vp, vp, vp, vp, i32, C.c_int, vp, i64, vp, C.POINTER(mw_totals), vp]
         L.mw_group_tokens_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.mw_read_device.argtypes = [vp, vp, vp, i64, vp]
@@ -118,10 +129,14 @@ def lib():
             getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:13]:
+        for name in EXPORTS[:14]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
+
+
+def mw_pair_balanced_direct_bytes(shard_bytes: int, ranks_per_domain: int, layout: int) -> int:
+    return int(lib().mw_pair_balanced_direct_bytes(shard_bytes, ranks_per_domain, layout))
 
 
 def strerror(code: int) -> str:
@@ -268,6 +283,15 @@ class Context:
                                      recv_stride_bytes, dst_rank_begin, cnt, C.byref(tot), _stream(stream))
         if check and rc != MW_OK:
             raise MwError(rc, "mw_allgather_pack")
+        return rc, tot.as_dict()
+
+    def mw_paired_allgather(self, shards, shard_bytes: int, direct_bytes: int, layout: int, relay_buf, recv,
+                            stream=None, check: bool = True):
+        tot = mw_pair_totals()
+        rc = lib().mw_paired_allgather(self._h, _ptr(shards), shard_bytes, direct_bytes, layout, _ptr(relay_buf),
+                                       _ptr(recv), C.byref(tot), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_paired_allgather")
         return rc, tot.as_dict()
 
     def mw_dispatch_host(self, topk_ids_host, expert_to_rank_host, x_host, T: int, layout: int, recv_host,

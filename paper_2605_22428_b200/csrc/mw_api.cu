@@ -332,6 +332,67 @@ int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int 
     return mw_copy_launch(ctx, a, as_stream(stream));
 }
 
+int64_t mw_pair_balanced_direct_bytes(int64_t shard_bytes, int32_t ranks_per_domain, int layout)
+{
+    if (ranks_per_domain <= 1) return shard_bytes;
+    const int64_t c = layout == MW_LAYOUT_MULTIWRITE ? 1 : ranks_per_domain - 1;
+    return (shard_bytes * c / (1 + c)) / 16 * 16;
+}
+
+int mw_paired_allgather(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int64_t direct_bytes, int layout,
+                        void *relay_buf, void *recv_base, mw_pair_totals *host_totals, void *stream)
+{
+    if (!ctx || !shards || !recv_base || shard_bytes < 16 || direct_bytes < 0 || direct_bytes > shard_bytes || check_layout(layout))
+        return MW_ERR_INVALID_ARG;
+    const int R = ctx->cfg.R;
+    if (R < 2 || R % 2) return MW_ERR_INVALID_ARG;
+    const int n = R / 2;
+    const int64_t relay_bytes = shard_bytes - direct_bytes;
+    const int copies = layout == MW_LAYOUT_MULTIWRITE ? 1 : n - 1;
+    if (relay_bytes > 0 && copies > 0 && !relay_buf) return MW_ERR_INVALID_ARG;
+    if (shard_bytes % 16 || direct_bytes % 16 || !aligned16(shards) || !aligned16(recv_base) || (relay_buf && !aligned16(relay_buf)))
+        return MW_ERR_ALIGNMENT;
+    if (host_totals) {
+        host_totals->direct_link_bytes = n > 1 ? direct_bytes : 0;
+        host_totals->pair_link_bytes = n > 1 ? copies * relay_bytes : 0;
+        host_totals->forward_link_bytes = n > 1 ? relay_bytes : 0;
+        int64_t m = host_totals->direct_link_bytes;
+        if (host_totals->pair_link_bytes > m) m = host_totals->pair_link_bytes;
+        if (host_totals->forward_link_bytes > m) m = host_totals->forward_link_bytes;
+        host_totals->max_link_bytes = m;
+        host_totals->total_bytes = (int64_t)R * ((n - 1) * direct_bytes + host_totals->pair_link_bytes +
+                                                 (n - 1) * host_totals->forward_link_bytes);
+    }
+    mw_copy_args a = base_args(ctx);
+    a.rows_from = 0;
+    a.capacity_rows = INT64_MAX;
+    a.shard_bytes = shard_bytes;
+    a.pair_n = n;
+    a.pair_copies = copies;
+    int rc = MW_OK;
+    if (direct_bytes > 0) {                    // direct segment to every member of the domain (own copy included, local)
+        a.mode = MW_CP_PAIR_DIRECT;
+        a.src = (const uint8_t *)shards; a.dst = (uint8_t *)recv_base;
+        a.row_bytes = direct_bytes; a.seg_off = 0; a.host_rows = R;
+        if ((rc = mw_copy_launch(ctx, a, as_stream(stream))) != MW_OK) return rc;
+    }
+    if (relay_bytes > 0) {
+        a.mode = MW_CP_PAIR_SEND;              // relayed segment to the partner's relay area (and own copy)
+        a.src = (const uint8_t *)shards; a.dst = (uint8_t *)relay_buf; a.dst2 = (uint8_t *)recv_base;
+        a.row_bytes = relay_bytes; a.seg_off = direct_bytes; a.host_rows = R;
+        a.keep_in_l2 = 1;                      // the forward launch reads the relay area next
+        if ((rc = mw_copy_launch(ctx, a, as_stream(stream))) != MW_OK) return rc;
+        if (n > 1) {
+            a.keep_in_l2 = 0;
+            a.mode = MW_CP_PAIR_FORWARD;       // the partner forwards it to the other members of the source's domain
+            a.src = (const uint8_t *)relay_buf; a.dst = (uint8_t *)recv_base;
+            a.host_rows = (int64_t)R * (n - 1);
+            rc = mw_copy_launch(ctx, a, as_stream(stream));
+        }
+    }
+    return rc;
+}
+
 int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int32_t *expert_to_rank_host,
                      const void *x_host, int32_t T, int layout, void *recv_host, int64_t recv_capacity_rows,
                      int32_t *rank_offsets_host, mw_totals *totals_host, void *stream)

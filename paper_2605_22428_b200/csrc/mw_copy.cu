@@ -120,6 +120,13 @@ __device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t
         const int64_t i = row / a.dst_count, d = row % a.dst_count;
         return (a.dst_begin + d == i) ? a.src2 + i * a.row_bytes : a.src + row * a.row_bytes;
     }
+    case MW_CP_PAIR_DIRECT:
+    case MW_CP_PAIR_SEND: return a.src + row * a.shard_bytes + a.seg_off;
+    case MW_CP_PAIR_FORWARD: {
+        const int64_t r = row / (a.pair_n - 1), k = row % (a.pair_n - 1);
+        const int64_t partner = (r + a.pair_n) % a.R;
+        return a.src + (partner * a.pair_copies + (a.pair_copies == 1 ? 0 : k)) * a.row_bytes;
+    }
     default: return a.src + row * a.row_bytes;
     }
 }
@@ -140,6 +147,8 @@ __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row)
     case MW_CP_SCATTER: return a.ndst[row];
     case MW_CP_AG_DELIVER_MW:
     case MW_CP_AG_PACK_UC: return a.dst_count;
+    case MW_CP_PAIR_DIRECT: return a.pair_n;
+    case MW_CP_PAIR_SEND: return a.pair_copies + 1;
     default: return 1;
     }
 }
@@ -187,6 +196,22 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
     case MW_CP_AG_DELIVER_UC: {
         const int64_t i = row / a.dst_count, d = row % a.dst_count;
         return a.dst + d * a.dst_stride + i * a.row_bytes;
+    }
+    // paired AllGather: receive region of rank d holds the n shards of d's domain, shard of rank r at slot r % n
+    case MW_CP_PAIR_DIRECT: {
+        const int64_t d = (row / a.pair_n) * a.pair_n + q;
+        return a.dst + (d * a.pair_n + row % a.pair_n) * a.shard_bytes + a.seg_off;
+    }
+    case MW_CP_PAIR_SEND: {
+        if (q == a.pair_copies) return a.dst2 + (row * a.pair_n + row % a.pair_n) * a.shard_bytes + a.seg_off;   // own copy, local
+        const int64_t partner = (row + a.pair_n) % a.R;
+        return a.dst + (partner * a.pair_copies + q) * a.row_bytes;
+    }
+    case MW_CP_PAIR_FORWARD: {
+        const int64_t r = row / (a.pair_n - 1), k = row % (a.pair_n - 1);
+        const int64_t qd = k < r % a.pair_n ? k : k + 1;                 // k-th member of r's domain other than r
+        const int64_t d = (r / a.pair_n) * a.pair_n + qd;
+        return a.dst + (d * a.pair_n + r % a.pair_n) * a.shard_bytes + a.seg_off;
     }
     }
     return nullptr;

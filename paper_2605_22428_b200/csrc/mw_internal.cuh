@@ -107,7 +107,10 @@ enum mw_copy_mode {
     MW_CP_AG_PACK_MW = 3,   // send[i] = shard[i]
     MW_CP_AG_DELIVER_MW = 4,// region(d)[i] = send[i] for every d of the window
     MW_CP_AG_PACK_UC = 5,   // send[i][d] = shard[i] for every d of the window except rank i itself
-    MW_CP_AG_DELIVER_UC = 6 // region(d)[i] = send[i][d] (own shard: taken from shards)
+    MW_CP_AG_DELIVER_UC = 6,// region(d)[i] = send[i][d] (own shard: taken from shards)
+    MW_CP_PAIR_DIRECT = 7,  // paired AllGather: direct segment of shard r to every member of r's domain
+    MW_CP_PAIR_SEND = 8,    // relayed segment of shard r to its partner's relay area (and to r itself)
+    MW_CP_PAIR_FORWARD = 9  // partner forwards the relayed segment to the other members of r's domain
 };
 
 struct mw_copy_args {
@@ -115,6 +118,7 @@ struct mw_copy_args {
     const uint8_t *src;        // source rows (x, send buffer or shards)
     const uint8_t *src2;       // AllGather unicast deliver: the shards (own copy is local)
     uint8_t *dst;              // destination base
+    uint8_t *dst2;             // paired AllGather, relayed segment: the receive area (own copy), dst being the relay area
     int64_t row_bytes;         // bytes per row (B, or the shard size)
     int64_t dst_stride;        // bytes between receive regions; 0 = compact
     int64_t capacity_rows;     // rows the destination may hold (per region when strided)
@@ -127,6 +131,8 @@ struct mw_copy_args {
     int keep_in_l2;            // destination rows are read again soon: do not mark them evict-first
     unsigned int *work_ctr;    // [2] ticket counter, finished-warp counter (both zero between launches)
     int Kd, R, dst_begin, dst_count;
+    int pair_n, pair_copies;   // paired AllGather: ranks per domain, copies of the relayed segment on the pair link
+    int64_t shard_bytes, seg_off;   // paired AllGather: whole shard size, offset of the segment being moved
     const int32_t *src_index;  // PACK_MW: mw_row_token
     const int32_t *ndst;       // SCATTER: destinations per row
     const int32_t *d_rank;     // SCATTER: [Kd, d_stride] destination ranks, entry i of row j at i * d_stride + j
