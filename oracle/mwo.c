@@ -485,3 +485,67 @@ int64_t mwo_balanced_direct_bytes(int64_t shard_bytes, int32_t n, int layout)
     if (n <= 1) return shard_bytes;
     return (shard_bytes * c / (1 + c)) / 16 * 16;
 }
+
+/*
+ * Combine: the reverse of dispatch (Section 2.3.2: "returns computation results from experts back to
+ * their original senders"; it carries no redundant data, so MultiWrite does not change it).
+ *
+ * Reading taken: every destination rank r of token t returns one row z[r][dest_pos(t, r)] of bf16
+ * values (its local experts' contribution), in the slot the dispatch delivered the token to; the source
+ * forms  y[t] = sum over the destinations of t, in ascending rank order, of w[t, i] * z[r_i][slot_i]
+ * with the sum carried in double precision here and rounded once to bf16 (round to nearest even).
+ * weights == NULL means all ones.  A token without destinations gets a row of zeros.
+ */
+#include <math.h>
+
+static double bf16_to_double(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+/* double -> bf16 bits, one rounding (nearest even), bf16 = sign, 8 exponent bits, 7 fraction bits */
+static uint16_t double_to_bf16(double x)
+{
+    if (isnan(x)) return 0x7FC0;
+    uint16_t sign = signbit(x) ? 0x8000 : 0;
+    double a = fabs(x);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return sign | 0x7F80;
+    int e;
+    frexp(a, &e);                                   /* a = m * 2^e, m in [0.5, 1)  ->  a in [2^(e-1), 2^e) */
+    int ex = e - 1;                                 /* unbiased exponent of a                               */
+    if (ex < -126) ex = -126;                       /* subnormal range: fixed scale                         */
+    double q = nearbyint(ldexp(a, 7 - ex));         /* significand in units of 2^(ex-7), ties to even       */
+    if (q >= 256.0) { q = 128.0; ++ex; }            /* rounding carried into the next binade                */
+    if (ex > 127) return sign | 0x7F80;
+    if (q < 128.0) return sign | (uint16_t)q;       /* subnormal (or zero)                                  */
+    return sign | (uint16_t)(((ex + 127) << 7) | ((int)q - 128));
+}
+
+void mwo_combine(const uint8_t *z_base, int64_t z_stride_bytes, const float *weights, int32_t T, int32_t R, int32_t K,
+                 int64_t row_bytes, const int32_t *dest_rank, const int32_t *dest_pos, const int32_t *rank_offsets,
+                 uint8_t *y)
+{
+    const int Kd = K < R ? K : R;
+    const int64_t H = row_bytes / 2;
+    for (int32_t t = 0; t < T; ++t) {
+        uint16_t *out = (uint16_t *)(y + (int64_t)t * row_bytes);
+        for (int64_t c = 0; c < H; ++c) {
+            double acc = 0.0;
+            int any = 0;
+            for (int i = 0; i < Kd; ++i) {
+                const int32_t r = dest_rank[(int64_t)t * Kd + i];
+                if (r < 0) break;
+                const uint8_t *row = region((uint8_t *)z_base, z_stride_bytes, rank_offsets, r, row_bytes) +
+                                     (int64_t)dest_pos[(int64_t)t * Kd + i] * row_bytes;
+                const double w = weights ? (double)weights[(int64_t)t * Kd + i] : 1.0;
+                acc += w * bf16_to_double(((const uint16_t *)row)[c]);
+                any = 1;
+            }
+            out[c] = any ? double_to_bf16(acc) : 0;
+        }
+    }
+}

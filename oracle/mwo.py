@@ -40,7 +40,7 @@ def build(force: bool = False) -> str:
     stale = force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
     if stale:
         tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC])
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -206,6 +206,18 @@ def relay(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: i
                            _p(fp.dest_rank), _p(fp.dest_pos), _p(fp.rank_offsets),
                            C.c_int32(fp.totals["status"]), recv_ptr, C.c_int64(recv_stride_bytes), C.byref(tot))
     return hp, fp, send, hop_buf, recv, tot.as_dict()
+
+
+def combine(p: Plan, z: np.ndarray, weights: np.ndarray | None = None, z_stride_bytes: int = 0) -> np.ndarray:
+    """y uint16 [T, H] (bf16 bits).  z: the receive area (uint8), laid out like the dispatch's."""
+    zz = np.ascontiguousarray(z).view(np.uint8).reshape(-1)
+    y = np.zeros((p.T, p.row_bytes // 2), np.uint16)
+    w = None if weights is None else np.ascontiguousarray(weights, dtype=np.float32)
+    lib().mwo_combine.restype = None
+    lib().mwo_combine(_p(zz), C.c_int64(z_stride_bytes), _p(w) if w is not None else C.c_void_p(0), C.c_int32(p.T),
+                      C.c_int32(p.R), C.c_int32(p.K), C.c_int64(p.row_bytes), _p(p.dest_rank), _p(p.dest_pos),
+                      _p(p.rank_offsets), _p(y))
+    return y
 
 
 class PairTotals(C.Structure):

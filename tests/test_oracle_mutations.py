@@ -6,13 +6,24 @@ import subprocess
 
 import pytest
 
+import test_oracle_combine_pins as cpins
+import test_oracle_pair_pins as ppins
 import test_oracle_pins as pins
+import test_oracle_relay_pins as rpins
 from oracle import mwo
 from paper_2605_22428_b200 import workloads as wl
 
 SRC = os.path.join(os.path.dirname(mwo.__file__), "mwo.c")
 
 MUTATIONS = {
+    "combine ignores the weights": ("acc += w * bf16_to_double(", "acc += bf16_to_double("),
+    "combine truncates instead of rounding": ("double q = nearbyint(ldexp(a, 7 - ex));", "double q = floor(ldexp(a, 7 - ex));"),
+    "combine reads the wrong slot": ("(int64_t)dest_pos[(int64_t)t * Kd + i] * row_bytes;\n                const double w",
+                                     "(int64_t)(dest_pos[(int64_t)t * Kd + i] > 0 ? dest_pos[(int64_t)t * Kd + i] - 1 : 0) * row_bytes;\n                const double w"),
+    "relay sends to rank 0 of the remote server": ("return (r / ranks_per_server) * ranks_per_server + src_rank % ranks_per_server;",
+                                                   "return (r / ranks_per_server) * ranks_per_server;"),
+    "paired allgather forwards the direct segment": ("relay_buf + ((int64_t)partner * copies + c) * relay_bytes, (size_t)relay_bytes);\n            ++k;",
+                                                     "mine, (size_t)relay_bytes);\n            ++k;"),
     "bit index taken modulo 32": ("(uint64_t)1 << (r % 64)", "(uint64_t)1 << (r % 32)"),
     "always word 0": ("m[r / 64] |=", "m[0] |="),
     "padding treated as an error": ("if (id == -1) continue;                         /* padding slot            */", ""),
@@ -51,6 +62,12 @@ def run_pins():
         pins.test_allgather_is_concatenate(layout, 5, 48, 1, 3)
         pins.test_allgather_is_concatenate(layout, 8, 64, 0, 8)
     pins.test_allgather_saved_closed_form_and_paper_example()
+    cpins.test_one_hot_weights_select_one_destination(False)
+    cpins.test_unit_weights_sum_small_integers_exactly()
+    cpins.test_rounding_is_nearest_even_with_a_single_rounding()
+    rpins.test_paper_example_four_local_four_remote()
+    rpins.test_relay_brute_force(1, 12, 3, 7, 24, 4)
+    ppins.test_every_rank_gets_its_domain_in_order(0, 8, 64, 32)
 
 
 def test_unmutated_oracle_passes_the_subset():
@@ -65,7 +82,7 @@ def test_planted_mistake_is_caught(name, tmp_path, monkeypatch):
     mutated = tmp_path / "mwo_mut.c"
     mutated.write_text(text.replace(old, new, 1))
     lib_path = tmp_path / "libmwo_mut.so"
-    subprocess.check_call(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-w", "-o", str(lib_path), str(mutated)])
+    subprocess.check_call(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-w", "-o", str(lib_path), str(mutated), "-lm"])
     lib = ctypes.CDLL(str(lib_path))
     lib.mwo_plan.restype = ctypes.c_int
     lib.mwo_allgather.restype = ctypes.c_int
