@@ -343,6 +343,35 @@ def relay_measure(mw, wl, torch) -> dict:
             "note": "step = both plans + descriptors + pack + first-level deliver + second-level expansion"}
 
 
+def combine_measure(mw, wl, torch) -> dict:
+    """Combine (Section 2.3.2) on the dsv3_prefill routing: every destination returns one bf16 row per token."""
+    inp = wl.make_dispatch(WORKLOAD, payload=False)
+    s = inp.shape
+    B, T = s.row_bytes, s.T
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+        ctx.mw_plan(ids, e2r, T)
+        SD = ctx.mw_get_totals()["total_dest"]
+        Kd = min(s.K, s.R)
+        zs = [torch.randn(SD * B // 2, dtype=torch.bfloat16, device="cuda") for _ in range(2)]     # 2 x 340 MB > L2
+        ys = [torch.empty(T * B, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        w = torch.rand(T * Kd, dtype=torch.float32, device="cuda")
+        for i in range(4):
+            ctx.mw_combine(zs[i % 2], 0, w, ys[i % 2])
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 40
+        a.record()
+        for i in range(n):
+            ctx.mw_combine(zs[i % 2], 0, w, ys[i % 2])
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) * 1e3 / n
+    moved = (SD + T) * B + T * Kd * 4
+    return {"rows_read": SD, "rows_written": T, "us": round(us, 1), "gbs": round(moved / us / 1e3, 1),
+            "note": "bf16 rows, fp32 accumulation; bytes = rows read + rows written + weights"}
+
+
 def paired_allgather_measure(mw, torch) -> list:
     """Paired-relay AllGather (Sections 3.1, 5.2): 8 ranks, two TP=4 domains, 16 MB per rank (the paper's size)."""
     R, S = 8, 16 << 20
@@ -486,6 +515,7 @@ def run_cuda(args):
     if args.kernels_only:
         sampler.stop()
         print(json.dumps({"kernels_only": True, "ms_per_step": total_ms / args.steps, "steps": args.steps,
+                          "combine": combine_measure(mw, wl, torch),
                           "stages_us": {"plan": statistics.mean(plan_ms) * 1e3, "pack": statistics.mean(pack_ms) * 1e3,
                                         "deliver": statistics.mean(deliver_ms) * 1e3}}))
         ctx.close()
@@ -556,6 +586,7 @@ def run_cuda(args):
             line["allgather_r64"] = allgather_sweep(mw, wl, torch)
             line["relay_two_level"] = relay_measure(mw, wl, torch)
             line["paired_allgather_8x16MB"] = paired_allgather_measure(mw, torch)
+            line["combine_dsv3_prefill"] = combine_measure(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:

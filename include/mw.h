@@ -228,6 +228,21 @@ MW_API int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_byte
                       mw_totals *host_totals, void *stream);
 
 /*
+ * Combine: the reverse of dispatch (Section 2.3.2: results return from the experts to their senders;
+ * the step carries no redundant data and is not changed by MultiWrite).  Uses the latest plan.
+ * Every destination rank r of token t has put one bf16 row into z at the slot the dispatch delivered
+ * the token to (same compact or strided layout as the receive area); the source computes
+ *     y[t] = sum over the destinations of t, in ascending rank order, of weights[t, i] * z[r_i][slot_i]
+ * with fp32 accumulation by fused multiply-add in that order and one rounding to bf16 (nearest even).
+ * Rows are row_bytes / 2 bf16 values; this is the only call that interprets the payload.
+ *   z_base          device, 16-byte aligned; z_stride_bytes as recv_stride_bytes of mw_deliver (0 = compact)
+ *   weights         device float32 [T, Kd] (entry i belongs to the i-th destination rank, ascending), or
+ *                   NULL for all ones
+ *   y               device, [T, row_bytes]; a token without destinations gets zeros
+ */
+MW_API int mw_combine(mw_ctx *ctx, const void *z_base, int64_t z_stride_bytes, const float *weights, void *y, void *stream);
+
+/*
  * Paired-relay AllGather with segment split (Section 3.1 "paired relaying", Section 5.2): cfg.R = 2n
  * ranks on a full mesh form two domains, [0, n) and [n, 2n); rank r is paired with (r + n) mod 2n.
  * Each domain gathers its own n shards: afterwards the receive region of every rank holds the shards

@@ -33,7 +33,7 @@ MW_FLAG_COPY_REG_STORE = 0x20
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
 EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
-           "mw_allgather_pack", "mw_paired_allgather", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
+           "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
            "mw_strerror", "mw_pair_balanced_direct_bytes") + RELAY_EXPORTS
 
 
@@ -114,6 +114,7 @@ def lib():
         L.mw_paired_allgather.argtypes = [vp, vp, i64, i64, C.c_int, vp, vp, C.POINTER(mw_pair_totals), vp]
         L.mw_pair_balanced_direct_bytes.argtypes = [i64, i32, C.c_int]
         L.mw_pair_balanced_direct_bytes.restype = i64
+        L.mw_combine.argtypes = [vp, vp, i64, vp, vp, vp]
         L.mw_dispatch_host.argtypes = [vp, vp, vp, vp, i32, C.c_int, vp, i64, vp, C.POINTER(mw_totals), vp]
         L.mw_group_tokens_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.mw_read_device.argtypes = [vp, vp, vp, i64, vp]
@@ -129,7 +130,7 @@ def lib():
             getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:14]:
+        for name in EXPORTS[:15]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -293,6 +294,12 @@ class Context:
         if check and rc != MW_OK:
             raise MwError(rc, "mw_paired_allgather")
         return rc, tot.as_dict()
+
+    def mw_combine(self, z, z_stride_bytes: int, weights, y, stream=None, check: bool = True) -> int:
+        rc = lib().mw_combine(self._h, _ptr(z), z_stride_bytes, _ptr(weights), _ptr(y), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_combine")
+        return rc
 
     def mw_dispatch_host(self, topk_ids_host, expert_to_rank_host, x_host, T: int, layout: int, recv_host,
                          recv_capacity_rows: int, rank_offsets_host, stream=None, check: bool = True):
