@@ -72,12 +72,15 @@ extern "C" {
 
 #define MW_FLAG_HOST_STAGING   0x1u  /* allocate device staging so mw_dispatch_host can be used */
 #define MW_FLAG_PLAN_MULTIPASS 0x2u  /* always take the tiled multi-kernel plan, even for small T */
-#define MW_FLAG_COPY_LDST      0x4u  /* row copies by 16-byte register loads/stores, not bulk copies */
+#define MW_FLAG_COPY_LDST      0x4u  /* row copies by a persistent grid of warps with 16-byte register loads/stores */
 #define MW_FLAG_PLAN_COOPERATIVE 0x8u /* launch the fused plan through the cooperative-launch API (the   */
                                       /* driver then guarantees that all its blocks are resident; costs   */
                                       /* about 20 us of host time per plan); default is an ordinary launch */
 #define MW_FLAG_NO_OVERLAP     0x10u /* do not let a kernel's start-up overlap the previous kernel's tail */
-#define MW_FLAG_COPY_REG_STORE 0x20u /* fan rows out with 16-byte register stores instead of shared->global bulk copies */
+#define MW_FLAG_COPY_REG_STORE 0x20u /* persistent grid, bulk loads into shared memory, 16-byte register stores */
+#define MW_FLAG_COPY_BULK      0x40u /* persistent grid, bulk (TMA) loads into shared memory and bulk stores out of it; */
+                                     /* without any MW_FLAG_COPY_* bit row copies run one block per (row, piece) with   */
+                                     /* plain 16-byte loads and stores, which measured fastest on B200                  */
 
 #define MW_MAX_RANKS   1024
 #define MW_MAX_TOPK    64

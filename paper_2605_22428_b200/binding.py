@@ -29,6 +29,7 @@ MW_FLAG_COPY_LDST = 0x4
 MW_FLAG_PLAN_COOPERATIVE = 0x8
 MW_FLAG_NO_OVERLAP = 0x10
 MW_FLAG_COPY_REG_STORE = 0x20
+MW_FLAG_COPY_BULK = 0x40
 
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")

@@ -111,9 +111,9 @@ __device__ __forceinline__ int64_t n_rows(const mw_copy_args &a)
     return a.host_rows;
 }
 
-__device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t row)
+__device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t row, int mode)
 {
-    switch (a.mode) {
+    switch (mode) {
     case MW_CP_PACK_MW: return a.src + (int64_t)a.src_index[row] * a.row_bytes;
     case MW_CP_SCATTER: return a.src + (a.src_index ? (int64_t)a.src_index[row] : row) * a.row_bytes;
     case MW_CP_AG_DELIVER_UC: {
@@ -132,18 +132,24 @@ __device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t
 }
 
 // Rows whose source is found through an index array: the index is loaded one item ahead of its use.
-__device__ __forceinline__ bool src_is_indexed(const mw_copy_args &a)
+__device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t row) { return src_row(a, row, a.mode); }
+__device__ __forceinline__ bool src_is_indexed(const mw_copy_args &a, int mode)
 {
-    return a.mode == MW_CP_PACK_MW || (a.mode == MW_CP_SCATTER && a.src_index);
+    return mode == MW_CP_PACK_MW || (mode == MW_CP_SCATTER && a.src_index);
+}
+__device__ __forceinline__ bool src_is_indexed(const mw_copy_args &a) { return src_is_indexed(a, a.mode); }
+__device__ __forceinline__ const uint8_t *src_row_with(const mw_copy_args &a, int64_t row, int index, int mode)
+{
+    return src_is_indexed(a, mode) ? a.src + (int64_t)index * a.row_bytes : src_row(a, row, mode);
 }
 __device__ __forceinline__ const uint8_t *src_row_with(const mw_copy_args &a, int64_t row, int index)
 {
-    return src_is_indexed(a) ? a.src + (int64_t)index * a.row_bytes : src_row(a, row);
+    return src_row_with(a, row, index, a.mode);
 }
 
-__device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row)
+__device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row, int mode)
 {
-    switch (a.mode) {
+    switch (mode) {
     case MW_CP_SCATTER: return a.ndst[row];
     case MW_CP_AG_DELIVER_MW:
     case MW_CP_AG_PACK_UC: return a.dst_count;
@@ -153,11 +159,13 @@ __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row)
     }
 }
 
+__device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row) { return n_dst(a, row, a.mode); }
+
 // Destination q of a row; nullptr when the copy must not happen (capacity exceeded -> status, or the
 // AllGather copy addressed to the shard's own rank, which is never transmitted).
-__device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, int q)
+__device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, int q, int mode)
 {
-    switch (a.mode) {
+    switch (mode) {
     case MW_CP_PACK_MW:
     case MW_CP_AG_PACK_MW:
         if (row >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
@@ -216,6 +224,8 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
     }
     return nullptr;
 }
+
+__device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, int q) { return dst_row(a, row, q, a.mode); }
 
 __device__ __forceinline__ bool plan_unusable(const mw_copy_args &a)
 {
@@ -579,6 +589,75 @@ __global__ void __launch_bounds__(kLdstThreads) k_copy_ldst(const __grid_constan
     }
 }
 
+// ---- one block per (row, piece): plain loads and stores, ordinary grid ---------------------------
+// The default.  A piece is blockDim.x * V 16-byte vectors (at most kRowsMaxVecs); a thread loads V vectors of
+// the piece once and stores them to every destination of the row.  With many more blocks than SMs the hardware
+// scheduler balances the load and hides each block's start-up behind its neighbours.  Blocks live for a few
+// microseconds, so every dependent step before the first store counts: measured on B200 (4096 rows of 14336
+// bytes, 7.7 copies each) a 64-bit division, inline-asm stores the compiler cannot schedule around, or one more
+// dependent round trip to L2 each cost 2 to 12 % of the run time.
+constexpr int kRowsMaxVecs = 512;
+constexpr int kRowsDstBatch = 64;
+
+__host__ __device__ constexpr bool mode_is_one_to_one(int mode)
+{
+    return mode == MW_CP_PACK_MW || mode == MW_CP_DELIVER_UC || mode == MW_CP_AG_PACK_MW || mode == MW_CP_AG_DELIVER_UC ||
+           mode == MW_CP_PAIR_FORWARD;
+}
+
+template <int V, int MODE>
+__global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constant__ mw_copy_args a)
+{
+    __shared__ uint8_t *dst_s[kRowsDstBatch];
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int tid = threadIdx.x;
+    // 32-bit on purpose: the division is on the way to the first load
+    const int row = blockIdx.x / a.chunks_per_row, piece = blockIdx.x % a.chunks_per_row;
+    // what decides whether the block has work is loaded together and looked at afterwards: one round trip
+    // (all of it lies inside the plan's arrays for any row below the launch bound)
+    const int status = (a.totals && a.rows_from != 0) ? a.totals->status : MW_OK;
+    const int64_t rows = n_rows(a);
+    const int nd = n_dst(a, row, MODE);
+    const int index = src_is_indexed(a, MODE) ? a.src_index[row] : 0;
+    if (status == MW_ERR_TIMEOUT || row >= rows) return;
+    const uint8_t *src = src_row_with(a, row, index, MODE);
+    const int64_t off = (int64_t)piece * a.chunk_bytes + tid * 16;      // vector k of this thread: off + k * blockDim.x * 16
+    const int64_t step = (int64_t)blockDim.x * 16;
+    uint4 v[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k)
+        if (off + k * step < a.row_bytes) v[k] = ld_stream(src + off + k * step);
+    if (mode_is_one_to_one(MODE)) {
+        uint8_t *d = dst_row(a, row, 0, MODE);
+        if (!d) return;
+#pragma unroll
+        for (int k = 0; k < V; ++k)
+            if (off + k * step < a.row_bytes) *(uint4 *)(d + off + k * step) = v[k];
+        return;
+    }
+    for (int qb = 0; qb < nd; qb += kRowsDstBatch) {
+        const int nq = min(kRowsDstBatch, nd - qb);
+        if (qb) __syncthreads();
+        if (tid < nq) dst_s[tid] = dst_row(a, row, qb + tid, MODE);
+        __syncthreads();
+        for (int q = 0; q < nq; ++q) {
+            uint8_t *d = dst_s[q];
+            if (!d) continue;
+#pragma unroll
+            for (int k = 0; k < V; ++k)
+                if (off + k * step < a.row_bytes) *(uint4 *)(d + off + k * step) = v[k];
+        }
+    }
+}
+
+// One instantiation per mode, so that the mode switches of the work list fold away.
+template <int V, int MODE>
+cudaError_t rows_launch(dim3 grid, dim3 block, cudaStream_t st, bool overlap, const mw_copy_args &a)
+{
+    return mw_launch(k_copy_rows<V, MODE>, grid, block, 0, st, overlap, a);
+}
+
 struct CopyShape { int warps; int stages; int64_t chunk; int batch; };
 
 // Rows longer than kMaxChunk are cut into equal pieces (multiples of 16 bytes); when that still leaves
@@ -626,13 +705,48 @@ int mw_copy_smem_setup(mw_ctx *ctx)
     return MW_OK;
 }
 
-// Chooses the work-item size and the pipeline shape, then launches a persistent grid.
+// Default: one block per (row, piece) on an ordinary grid.  With MW_FLAG_COPY_BULK / _REG_STORE / _LDST (or a grid
+// too large for 32-bit block indices): chooses the work-item size and the pipeline shape and launches a persistent grid.
 int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
 {
     const bool overlap = !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP);
     const int64_t est_rows = a.host_rows >= 0 ? a.host_rows : 0;
     cudaError_t err;
-    if (ctx->cfg.flags & MW_FLAG_COPY_LDST) {
+    const uint32_t other = MW_FLAG_COPY_LDST | MW_FLAG_COPY_REG_STORE | MW_FLAG_COPY_BULK;
+    int64_t pieces = 0;
+    int threads = 0;
+    // one-to-one copies need more loads in flight per thread; fan-out copies are bound by their stores
+    const int V = mode_is_one_to_one(a.mode) ? 2 : 1;
+    if (!(ctx->cfg.flags & other) && a.host_rows >= 0 && !a.loose_bound) {
+        // near-equal pieces of at most kRowsMaxVecs vectors; smaller ones while the grid would leave SMs idle
+        const int64_t vecs = a.row_bytes / 16;
+        pieces = (vecs + kRowsMaxVecs - 1) / kRowsMaxVecs;
+        while (a.host_rows * pieces < 4 * (int64_t)ctx->sm_count && (vecs + pieces - 1) / pieces > 128) pieces *= 2;
+        const int64_t piece_vecs = (vecs + pieces - 1) / pieces;
+        threads = (int)(((piece_vecs + V - 1) / V + 31) / 32 * 32);
+        if (threads < kRowsDstBatch) threads = kRowsDstBatch;
+        a.chunk_bytes = threads * V * 16;
+        pieces = (a.row_bytes + a.chunk_bytes - 1) / a.chunk_bytes;
+        a.chunks_per_row = (int32_t)pieces;
+    }
+    if (pieces > 0 && a.host_rows * pieces <= 0x7fffffff) {
+        if (a.host_rows == 0) return MW_OK;
+        const dim3 grid((unsigned)(a.host_rows * pieces));
+        const dim3 block(threads);
+        switch (a.mode) {
+        case MW_CP_PACK_MW: err = rows_launch<2, MW_CP_PACK_MW>(grid, block, st, overlap, a); break;
+        case MW_CP_SCATTER: err = rows_launch<1, MW_CP_SCATTER>(grid, block, st, overlap, a); break;
+        case MW_CP_DELIVER_UC: err = rows_launch<2, MW_CP_DELIVER_UC>(grid, block, st, overlap, a); break;
+        case MW_CP_AG_PACK_MW: err = rows_launch<2, MW_CP_AG_PACK_MW>(grid, block, st, overlap, a); break;
+        case MW_CP_AG_DELIVER_MW: err = rows_launch<1, MW_CP_AG_DELIVER_MW>(grid, block, st, overlap, a); break;
+        case MW_CP_AG_PACK_UC: err = rows_launch<1, MW_CP_AG_PACK_UC>(grid, block, st, overlap, a); break;
+        case MW_CP_AG_DELIVER_UC: err = rows_launch<2, MW_CP_AG_DELIVER_UC>(grid, block, st, overlap, a); break;
+        case MW_CP_PAIR_DIRECT: err = rows_launch<1, MW_CP_PAIR_DIRECT>(grid, block, st, overlap, a); break;
+        case MW_CP_PAIR_SEND: err = rows_launch<1, MW_CP_PAIR_SEND>(grid, block, st, overlap, a); break;
+        case MW_CP_PAIR_FORWARD: err = rows_launch<2, MW_CP_PAIR_FORWARD>(grid, block, st, overlap, a); break;
+        default: return MW_ERR_INVALID_ARG;
+        }
+    } else if (ctx->cfg.flags & MW_FLAG_COPY_LDST) {
         const int64_t chunk = choose_chunk(a.row_bytes, est_rows, (int64_t)ctx->sm_count * 2 * (kLdstThreads / 32));
         a.chunk_bytes = (int32_t)chunk;
         a.chunks_per_row = (int32_t)((a.row_bytes + chunk - 1) / chunk);

@@ -129,6 +129,7 @@ struct mw_copy_args {
     int stages;                // bulk-copy pipeline depth per warp
     int batch;                 // consecutive items claimed per work ticket
     int keep_in_l2;            // destination rows are read again soon: do not mark them evict-first
+    int loose_bound;           // host_rows may be far above the row count: take the persistent grid, which pays nothing for absent rows
     unsigned int *work_ctr;    // [2] ticket counter, finished-warp counter (both zero between launches)
     int Kd, R, dst_begin, dst_count;
     int pair_n, pair_copies;   // paired AllGather: ranks per domain, copies of the relayed segment on the pair link

@@ -233,6 +233,7 @@ int mw_relay_dispatch(mw_relay *relay, const void *x, void *send_buf, int64_t se
     a.dst_stride = recv_stride_bytes;
     a.capacity_rows = recv_capacity_rows;
     a.rows_from = 2;                                      // rows of the hop area = total_dest of the first-level plan
+    a.loose_bound = 1;                                    // T * Kd is far above the hop rows (70 % on the prefill shape)
     a.host_rows = (int64_t)hop->planned_T * hop->Kd;      // estimate for the chunking heuristic
     a.Kd = hop->Kd; a.R = hop->cfg.R;
     a.ndst = relay->s2_ndst;

@@ -11,10 +11,11 @@ from gpu_util import Guarded, SENTINEL, torch_mod
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
 @pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
 @pytest.mark.parametrize("R,S,direct", [(8, 64, 32), (8, 4112, 3072), (8, 64, 0), (8, 64, 64), (4, 48, 16), (2, 32, 16),
                                         (16, 160, 96), (8, 1 << 20, None), (8, 16 << 20, None), (80, 4096, 2048)])
-def test_paired_allgather_parity(layout, R, S, direct):
+def test_paired_allgather_parity(layout, R, S, direct, flags):
     torch = torch_mod()
     n = R // 2
     if direct is None:
@@ -25,7 +26,7 @@ def test_paired_allgather_parity(layout, R, S, direct):
     assert ret == 0
     sh_d = torch.from_numpy(sh).cuda()
     relay, recv = Guarded(max(len(want_relay), 16)), Guarded(len(want_recv))
-    with mw.Context(R, 8, 2, 16, 32) as ctx:
+    with mw.Context(R, 8, 2, 16, 32, flags=flags) as ctx:
         rc, tot = ctx.mw_paired_allgather(sh_d, S, direct, layout, relay.ptr(), recv.ptr())
         torch.cuda.synchronize()
     assert tot == want_tot

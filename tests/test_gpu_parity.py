@@ -29,12 +29,13 @@ def test_dispatch_parity_small_configurations_full_size(cfg):
     run_dispatch(wl.make_dispatch(cfg))
 
 
+@pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
 @pytest.mark.parametrize("cfg", [1, 2])
-def test_dispatch_parity_large_configurations_full_size(cfg):
+def test_dispatch_parity_large_configurations_full_size(cfg, flags):
     # full T and full hidden size, the shapes the benchmark times; compact MultiWrite + strided unicast
     inp = wl.make_dispatch(cfg)
-    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",))
-    run_dispatch(inp, layouts=(mw.MW_LAYOUT_UNICAST,), strides=("strided",))
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",), flags=flags)
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_UNICAST,), strides=("strided",), flags=flags)
 
 
 @pytest.mark.parametrize("cfg", [1, 2])
@@ -50,7 +51,7 @@ def test_register_copy_variant_matches(cfg):
 
 
 @pytest.mark.parametrize("flags", [mw.MW_FLAG_PLAN_MULTIPASS, mw.MW_FLAG_PLAN_COOPERATIVE, mw.MW_FLAG_NO_OVERLAP,
-                                   mw.MW_FLAG_COPY_REG_STORE,
+                                   mw.MW_FLAG_COPY_REG_STORE, mw.MW_FLAG_COPY_BULK,
                                    mw.MW_FLAG_PLAN_MULTIPASS | mw.MW_FLAG_COPY_LDST | mw.MW_FLAG_NO_OVERLAP])
 def test_launch_and_plan_variants_match(flags):
     """The multi-pass plan, the grid plan (ordinary and cooperative launch), the non-overlapped launches
@@ -322,12 +323,13 @@ def test_host_side_argument_errors():
 
 
 # ---- AllGather ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
 @pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
 @pytest.mark.parametrize("R,S,begin,count,strided", [
     (8, 48, 0, 8, False), (5, 4112, 1, 3, True), (64, 4096, 0, 64, False), (64, 16384, 0, 64, False),
     (64, 65536, 0, 64, True), (64, 1 << 18, 0, 64, False), (64, 1 << 20, 16, 16, False),
     (64, 4 << 20, 60, 4, False), (64, 16 << 20, 63, 1, False), (1, 64, 0, 1, False), (3, 16, 2, 0, False)])
-def test_allgather_parity(layout, R, S, begin, count, strided):
+def test_allgather_parity(layout, R, S, begin, count, strided, flags):
     torch = torch_mod()
     sh = wl.make_allgather_shards(R, S, seed=4)
     stride = R * S + 4096 if strided else 0
@@ -335,7 +337,7 @@ def test_allgather_parity(layout, R, S, begin, count, strided):
     assert ret == 0
     sh_d = torch.from_numpy(sh).cuda()
     send, recv = Guarded(len(want_send)), Guarded(max(len(want_recv), 16))
-    with mw.Context(R, 8, 2, 16, 32) as ctx:
+    with mw.Context(R, 8, 2, 16, 32, flags=flags) as ctx:
         rc, tot = ctx.mw_allgather_pack(sh_d, S, layout, send.ptr(), recv.ptr(), stride, begin, count)
         torch.cuda.synchronize()
     assert tot == want_tot
