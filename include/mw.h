@@ -195,7 +195,11 @@ MW_API int mw_pack(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64
 MW_API int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_base, int64_t recv_stride_bytes,
                int64_t recv_capacity_rows, void *stream);
 
-/* mw_pack followed by mw_deliver on the same stream: the whole data movement of one dispatch. */
+/*
+ * The whole data movement of one dispatch, with the results of mw_pack followed by mw_deliver (same send buffer,
+ * same receive regions, bit for bit) but in one pass: every hidden row is read once and written to its send
+ * slot(s) and to all its receive slots.  With a MW_FLAG_COPY_* bit set it is the two calls in sequence.
+ */
 MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows,
                 void *recv_base, int64_t recv_stride_bytes, int64_t recv_capacity_rows, void *stream);
 

@@ -254,9 +254,31 @@ int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t 
 {
     if (!ctx || !x || !send_buf || !recv_base) return MW_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
-    int rc = mw_pack(ctx, x, layout, send_buf, send_capacity_rows, stream);
-    if (rc != MW_OK) return rc;
-    return mw_deliver(ctx, layout, send_buf, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
+    if (ctx->cfg.flags & (MW_FLAG_COPY_BULK | MW_FLAG_COPY_REG_STORE | MW_FLAG_COPY_LDST)) {
+        int rc = mw_pack(ctx, x, layout, send_buf, send_capacity_rows, stream);
+        if (rc != MW_OK) return rc;
+        return mw_deliver(ctx, layout, send_buf, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
+    }
+    // one pass: every hidden row is read once and written to its send slot(s) and to all its receive slots
+    if (recv_stride_bytes < 0 || recv_capacity_rows < 0 || send_capacity_rows < 0 || check_layout(layout)) return MW_ERR_INVALID_ARG;
+    if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
+    if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
+    mw_copy_args a = base_args(ctx);
+    a.mode = layout == MW_LAYOUT_MULTIWRITE ? MW_CP_DISPATCH_MW : MW_CP_DISPATCH_UC;
+    a.src = (const uint8_t *)x;
+    a.src_index = ctx->d.mw_row_token;
+    a.dst = (uint8_t *)recv_base;
+    a.dst_stride = recv_stride_bytes;
+    a.capacity_rows = recv_capacity_rows;
+    a.dst2 = (uint8_t *)send_buf;
+    a.capacity2_rows = send_capacity_rows;
+    a.rows_from = 1;
+    a.host_rows = ctx->planned_T;
+    a.ndst = ctx->d.row_ndest;
+    a.d_rank = ctx->d.row_dest_rank;
+    a.d_pos = ctx->d.row_dest_pos;
+    a.d_flat = ctx->d.row_dest_flat;
+    return mw_copy_launch(ctx, a, as_stream(stream));
 }
 
 int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x,

@@ -114,7 +114,9 @@ __device__ __forceinline__ int64_t n_rows(const mw_copy_args &a)
 __device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t row, int mode)
 {
     switch (mode) {
-    case MW_CP_PACK_MW: return a.src + (int64_t)a.src_index[row] * a.row_bytes;
+    case MW_CP_PACK_MW:
+    case MW_CP_DISPATCH_MW:
+    case MW_CP_DISPATCH_UC: return a.src + (int64_t)a.src_index[row] * a.row_bytes;
     case MW_CP_SCATTER: return a.src + (a.src_index ? (int64_t)a.src_index[row] : row) * a.row_bytes;
     case MW_CP_AG_DELIVER_UC: {
         const int64_t i = row / a.dst_count, d = row % a.dst_count;
@@ -135,7 +137,7 @@ __device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t
 __device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t row) { return src_row(a, row, a.mode); }
 __device__ __forceinline__ bool src_is_indexed(const mw_copy_args &a, int mode)
 {
-    return mode == MW_CP_PACK_MW || (mode == MW_CP_SCATTER && a.src_index);
+    return mode == MW_CP_PACK_MW || mode == MW_CP_DISPATCH_MW || mode == MW_CP_DISPATCH_UC || (mode == MW_CP_SCATTER && a.src_index);
 }
 __device__ __forceinline__ bool src_is_indexed(const mw_copy_args &a) { return src_is_indexed(a, a.mode); }
 __device__ __forceinline__ const uint8_t *src_row_with(const mw_copy_args &a, int64_t row, int index, int mode)
@@ -151,6 +153,8 @@ __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row, int mod
 {
     switch (mode) {
     case MW_CP_SCATTER: return a.ndst[row];
+    case MW_CP_DISPATCH_MW: return a.ndst[row] + 1;
+    case MW_CP_DISPATCH_UC: return 2 * a.ndst[row];
     case MW_CP_AG_DELIVER_MW:
     case MW_CP_AG_PACK_UC: return a.dst_count;
     case MW_CP_PAIR_DIRECT: return a.pair_n;
@@ -161,6 +165,21 @@ __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row, int mod
 
 __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row) { return n_dst(a, row, a.mode); }
 
+// Receive slot of destination q of send row `row` (plan descriptors in plane layout).
+__device__ __forceinline__ uint8_t *scatter_dst(const mw_copy_args &a, int64_t row, int q)
+{
+    if (a.dst_stride) {
+        const int r = a.d_rank[q * a.d_stride + row], p = a.d_pos[q * a.d_stride + row];
+        if (r < 0) return nullptr;
+        if (p >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+        return a.dst + (int64_t)r * a.dst_stride + (int64_t)p * a.row_bytes;
+    }
+    const int64_t at = a.d_flat[q * a.d_stride + row];
+    if (at < 0) return nullptr;
+    if (at >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+    return a.dst + at * a.row_bytes;
+}
+
 // Destination q of a row; nullptr when the copy must not happen (capacity exceeded -> status, or the
 // AllGather copy addressed to the shard's own rank, which is never transmitted).
 __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, int q, int mode)
@@ -170,17 +189,19 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
     case MW_CP_AG_PACK_MW:
         if (row >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
         return a.dst + row * a.row_bytes;
-    case MW_CP_SCATTER: {
-        if (a.dst_stride) {
-            const int r = a.d_rank[q * a.d_stride + row], p = a.d_pos[q * a.d_stride + row];
-            if (r < 0) return nullptr;
-            if (p >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
-            return a.dst + (int64_t)r * a.dst_stride + (int64_t)p * a.row_bytes;
-        }
+    case MW_CP_SCATTER: return scatter_dst(a, row, q);
+    case MW_CP_DISPATCH_MW:
+        if (q > 0) return scatter_dst(a, row, q - 1);
+        if (row >= a.capacity2_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+        return a.dst2 + row * a.row_bytes;
+    case MW_CP_DISPATCH_UC: {
+        // the unicast send buffer is laid out like the compact receive area: slot = d_flat
+        const int n0 = a.ndst[row];
+        if (q >= n0) return scatter_dst(a, row, q - n0);
         const int64_t at = a.d_flat[q * a.d_stride + row];
         if (at < 0) return nullptr;
-        if (at >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
-        return a.dst + at * a.row_bytes;
+        if (at >= a.capacity2_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+        return a.dst2 + at * a.row_bytes;
     }
     case MW_CP_DELIVER_UC: {
         if (!a.dst_stride) {
@@ -628,25 +649,25 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
 #pragma unroll
     for (int k = 0; k < V; ++k)
         if (off + k * step < a.row_bytes) v[k] = ld_stream(src + off + k * step);
-    if (mode_is_one_to_one(MODE)) {
+    if constexpr (mode_is_one_to_one(MODE)) {
         uint8_t *d = dst_row(a, row, 0, MODE);
         if (!d) return;
 #pragma unroll
         for (int k = 0; k < V; ++k)
             if (off + k * step < a.row_bytes) *(uint4 *)(d + off + k * step) = v[k];
-        return;
-    }
-    for (int qb = 0; qb < nd; qb += kRowsDstBatch) {
-        const int nq = min(kRowsDstBatch, nd - qb);
-        if (qb) __syncthreads();
-        if (tid < nq) dst_s[tid] = dst_row(a, row, qb + tid, MODE);
-        __syncthreads();
-        for (int q = 0; q < nq; ++q) {
-            uint8_t *d = dst_s[q];
-            if (!d) continue;
+    } else {
+        for (int qb = 0; qb < nd; qb += kRowsDstBatch) {
+            const int nq = min(kRowsDstBatch, nd - qb);
+            if (qb) __syncthreads();
+            if (tid < nq) dst_s[tid] = dst_row(a, row, qb + tid, MODE);
+            __syncthreads();
+            for (int q = 0; q < nq; ++q) {
+                uint8_t *d = dst_s[q];
+                if (!d) continue;
 #pragma unroll
-            for (int k = 0; k < V; ++k)
-                if (off + k * step < a.row_bytes) *(uint4 *)(d + off + k * step) = v[k];
+                for (int k = 0; k < V; ++k)
+                    if (off + k * step < a.row_bytes) *(uint4 *)(d + off + k * step) = v[k];
+            }
         }
     }
 }
@@ -744,6 +765,8 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_PAIR_DIRECT: err = rows_launch<1, MW_CP_PAIR_DIRECT>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_SEND: err = rows_launch<1, MW_CP_PAIR_SEND>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_FORWARD: err = rows_launch<2, MW_CP_PAIR_FORWARD>(grid, block, st, overlap, a); break;
+        case MW_CP_DISPATCH_MW: err = rows_launch<1, MW_CP_DISPATCH_MW>(grid, block, st, overlap, a); break;
+        case MW_CP_DISPATCH_UC: err = rows_launch<1, MW_CP_DISPATCH_UC>(grid, block, st, overlap, a); break;
         default: return MW_ERR_INVALID_ARG;
         }
     } else if (ctx->cfg.flags & MW_FLAG_COPY_LDST) {

@@ -110,7 +110,9 @@ enum mw_copy_mode {
     MW_CP_AG_DELIVER_UC = 6,// region(d)[i] = send[i][d] (own shard: taken from shards)
     MW_CP_PAIR_DIRECT = 7,  // paired AllGather: direct segment of shard r to every member of r's domain
     MW_CP_PAIR_SEND = 8,    // relayed segment of shard r to its partner's relay area (and to r itself)
-    MW_CP_PAIR_FORWARD = 9  // partner forwards the relayed segment to the other members of r's domain
+    MW_CP_PAIR_FORWARD = 9, // partner forwards the relayed segment to the other members of r's domain
+    MW_CP_DISPATCH_MW = 10, // pack and deliver in one pass: x[mw_row_token[j]] -> send[j] and every destination of row j
+    MW_CP_DISPATCH_UC = 11  // x[mw_row_token[j]] -> its unicast send slots and every destination of row j
 };
 
 struct mw_copy_args {
@@ -118,10 +120,12 @@ struct mw_copy_args {
     const uint8_t *src;        // source rows (x, send buffer or shards)
     const uint8_t *src2;       // AllGather unicast deliver: the shards (own copy is local)
     uint8_t *dst;              // destination base
-    uint8_t *dst2;             // paired AllGather, relayed segment: the receive area (own copy), dst being the relay area
+    uint8_t *dst2;             // paired AllGather, relayed segment: the receive area (own copy), dst being the relay area;
+                               // fused dispatch: the send buffer
     int64_t row_bytes;         // bytes per row (B, or the shard size)
     int64_t dst_stride;        // bytes between receive regions; 0 = compact
     int64_t capacity_rows;     // rows the destination may hold (per region when strided)
+    int64_t capacity2_rows;    // fused dispatch: rows the send buffer (dst2) may hold
     int64_t host_rows;         // row count known on the host (-1: read from totals)
     int rows_from;             // 0: host_rows, 1: totals->T_nonempty, 2: totals->total_dest
     int32_t chunk_bytes;       // bytes moved per work item (multiple of 16)

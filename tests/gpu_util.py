@@ -57,7 +57,7 @@ def assert_plan_equal(got: dict, p: mwo.Plan, totals: dict):
 
 def run_dispatch(inp, *, layouts=(mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST), strides=("compact", "strided"),
                  flags: int = 0, src_rank: int = -1, max_tokens: int | None = None, check_payload: bool = True,
-                 repeats: int = 1, one_call: bool = False):
+                 repeats: int = 1, one_call: bool = False, separate: bool = False):
     """Plans and dispatches `inp` on the GPU, checks everything against the oracle, returns (plan, totals)."""
     torch = torch_mod()
     s = inp.shape
@@ -92,6 +92,11 @@ def run_dispatch(inp, *, layouts=(mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST)
                     ctx.mw_plan_dispatch(ids_d, e2r_d, T, x_d.data_ptr(), layout, send.ptr(), nsend, recv.ptr(), stride, cap)
                     tot2 = ctx.mw_get_totals()
                     assert_plan_equal(ctx.plan_arrays(T), p, tot2)
+                elif separate:
+                    # the two steps as calls of their own (mw_dispatch does both in one pass over the rows)
+                    ctx.mw_pack(x_d.data_ptr(), layout, send.ptr(), nsend)
+                    ctx.mw_deliver(layout, send.ptr(), recv.ptr(), stride, cap)
+                    tot2 = ctx.mw_get_totals()
                 else:
                     ctx.mw_dispatch(x_d.data_ptr(), layout, send.ptr(), nsend, recv.ptr(), stride, cap)
                     tot2 = ctx.mw_get_totals()

@@ -24,24 +24,26 @@ def test_plan_parity_full_configurations(cfg, seed):
     run_dispatch(inp, check_payload=False, repeats=2)
 
 
+@pytest.mark.parametrize("separate", [False, True])
 @pytest.mark.parametrize("cfg", [0, 3])
-def test_dispatch_parity_small_configurations_full_size(cfg):
-    run_dispatch(wl.make_dispatch(cfg))
+def test_dispatch_parity_small_configurations_full_size(cfg, separate):
+    run_dispatch(wl.make_dispatch(cfg), separate=separate)
 
 
-@pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
+@pytest.mark.parametrize("flags,separate", [(0, False), (0, True), (mw.MW_FLAG_COPY_BULK, False)])
 @pytest.mark.parametrize("cfg", [1, 2])
-def test_dispatch_parity_large_configurations_full_size(cfg, flags):
+def test_dispatch_parity_large_configurations_full_size(cfg, flags, separate):
     # full T and full hidden size, the shapes the benchmark times; compact MultiWrite + strided unicast
     inp = wl.make_dispatch(cfg)
-    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",), flags=flags)
-    run_dispatch(inp, layouts=(mw.MW_LAYOUT_UNICAST,), strides=("strided",), flags=flags)
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",), flags=flags, separate=separate)
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_UNICAST,), strides=("strided",), flags=flags, separate=separate)
 
 
+@pytest.mark.parametrize("separate", [False, True])
 @pytest.mark.parametrize("cfg", [1, 2])
 @pytest.mark.parametrize("seed", [100, 101])
-def test_dispatch_parity_large_configurations_reduced_hidden(cfg, seed):
-    run_dispatch(wl.make_dispatch(cfg, seed, H=264))          # 528-byte rows: ragged against every tile size
+def test_dispatch_parity_large_configurations_reduced_hidden(cfg, seed, separate):
+    run_dispatch(wl.make_dispatch(cfg, seed, H=264), separate=separate)          # 528-byte rows: ragged against every tile size
 
 
 @pytest.mark.parametrize("cfg", [0, 1])
@@ -75,10 +77,11 @@ def test_rank_word_boundaries(R):
     run_dispatch(inp)
 
 
+@pytest.mark.parametrize("separate", [False, True])
 @pytest.mark.parametrize("T", [0, 1, 31, 255, 256, 257, 1000, 1025])
-def test_token_counts_around_tile_edges(T):
+def test_token_counts_around_tile_edges(T, separate):
     inp = wl.make_random_dispatch(T + 3, T=T, K=3, E=40, R=10, H=40)
-    run_dispatch(inp, max_tokens=1100)
+    run_dispatch(inp, max_tokens=1100, separate=separate)
 
 
 def test_top1_and_few_large_groups():
