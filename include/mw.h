@@ -64,7 +64,8 @@ extern "C" {
 #define MW_ERR_CAPACITY     (-3)  /* a buffer cannot hold the rows the plan assigns to it     */
 #define MW_ERR_CUDA         (-4)  /* a CUDA runtime call failed                               */
 #define MW_ERR_BAD_INDEX    (-5)  /* expert id or expert->rank entry out of range (ignored)   */
-#define MW_ERR_TIMEOUT      (-6)  /* a bounded device-side wait gave up; the plan is invalid  */
+#define MW_ERR_TIMEOUT      (-6)  /* a bounded device-side wait gave up; the plan is invalid; */
+                                  /* destroy the context (its counters may be out of step)    */
 #define MW_ERR_NO_PLAN      (-7)  /* dispatch called before any plan                          */
 
 #define MW_LAYOUT_MULTIWRITE 0    /* send buffer holds each row once (one row per group member) */
