@@ -549,3 +549,103 @@ void mwo_combine(const uint8_t *z_base, int64_t z_stride_bytes, const float *wei
         }
     }
 }
+
+/*
+ * Group-major receive order (Section 4.3.1: one MultiWrite writes ONE source buffer B_S into ONE target buffer
+ * B_i at every destination D_i; Section 4.3.2: the call takes an array of remote buffer addresses).
+ * With the receive region of rank r laid out group by group (groups in id order, members in token order), the
+ * group g is exactly one such call: B_S = send_mw[group_offsets[g] .. +size), B_i = region(D_i)[start .. +size)
+ * with start = group_dest_offset[g][i].
+ *
+ *   group_dest_rank   [G, Kd]  destination ranks of group g, ascending, -1 padded
+ *   group_dest_offset [G, Kd]  first slot of the group's block inside the region of that rank, -1 padded
+ *   dest_pos_gm       [T, Kd]  slot of token t in the region of its i-th destination rank, -1 padded
+ * Rows of the three arrays beyond G (or T) are not touched.  Region sizes are those of the plan (rank_offsets).
+ */
+void mwo_group_major(int32_t T, int32_t R, int32_t K, int64_t G, const uint64_t *group_mask, const int32_t *group_offsets,
+                     const int32_t *token_group, const int32_t *token_mw_row,
+                     int32_t *group_dest_rank, int32_t *group_dest_offset, int32_t *dest_pos_gm)
+{
+    const int W = mwo_words(R);
+    const int Kd = K < R ? K : R;
+    int32_t *filled = (int32_t *)calloc((size_t)R, sizeof(int32_t));      /* slots used so far in each region */
+    if (!filled) return;
+    for (int64_t g = 0; g < G; ++g) {
+        const int32_t size = group_offsets[g + 1] - group_offsets[g];
+        int i = 0;
+        for (int32_t r = 0; r < R; ++r) {
+            if (!(group_mask[g * W + r / 64] >> (r % 64) & 1)) continue;
+            group_dest_rank[g * Kd + i] = r;
+            group_dest_offset[g * Kd + i] = filled[r];
+            filled[r] += size;
+            ++i;
+        }
+        for (; i < Kd; ++i) { group_dest_rank[g * Kd + i] = -1; group_dest_offset[g * Kd + i] = -1; }
+    }
+    free(filled);
+    for (int32_t t = 0; t < T; ++t) {
+        const int32_t g = token_group[t];
+        for (int i = 0; i < Kd; ++i) {
+            if (g < 0 || group_dest_rank[(int64_t)g * Kd + i] < 0) { dest_pos_gm[(int64_t)t * Kd + i] = -1; continue; }
+            const int32_t within = token_mw_row[t] - group_offsets[g];
+            dest_pos_gm[(int64_t)t * Kd + i] = group_dest_offset[(int64_t)g * Kd + i] + within;
+        }
+    }
+}
+
+/* One MultiWrite per group: the group's slice of the send buffer goes, as one block, to every destination. */
+void mwo_deliver_group_major(const uint8_t *send_mw, int64_t row_bytes, int32_t R, int32_t K, int64_t G,
+                             const int32_t *group_offsets, const int32_t *group_dest_rank, const int32_t *group_dest_offset,
+                             const int32_t *rank_offsets, uint8_t *recv_base, int64_t recv_stride_bytes)
+{
+    const int Kd = K < R ? K : R;
+    for (int64_t g = 0; g < G; ++g) {
+        const int64_t size = group_offsets[g + 1] - group_offsets[g];
+        const uint8_t *b_s = send_mw + (int64_t)group_offsets[g] * row_bytes;
+        for (int i = 0; i < Kd; ++i) {
+            const int32_t r = group_dest_rank[g * Kd + i];
+            if (r < 0) continue;
+            uint8_t *b_i = region(recv_base, recv_stride_bytes, rank_offsets, r, row_bytes) +
+                           (int64_t)group_dest_offset[g * Kd + i] * row_bytes;
+            memcpy(b_i, b_s, (size_t)(size * row_bytes));
+        }
+    }
+}
+
+/*
+ * Expert index of the receive regions (Section 2.3.2: a token goes to the nodes that host its selected experts;
+ * on arrival each local expert must find its tokens).  A row is stored once per rank, so a token chosen by two
+ * experts of one rank cannot sit in two places: the region keeps its order and every expert gets a list instead.
+ *
+ *   expert_offsets [E + 1]  exclusive prefix sum of the number of distinct tokens that selected expert e
+ *                           (experts whose table entry is outside [0, R) count nothing)
+ *   expert_token   [T * K]  for each expert in id order, its tokens in ascending order; -1 beyond the total
+ *   expert_slot    [T * K]  the slot of that token inside the region of the expert's rank (token-major order)
+ * Returns the total number of (token, expert) pairs.
+ */
+int64_t mwo_expert_index(const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, int32_t K, int32_t E, int32_t R,
+                         const int32_t *dest_rank, const int32_t *dest_pos,
+                         int32_t *expert_offsets, int32_t *expert_token, int32_t *expert_slot)
+{
+    const int Kd = K < R ? K : R;
+    int64_t P = 0;
+    for (int32_t e = 0; e < E; ++e) {
+        expert_offsets[e] = (int32_t)P;
+        const int32_t r = expert_to_rank[e];
+        if (r < 0 || r >= R) continue;
+        for (int32_t t = 0; t < T; ++t) {
+            int hit = 0;
+            for (int32_t k = 0; k < K; ++k) hit |= (topk_ids[(int64_t)t * K + k] == e);
+            if (!hit) continue;
+            int32_t slot = -1;
+            for (int i = 0; i < Kd; ++i)
+                if (dest_rank[(int64_t)t * Kd + i] == r) slot = dest_pos[(int64_t)t * Kd + i];
+            expert_token[P] = t;
+            expert_slot[P] = slot;
+            ++P;
+        }
+    }
+    expert_offsets[E] = (int32_t)P;
+    for (int64_t i = P; i < (int64_t)T * K; ++i) { expert_token[i] = -1; expert_slot[i] = -1; }
+    return P;
+}

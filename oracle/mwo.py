@@ -220,6 +220,47 @@ def combine(p: Plan, z: np.ndarray, weights: np.ndarray | None = None, z_stride_
     return y
 
 
+def group_major(p: Plan):
+    """Group-major receive order.  Returns (group_dest_rank [G,Kd], group_dest_offset [G,Kd], dest_pos_gm [T,Kd])."""
+    G, Kd = int(p.totals["G"]), p.Kd
+    gdr = np.full((max(G, 1), Kd), -1, np.int32)
+    gdo = np.full((max(G, 1), Kd), -1, np.int32)
+    gm = np.full((max(p.T, 1), Kd), -1, np.int32)
+    lib().mwo_group_major.restype = None
+    lib().mwo_group_major(C.c_int32(p.T), C.c_int32(p.R), C.c_int32(p.K), C.c_int64(G), _p(p.group_mask), _p(p.group_offsets),
+                          _p(p.token_group), _p(p.token_mw_row), _p(gdr), _p(gdo), _p(gm))
+    return gdr[:G], gdo[:G], gm[:p.T]
+
+
+def deliver_group_major(p: Plan, send_mw: np.ndarray, gdr: np.ndarray, gdo: np.ndarray, recv_stride_bytes: int = 0,
+                        fill: int = 0) -> np.ndarray:
+    """Receive area (uint8, flat) after one MultiWrite per group, regions in group-major order."""
+    recv = np.full(recv_bytes_needed(p, recv_stride_bytes), fill, np.uint8)
+    G = int(p.totals["G"])
+    if G == 0:
+        return recv
+    send = np.ascontiguousarray(send_mw).view(np.uint8).reshape(-1)
+    a, b = np.ascontiguousarray(gdr, dtype=np.int32), np.ascontiguousarray(gdo, dtype=np.int32)
+    lib().mwo_deliver_group_major.restype = None
+    lib().mwo_deliver_group_major(_p(send), C.c_int64(p.row_bytes), C.c_int32(p.R), C.c_int32(p.K), C.c_int64(G),
+                                  _p(p.group_offsets), _p(a), _p(b), _p(p.rank_offsets), _p(recv), C.c_int64(recv_stride_bytes))
+    return recv
+
+
+def expert_index(p: Plan, topk_ids: np.ndarray, expert_to_rank: np.ndarray):
+    """Returns (expert_offsets [E+1], expert_token [T*K], expert_slot [T*K], pairs)."""
+    ids = np.ascontiguousarray(topk_ids, dtype=np.int32).reshape(p.T, p.K)
+    e2r = np.ascontiguousarray(expert_to_rank, dtype=np.int32)
+    E = len(e2r)
+    off = np.zeros(E + 1, np.int32)
+    tok = np.full(max(p.T * p.K, 1), -1, np.int32)
+    slot = np.full(max(p.T * p.K, 1), -1, np.int32)
+    lib().mwo_expert_index.restype = C.c_int64
+    n = lib().mwo_expert_index(_p(ids), _p(e2r), C.c_int32(p.T), C.c_int32(p.K), C.c_int32(E), C.c_int32(p.R),
+                               _p(p.dest_rank), _p(p.dest_pos), _p(off), _p(tok), _p(slot))
+    return off, tok[:p.T * p.K], slot[:p.T * p.K], int(n)
+
+
 class PairTotals(C.Structure):
     _fields_ = [("direct_link_bytes", C.c_int64), ("pair_link_bytes", C.c_int64), ("forward_link_bytes", C.c_int64),
                 ("max_link_bytes", C.c_int64), ("total_bytes", C.c_int64)]

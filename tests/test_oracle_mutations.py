@@ -7,6 +7,7 @@ import subprocess
 import pytest
 
 import test_oracle_combine_pins as cpins
+import test_oracle_order_pins as opins
 import test_oracle_pair_pins as ppins
 import test_oracle_pins as pins
 import test_oracle_relay_pins as rpins
@@ -16,6 +17,16 @@ from paper_2605_22428_b200 import workloads as wl
 SRC = os.path.join(os.path.dirname(mwo.__file__), "mwo.c")
 
 MUTATIONS = {
+    "group-major blocks advance by one row": ("filled[r] += size;", "filled[r] += 1;"),
+    "group-major ignores the position inside the group": ("group_dest_offset[(int64_t)g * Kd + i] + within;", "group_dest_offset[(int64_t)g * Kd + i];"),
+    "group-major block copied from the start of the send buffer": ("const uint8_t *b_s = send_mw + (int64_t)group_offsets[g] * row_bytes;",
+                                                                   "const uint8_t *b_s = send_mw;"),
+    "expert index looks at the first slot only": ("for (int32_t k = 0; k < K; ++k) hit |= (topk_ids[(int64_t)t * K + k] == e);",
+                                                  "hit = (topk_ids[(int64_t)t * K] == e);"),
+    "expert index takes the slot of the first destination": ("if (dest_rank[(int64_t)t * Kd + i] == r) slot = dest_pos[(int64_t)t * Kd + i];",
+                                                             "if (i == 0) slot = dest_pos[(int64_t)t * Kd + i];"),
+    "expert index counts experts with a bad table entry": ("        if (r < 0 || r >= R) continue;\n        for (int32_t t = 0; t < T; ++t) {\n            int hit = 0;",
+                                                           "        for (int32_t t = 0; t < T; ++t) {\n            int hit = 0;"),
     "combine ignores the weights": ("acc += w * bf16_to_double(", "acc += bf16_to_double("),
     "combine truncates instead of rounding": ("double q = nearbyint(ldexp(a, 7 - ex));", "double q = floor(ldexp(a, 7 - ex));"),
     "combine reads the wrong slot": ("(int64_t)dest_pos[(int64_t)t * Kd + i] * row_bytes;\n                const double w",
@@ -68,6 +79,10 @@ def run_pins():
     rpins.test_paper_example_four_local_four_remote()
     rpins.test_relay_brute_force(1, 12, 3, 7, 24, 4)
     ppins.test_every_rank_gets_its_domain_in_order(0, 8, 64, 32)
+    opins.test_group_major_brute_force(1, 8, 32, 4, 0.2)
+    opins.test_group_major_with_few_large_groups()
+    opins.test_expert_index_brute_force(1, 8, 32, 4, 0.2, True)
+    opins.test_expert_index_ignores_invalid_table_entries_and_ids()
 
 
 def test_unmutated_oracle_passes_the_subset():
@@ -86,6 +101,7 @@ def test_planted_mistake_is_caught(name, tmp_path, monkeypatch):
     lib = ctypes.CDLL(str(lib_path))
     lib.mwo_plan.restype = ctypes.c_int
     lib.mwo_allgather.restype = ctypes.c_int
+    lib.mwo_expert_index.restype = ctypes.c_int64
     for fn in ("mwo_pack_mw", "mwo_pack_uc", "mwo_deliver_mw", "mwo_deliver_uc", "mwo_deliver_definition"):
         getattr(lib, fn).restype = None
     monkeypatch.setattr(mwo, "_lib", lib)
