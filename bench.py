@@ -387,6 +387,44 @@ def fused_dispatch_measure(mw, wl, torch) -> dict:
     return out
 
 
+def order_measure(mw, wl, torch) -> dict:
+    """Group-major receive order (Sections 4.3.1, 4.3.2) and expert index (Section 2.3.2) on the headline workload."""
+    inp = wl.make_dispatch(WORKLOAD, payload=False)
+    s = inp.shape
+    B, T = s.row_bytes, s.T
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+        ctx.mw_plan(ids, e2r, T)
+        tot = ctx.mw_get_totals()
+        Tn, SD = tot["T_nonempty"], tot["total_dest"]
+        ctx.mw_group_major()
+        sends = [torch.empty(Tn * B, dtype=torch.uint8, device="cuda").random_(0, 256) for _ in range(2)]
+        recvs = [torch.empty(SD * B, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        off = torch.empty(s.E + 1, dtype=torch.int32, device="cuda")
+        tok = torch.empty(T * s.K, dtype=torch.int32, device="cuda")
+        slot = torch.empty(T * s.K, dtype=torch.int32, device="cuda")
+        cases = (("group_major_arrays_us", lambda i: ctx.mw_group_major(), 200),
+                 ("deliver_group_major_us", lambda i: ctx.mw_deliver_group_major(sends[i % 2], recvs[i % 2], 0, SD), 100),
+                 ("expert_index_us", lambda i: ctx.mw_expert_index(ids, e2r, off, tok, slot), 200))
+        out = {}
+        for name, fn, n in cases:
+            for i in range(5):
+                fn(i)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(n):
+                fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            out[name] = round(a.elapsed_time(b) * 1e3 / n, 1)
+        assert ctx.mw_get_totals()["status"] == 0
+    out["deliver_group_major_gbs"] = round((Tn + SD) * B / out["deliver_group_major_us"] / 1e3, 1)
+    out["groups"] = tot["G"]
+    out["note"] = "4 + 3 short kernels over the plan (latency-bound); the deliver is the same row-copy kernel with other slots"
+    return out
+
+
 def combine_measure(mw, wl, torch) -> dict:
     """Combine (Section 2.3.2) on the dsv3_prefill routing: every destination returns one bf16 row per token."""
     inp = wl.make_dispatch(WORKLOAD, payload=False)
@@ -632,6 +670,7 @@ def run_cuda(args):
             line["paired_allgather_8x16MB"] = paired_allgather_measure(mw, torch)
             line["combine_dsv3_prefill"] = combine_measure(mw, wl, torch)
             line["dispatch_fused"] = fused_dispatch_measure(mw, wl, torch)
+            line["receiver_order"] = order_measure(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:

@@ -251,6 +251,51 @@ MW_API int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_byte
 MW_API int mw_combine(mw_ctx *ctx, const void *z_base, int64_t z_stride_bytes, const float *weights, void *y, void *stream);
 
 /*
+ * Group-major receive order.  Section 4.3.1 defines MultiWrite(S, M, B_S) as writing ONE source buffer B_S into
+ * ONE target buffer B_i at every destination D_i, and Section 4.3.2 gives the call an array of remote buffer
+ * addresses.  With the region of every rank laid out group by group (groups in id order, members in ascending
+ * token order) each group of the latest plan is exactly one such call:
+ *     B_S = send buffer rows [group_offsets[g], group_offsets[g + 1])      (MultiWrite layout)
+ *     D_i = group_dest_rank[g][i],   B_i = region(D_i) rows [group_dest_offset[g][i], + size of the group)
+ * mw_group_major derives these arrays from the latest plan (region sizes and rank_offsets are unchanged; only
+ * the order of the rows inside a region differs from mw_deliver's token-major order):
+ *     group_dest_rank    device int32 [max_tokens, Kd]   first G rows defined, -1 padded
+ *     group_dest_offset  device int32 [max_tokens, Kd]   first G rows defined, -1 padded
+ *     dest_pos_gm        device int32 [max_tokens, Kd]   first T rows: slot of token t at its i-th destination
+ * The arrays belong to the context and are overwritten by the next mw_group_major.  view (host, optional)
+ * receives their addresses.  mw_deliver_group_major expands the MultiWrite-layout send buffer into regions in
+ * that order (arguments as mw_deliver); it needs mw_group_major to have run after the latest plan
+ * (else MW_ERR_NO_PLAN).
+ */
+typedef struct mw_group_major_view {
+    int32_t *group_dest_rank;
+    int32_t *group_dest_offset;
+    int32_t *dest_pos_gm;
+    int32_t  Kd;
+    int32_t  reserved;
+} mw_group_major_view;
+
+MW_API int mw_group_major(mw_ctx *ctx, mw_group_major_view *view, void *stream);
+MW_API int mw_deliver_group_major(mw_ctx *ctx, const void *send_buf, void *recv_base, int64_t recv_stride_bytes,
+                           int64_t recv_capacity_rows, void *stream);
+
+/*
+ * Expert index of the receive regions (Section 2.3.2: a token is sent to the nodes that host its selected
+ * experts; each local expert then has to find its tokens).  A row is stored once per rank, so the regions keep
+ * their order and every expert gets a list.  Uses the latest plan; topk_ids / expert_to_rank must be the arrays
+ * that plan was made from.
+ *     expert_offsets  device int32 [E + 1]  exclusive prefix sum of the number of distinct tokens that selected
+ *                                           expert e (experts whose table entry is outside [0, R) count nothing)
+ *     expert_token    device int32 [T * K]  per expert in id order, its tokens ascending; -1 beyond the total
+ *     expert_slot     device int32 [T * K]  slot of that token in the region of the expert's rank (token-major
+ *                                           order, i.e. the order mw_deliver and mw_dispatch produce)
+ * MW_ERR_CAPACITY when E is too large for the kernel's shared-memory bit matrix (32 bytes per expert) or for
+ * the per-tile count table (max_tokens / 256 x E entries, at most 256 MB).
+ */
+MW_API int mw_expert_index(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t *expert_offsets,
+                    int32_t *expert_token, int32_t *expert_slot, void *stream);
+
+/*
  * Paired-relay AllGather with segment split (Section 3.1 "paired relaying", Section 5.2): cfg.R = 2n
  * ranks on a full mesh form two domains, [0, n) and [n, 2n); rank r is paired with (r + n) mod 2n.
  * Each domain gathers its own n shards: afterwards the receive region of every rank holds the shards

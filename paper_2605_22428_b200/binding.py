@@ -34,7 +34,8 @@ MW_FLAG_COPY_BULK = 0x40
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
 EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
-           "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
+           "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_group_major", "mw_deliver_group_major", "mw_expert_index",
+           "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
            "mw_strerror", "mw_pair_balanced_direct_bytes") + RELAY_EXPORTS
 
 
@@ -69,6 +70,11 @@ class mw_pair_totals(C.Structure):
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+class mw_group_major_view(C.Structure):
+    _fields_ = [("group_dest_rank", C.c_void_p), ("group_dest_offset", C.c_void_p), ("dest_pos_gm", C.c_void_p),
+                ("Kd", C.c_int32), ("reserved", C.c_int32)]
 
 
 class mw_plan_view(C.Structure):
@@ -116,6 +122,9 @@ def lib():
         L.mw_pair_balanced_direct_bytes.argtypes = [i64, i32, C.c_int]
         L.mw_pair_balanced_direct_bytes.restype = i64
         L.mw_combine.argtypes = [vp, vp, i64, vp, vp, vp]
+        L.mw_group_major.argtypes = [vp, C.POINTER(mw_group_major_view), vp]
+        L.mw_deliver_group_major.argtypes = [vp, vp, vp, i64, i64, vp]
+        L.mw_expert_index.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.mw_dispatch_host.argtypes = [vp, vp, vp, vp, i32, C.c_int, vp, i64, vp, C.POINTER(mw_totals), vp]
         L.mw_group_tokens_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.mw_read_device.argtypes = [vp, vp, vp, i64, vp]
@@ -131,7 +140,7 @@ def lib():
             getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:15]:
+        for name in EXPORTS[:18]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -300,6 +309,44 @@ class Context:
         rc = lib().mw_combine(self._h, _ptr(z), z_stride_bytes, _ptr(weights), _ptr(y), _stream(stream))
         if check and rc != MW_OK:
             raise MwError(rc, "mw_combine")
+        return rc
+
+    def mw_group_major(self, stream=None, check: bool = True):
+        """Returns (rc, view); the view's fields are device addresses of context-owned arrays."""
+        view = mw_group_major_view()
+        rc = lib().mw_group_major(self._h, C.byref(view), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_group_major")
+        return rc, view
+
+    def group_major_arrays(self, T: int, G: int, view) -> dict:
+        """Host copies (numpy) of the arrays mw_group_major filled: first G groups, first T tokens."""
+        import numpy as np
+        Kd = view.Kd
+        out = {}
+        for name, rows in (("group_dest_rank", G), ("group_dest_offset", G), ("dest_pos_gm", T)):
+            a = np.empty((rows, Kd), np.int32)
+            if rows:
+                rc = lib().mw_read_device(self._h, _ptr(a), C.c_void_p(getattr(view, name)), a.nbytes, None)
+                if rc != MW_OK:
+                    raise MwError(rc, "mw_read_device")
+            out[name] = a
+        return out
+
+    def mw_deliver_group_major(self, send_buf, recv_base, recv_stride_bytes: int, recv_capacity_rows: int, stream=None,
+                               check: bool = True) -> int:
+        rc = lib().mw_deliver_group_major(self._h, _ptr(send_buf), _ptr(recv_base), recv_stride_bytes, recv_capacity_rows,
+                                          _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_deliver_group_major")
+        return rc
+
+    def mw_expert_index(self, topk_ids, expert_to_rank, expert_offsets, expert_token, expert_slot, stream=None,
+                        check: bool = True) -> int:
+        rc = lib().mw_expert_index(self._h, _ptr(topk_ids), _ptr(expert_to_rank), _ptr(expert_offsets), _ptr(expert_token),
+                                   _ptr(expert_slot), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_expert_index")
         return rc
 
     def mw_dispatch_host(self, topk_ids_host, expert_to_rank_host, x_host, T: int, layout: int, recv_host,

@@ -9,7 +9,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB_DIR = os.path.join(_PKG, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libmw.so")
-SOURCES = ("mw_api.cu", "mw_plan.cu", "mw_copy.cu", "mw_small.cu", "mw_relay.cu", "mw_combine.cu", "mw_static.cu")
+SOURCES = ("mw_api.cu", "mw_plan.cu", "mw_copy.cu", "mw_small.cu", "mw_relay.cu", "mw_combine.cu", "mw_order.cu", "mw_static.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-shared"]
 

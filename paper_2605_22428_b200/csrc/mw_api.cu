@@ -49,6 +49,16 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.row_dest_rank = k.take<int32_t>(Tm * Kd);
     d.row_dest_pos = k.take<int32_t>(Tm * Kd);
     d.row_dest_flat = k.take<int32_t>(Tm * Kd);
+    d.gm_rank = k.take<int32_t>(Tm * Kd);
+    d.gm_offset = k.take<int32_t>(Tm * Kd);
+    d.dest_pos_gm = k.take<int32_t>(Tm * Kd);
+    d.row_dest_pos_gm = k.take<int32_t>(Tm * Kd);
+    d.row_dest_flat_gm = k.take<int32_t>(Tm * Kd);
+    d.gm_tile_sum = k.take<int32_t>((size_t)c->max_tiles * R);
+    {
+        const size_t n = (size_t)c->max_tiles * (size_t)c->cfg.E;     // beyond 256 MB the expert index is not offered
+        d.ex_tile_cnt = n * sizeof(int32_t) <= ((size_t)256 << 20) ? k.take<int32_t>(n) : nullptr;
+    }
     d.slot_key = k.take<unsigned long long>((size_t)c->HS);
     d.slot_leader = k.take<int32_t>((size_t)c->HS);
     d.slot_count = k.take<int32_t>((size_t)c->HS);
@@ -140,6 +150,7 @@ int mw_create(mw_ctx **out, const mw_config *cfg)
     if (rc == MW_OK) rc = mw_plan_smem_setup(c);
     if (rc == MW_OK) rc = mw_copy_smem_setup(c);
     if (rc == MW_OK) rc = mw_small_setup(c);
+    if (rc == MW_OK) rc = mw_order_smem_setup(c);
     if (rc != MW_OK) { cudaFree(c->slab); cudaGetLastError(); delete c; return rc; }
     *out = c;
     return MW_OK;

@@ -35,6 +35,13 @@ struct mw_dev {
     int32_t *row_dest_rank;  // [Kd, Tm]  destination ranks of send row j (entry i of row j at i * Tm + j)
     int32_t *row_dest_pos;   // [Kd, Tm]  slots of send row j
     int32_t *row_dest_flat;  // [Kd, Tm]  row of the compact receive area for each destination of send row j, -1 pad
+    // group-major receive order (mw_order.cu)
+    int32_t *gm_rank, *gm_offset;   // [Tm, Kd] destination ranks of group g / first slot of its block in each region
+    int32_t *dest_pos_gm;           // [Tm, Kd] slot of token t in the region of its i-th destination, group-major order
+    int32_t *row_dest_pos_gm;       // [Kd, Tm] the same per send row, plane layout
+    int32_t *row_dest_flat_gm;      // [Kd, Tm] row of the compact receive area per send row and destination
+    int32_t *gm_tile_sum;           // [max_tiles, R] rows each tile of 256 groups adds to each region
+    int32_t *ex_tile_cnt;           // [max_tiles, E] tokens of each tile that selected each expert (nullptr: too large)
     // scratch
     unsigned long long *slot_key;                  // [HS] open-addressed table keyed by bitmap: (hash tag, first token)
     int32_t *slot_leader, *slot_count;             // [HS] smallest token index / number of tokens with that bitmap
@@ -57,6 +64,7 @@ struct mw_ctx {
     uint32_t gbar_arrivals; // grid-barrier arrivals made by all previous fused plans
     int coop_ok;            // device supports cooperative launch
     int32_t planned_T;      // T of the latest plan, -1 before the first
+    uint32_t gm_epoch;      // epoch of the plan the group-major arrays were made from (0: none)
     int64_t launches;
     // host staging (MW_FLAG_HOST_STAGING)
     int32_t *st_ids, *st_e2r;
@@ -98,6 +106,9 @@ int mw_small_setup(mw_ctx *ctx);
 int mw_small_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x,
                     void *send_buf, int64_t send_capacity_rows, void *recv_base, int64_t recv_stride_bytes,
                     int64_t recv_capacity_rows, cudaStream_t st);
+
+// ---- group-major order and expert index (mw_order.cu) ----
+int mw_order_smem_setup(mw_ctx *ctx);
 
 // ---- row copies (mw_copy.cu) ----
 enum mw_copy_mode {
