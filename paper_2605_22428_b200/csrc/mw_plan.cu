@@ -69,6 +69,19 @@ __device__ __forceinline__ int table_insert(unsigned long long *slot_key, int hs
     return -1;
 }
 
+// One-word bitmaps with fewer than 64 bits set can never equal the all-ones empty marker, so the bitmap itself
+// is the key: no tag, no comparison with another token's bitmap, and nothing that must be visible beforehand.
+__device__ __forceinline__ int table_insert_word(unsigned long long *slot_key, int hs_mask, uint64_t h, unsigned long long word)
+{
+    int slot = (int)(h & (uint64_t)hs_mask);
+    for (int probes = 0; probes <= hs_mask; ++probes) {
+        const unsigned long long cur = atomicCAS(slot_key + slot, kEmptyKey, word);
+        if (cur == kEmptyKey || cur == word) return slot;
+        slot = (slot + 1) & hs_mask;
+    }
+    return -1;
+}
+
 // ------------------------------------------------------------------------------------------
 // Kernel 1: bitmaps (Section 4.1: bit r set <=> rank r is a target) and the bitmap table.
 // ------------------------------------------------------------------------------------------
@@ -412,6 +425,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
 // ------------------------------------------------------------------------------------------
 // Fused plan: the three phases in one cooperative launch.
 // ------------------------------------------------------------------------------------------
+constexpr int kLookBack = 8;                  // predecessors a look-back reads per round trip (16 measured slower: more records not ready yet)
 constexpr int kBarrierSpinLimit = 1 << 21;   // polls of the arrival counter before a block gives up (about a second)
 
 __device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p)
@@ -525,16 +539,20 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                     if ((a.src_rank >> 6) == w) self_only = (m[w] >> (a.src_rank & 63)) & 1;
             }
             if (nd > 0) {
-                __threadfence();                                      // bitmap visible before the slot is claimed
-                const int W = a.W;
-                const uint64_t *masks = a.d.token_mask;
-                slot = table_insert(a.d.slot_key, a.hs_mask, h, t, [&](int other) {
-                    bool same = true;
+                if (WT == 1 && a.Kd < 64) {
+                    slot = table_insert_word(a.d.slot_key, a.hs_mask, h, m[0]);
+                } else {
+                    __threadfence();                                  // bitmap visible before the slot is claimed
+                    const int W = a.W;
+                    const uint64_t *masks = a.d.token_mask;
+                    slot = table_insert(a.d.slot_key, a.hs_mask, h, t, [&](int other) {
+                        bool same = true;
 #pragma unroll
-                    for (int w = 0; w < WT; ++w)
-                        if (w < W) same &= (__ldcg(masks + (int64_t)other * W + w) == m[w]);
-                    return same;
-                });
+                        for (int w = 0; w < WT; ++w)
+                            if (w < W) same &= (__ldcg(masks + (int64_t)other * W + w) == m[w]);
+                        return same;
+                    });
+                }
                 if (slot < 0) { set_status(&acc->status, MW_ERR_CAPACITY); nd = 0; a.d.token_ndest[t] = 0; }
                 else { atomicMin(a.d.slot_leader + slot, t); atomicAdd(a.d.slot_count + slot, 1); }
             }
@@ -548,7 +566,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             if (bad) set_status(&acc->status, MW_ERR_BAD_INDEX);
         }
     }
-    // Decoupled look-back over tiles for counters [c0, c1): one thread per counter, eight predecessors
+    // Decoupled look-back over tiles for counters [c0, c1): one thread per counter, kLookBack predecessors
     // fetched per round trip.  A record is one 64-bit word (epoch, flag, value), so flag and value are
     // always read together; the epoch makes records of earlier plans invisible.
     auto look_back = [&](int c0, int c1) {
@@ -561,13 +579,13 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             } else {
                 *rec = pack_state(a.epoch, kFlagAgg, mine);
                 bool done = false;
-                for (int j = tile - 1; j >= 0 && !done; j -= 8) {
-                    unsigned long long s[8];
+                for (int j = tile - 1; j >= 0 && !done; j -= kLookBack) {
+                    unsigned long long s[kLookBack];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
+                    for (int i = 0; i < kLookBack; ++i)
                         s[i] = (j - i >= 0) ? *(volatile unsigned long long *)(a.d.tile_state + (size_t)(j - i) * a.NC + c) : 0ull;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int i = 0; i < kLookBack; ++i) {
                         if (done || j - i < 0) continue;
                         int spins = 0;
                         while (true) {
@@ -610,19 +628,43 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     look_back(0, a.R);
     __syncthreads();
     if (active) {
-        int i = 0;
         int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
-        if (nd > 0) {
+        if (a.Kd == 8) {
+            // the usual top-8: the token's eight (rank, slot) pairs leave as four 16-byte stores instead of sixteen
+            int rr[8], pp[8];
 #pragma unroll
-            for (int w = 0; w < WT; ++w)
-                for (uint64_t word = m[w]; word; word &= word - 1) {
-                    const int r = w * 64 + __ffsll((long long)word) - 1;
-                    dr[i] = r;
-                    dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
-                    ++i;
-                }
+            for (int i = 0; i < 8; ++i) { rr[i] = -1; pp[i] = -1; }
+            if (nd > 0) {
+                int i = 0;
+#pragma unroll
+                for (int w = 0; w < WT; ++w)
+                    for (uint64_t word = m[w]; word; word &= word - 1) {
+                        const int r = w * 64 + __ffsll((long long)word) - 1;
+                        const int p = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (j == i) { rr[j] = r; pp[j] = p; }
+                        ++i;
+                    }
+            }
+            ((int4 *)dr)[0] = make_int4(rr[0], rr[1], rr[2], rr[3]);
+            ((int4 *)dr)[1] = make_int4(rr[4], rr[5], rr[6], rr[7]);
+            ((int4 *)dp)[0] = make_int4(pp[0], pp[1], pp[2], pp[3]);
+            ((int4 *)dp)[1] = make_int4(pp[4], pp[5], pp[6], pp[7]);
+        } else {
+            int i = 0;
+            if (nd > 0) {
+#pragma unroll
+                for (int w = 0; w < WT; ++w)
+                    for (uint64_t word = m[w]; word; word &= word - 1) {
+                        const int r = w * 64 + __ffsll((long long)word) - 1;
+                        dr[i] = r;
+                        dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
+                        ++i;
+                    }
+            }
+            for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
         }
-        for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
     }
     bool alive = grid_barrier_wait(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
 
@@ -682,6 +724,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     const int Tn = (int)__ldcg(&a.d.totals->T_nonempty), G = (int)__ldcg(&a.d.totals->G);
     const int SD = (int)__ldcg(&a.d.totals->total_dest);
     if (__ldcg(&a.d.totals->status) == MW_ERR_TIMEOUT) return;      // a look-back gave up somewhere: nothing below can be trusted
+    // the region starts, once per block (the tile's own counts in cnt[] are no longer needed); the barrier inside
+    // group_rank_in_tile orders these stores before their use below
+    for (int r = tid; r < a.R; r += MW_TILE) cnt[r] = __ldcg(a.d.rank_offsets + r);
     // tails: every index up to T (inclusive for group_offsets) is covered by some thread of the grid
     for (int u = t; u <= a.T; u += a.ntiles * MW_TILE) {
         if (u > G) a.d.group_offsets[u] = -1;
@@ -717,7 +762,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                 const int p = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
                 a.d.row_dest_rank[(int64_t)i * a.Tm + row] = r;
                 a.d.row_dest_pos[(int64_t)i * a.Tm + row] = p;
-                const int at = __ldcg(a.d.rank_offsets + r) + p;
+                const int at = cnt[r] + p;
                 a.d.row_dest_flat[(int64_t)i * a.Tm + row] = at;
                 a.d.rank_tokens[at] = t;
                 ++i;
