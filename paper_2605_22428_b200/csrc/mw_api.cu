@@ -63,6 +63,7 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.slot_leader = k.take<int32_t>((size_t)c->HS);
     d.slot_count = k.take<int32_t>((size_t)c->HS);
     d.tile_state = k.take<unsigned long long>((size_t)c->max_tiles * (size_t)c->NC);
+    d.tile_agg = k.take<unsigned long long>((size_t)c->max_tiles);
     d.ticket = k.take<unsigned int>(1);
     d.gbar = k.take<unsigned int>(1);
     d.copy_ctr = k.take<unsigned int>(2);

@@ -46,6 +46,7 @@ struct mw_dev {
     unsigned long long *slot_key;                  // [HS] open-addressed table keyed by bitmap: (hash tag, first token)
     int32_t *slot_leader, *slot_count;             // [HS] smallest token index / number of tokens with that bitmap
     unsigned long long *tile_state;                // [max_tiles, NC] look-back records
+    unsigned long long *tile_agg;                  // [max_tiles] (members << 32 | leaders) of each tile, fused plan
     unsigned int *ticket;                          // tile ticket counter
     unsigned int *gbar;                            // arrival counter of the fused plan's grid barriers
     unsigned int *copy_ctr;                        // [2] work-ticket and finished-warp counters of the copy kernels

@@ -668,22 +668,22 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     }
     bool alive = grid_barrier_wait(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
 
-    // ---- phase B2: leaders and group sizes are final; group ids and offsets ----
-    int leader = -1, gcount = 0;
+    // ---- phase B2: leaders and group sizes are final; every tile publishes its two totals ----
+    int leader = -1, gcount = 0, lead_excl = 0, gc_excl = 0;
+    int64_t SD_last = 0, self_copies = 0;          // thread 0 of the last tile
     if (alive) {
         if (nd > 0) { leader = __ldcg(a.d.slot_leader + slot); gcount = __ldcg(a.d.slot_count + slot); }
         const bool is_leader = nd > 0 && leader == t;
         if (active) a.d.token_leader[t] = leader;
         int lead_total, gc_total;
-        const int lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
-        const int gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
-        if (tid == 0) { cnt[a.R] = lead_total; cnt[a.R + 1] = gc_total; }
-        __syncthreads();
-        look_back(a.R, a.R + 2);
-        __syncthreads();
-        if (is_leader) { a.d.gid_at[t] = base[a.R] + lead_excl; a.d.goff_at[t] = base[a.R + 1] + gc_excl; }
+        lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
+        gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
+        // group id and offset relative to the tile, stored at the leader; the sums over earlier tiles are added
+        // by whoever reads them, after the barrier (no second look-back chain)
+        if (is_leader) { a.d.gid_at[t] = lead_excl; a.d.goff_at[t] = gc_excl; }
+        if (tid == 0) a.d.tile_agg[tile] = ((unsigned long long)(uint32_t)gc_total << 32) | (uint32_t)lead_total;
         if (tile == a.ntiles - 1) {
-            // this tile's inclusive prefix is the grand total of every counter
+            // this tile's inclusive prefix is the grand total of every rank counter
             int carry = 0;
             for (int r0 = 0; r0 < a.R; r0 += MW_TILE) {
                 const int r = r0 + tid;
@@ -694,23 +694,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                 carry += total;
             }
             if (tid == 0) {
-                const int64_t G = base[a.R] + cnt[a.R], Tn = base[a.R + 1] + cnt[a.R + 1], SD = carry;
-                const int64_t self_copies = a.src_rank >= 0 ? base[a.src_rank] + cnt[a.src_rank] : 0;
-                const int64_t sent_rows = Tn - (int64_t)acc->self_only;
-                a.d.rank_offsets[a.R] = (int32_t)SD;
-                a.d.group_offsets[G] = (int32_t)Tn;
-                mw_totals tt;
-                tt.T_nonempty = Tn; tt.G = G; tt.total_dest = SD;
-                tt.mw_bytes = sent_rows * a.row_bytes;
-                tt.unicast_bytes = (SD - self_copies) * a.row_bytes;
-                tt.unicast_per_expert_bytes = (int64_t)acc->valid_slots * a.row_bytes;
-                // Section 6.4: beyond 64 ranks the bitmap travels in the payload, once per 4096-byte packet
-                tt.meta_bytes = a.R <= 64 ? 0 : sent_rows * ((a.row_bytes + 4095) / 4096) * (int64_t)(8 * a.W);
-                tt.status = acc->status;
-                tt.reserved = 0;
-                *a.d.totals = tt;
-                mw_acc *next = a.d.acc + ((a.epoch + 1u) & 1u);
-                next->valid_slots = 0; next->self_only = 0; next->status = 0;
+                a.d.rank_offsets[a.R] = carry;
+                SD_last = carry;
+                self_copies = a.src_rank >= 0 ? base[a.src_rank] + cnt[a.src_rank] : 0;
             }
         }
     }
@@ -721,12 +707,36 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     }
 
     // ---- phase C: group ids, send rows, inverse maps, delivery descriptors, table clean-up ----
-    const int Tn = (int)__ldcg(&a.d.totals->T_nonempty), G = (int)__ldcg(&a.d.totals->G);
-    const int SD = (int)__ldcg(&a.d.totals->total_dest);
-    if (__ldcg(&a.d.totals->status) == MW_ERR_TIMEOUT) return;      // a look-back gave up somewhere: nothing below can be trusted
-    // the region starts, once per block (the tile's own counts in cnt[] are no longer needed); the barrier inside
-    // group_rank_in_tile orders these stores before their use below
-    for (int r = tid; r < a.R; r += MW_TILE) cnt[r] = __ldcg(a.d.rank_offsets + r);
+    // Every block reads all tiles' totals (one record each, one round trip) and scans them in shared memory.
+    __shared__ int tile_lead_pre[MW_TILE], tile_gc_pre[MW_TILE];
+    int G, Tn;
+    {
+        const unsigned long long ag = tid < a.ntiles ? __ldcg(a.d.tile_agg + tid) : 0ull;
+        const int plan_status = __ldcg(&acc->status);
+        for (int r = tid; r <= a.R; r += MW_TILE) cnt[r] = __ldcg(a.d.rank_offsets + r);      // see below
+        tile_lead_pre[tid] = block_excl_scan((int)(uint32_t)ag, warp_sums, G);
+        tile_gc_pre[tid] = block_excl_scan((int)(uint32_t)(ag >> 32), warp_sums, Tn);
+        if (tile == a.ntiles - 1 && tid == 0) {
+            const int64_t sent_rows = (int64_t)Tn - (int64_t)acc->self_only;
+            a.d.group_offsets[G] = Tn;
+            mw_totals tt;
+            tt.T_nonempty = Tn; tt.G = G; tt.total_dest = SD_last;
+            tt.mw_bytes = sent_rows * a.row_bytes;
+            tt.unicast_bytes = (SD_last - self_copies) * a.row_bytes;
+            tt.unicast_per_expert_bytes = (int64_t)acc->valid_slots * a.row_bytes;
+            // Section 6.4: beyond 64 ranks the bitmap travels in the payload, once per 4096-byte packet
+            tt.meta_bytes = a.R <= 64 ? 0 : sent_rows * ((a.row_bytes + 4095) / 4096) * (int64_t)(8 * a.W);
+            tt.status = plan_status;
+            tt.reserved = 0;
+            *a.d.totals = tt;
+            mw_acc *next = a.d.acc + ((a.epoch + 1u) & 1u);
+            next->valid_slots = 0; next->self_only = 0; next->status = 0;
+        }
+        if (plan_status == MW_ERR_TIMEOUT) return;      // a look-back gave up somewhere: nothing below can be trusted
+    }
+    // cnt[] now holds the region starts (the tile's own counts are no longer needed); the barriers of the scans
+    // above order those stores before their use below
+    const int SD = cnt[a.R];
     // tails: every index up to T (inclusive for group_offsets) is covered by some thread of the grid
     for (int u = t; u <= a.T; u += a.ntiles * MW_TILE) {
         if (u > G) a.d.group_offsets[u] = -1;
@@ -741,7 +751,10 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     const int within = group_rank_in_tile(&rank_scratch, a.d.token_leader, tile, nd > 0 ? leader : -1, gcount);
     if (!active) return;
     if (nd == 0) { a.d.token_group[t] = -1; a.d.token_mw_row[t] = -1; return; }
-    const int g = __ldcg(a.d.gid_at + leader), goff = __ldcg(a.d.goff_at + leader);
+    // the leader's values are relative to its tile; a leader has its own in registers
+    const int lt = leader / MW_TILE;
+    const int g = tile_lead_pre[lt] + (leader == t ? lead_excl : __ldcg(a.d.gid_at + leader));
+    const int goff = tile_gc_pre[lt] + (leader == t ? gc_excl : __ldcg(a.d.goff_at + leader));
     const int row = goff + within;
     a.d.token_group[t] = g;
     a.d.token_mw_row[t] = row;
@@ -814,7 +827,7 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.bar_base = ctx->gbar_arrivals;
     const int blocks = a.ntiles;
     ctx->planned_T = T;
-    if (blocks <= ctx->sm_count && !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS)) {
+    if (blocks <= ctx->sm_count && blocks <= MW_TILE && !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS)) {
         // One launch, at most one block per SM, phases separated by grid barriers.  The blocks wait for
         // one another, so all of them must become resident: an ordinary launch achieves that as soon
         // as earlier kernels of the stream have drained (the grid never exceeds the SM count and needs
