@@ -82,6 +82,10 @@ def test_rank_word_boundaries(R, E):
     run_order(wl.make_random_dispatch(R, T=700, K=4, E=E, R=R, H=16))
 
 
+def test_more_tokens_than_one_resident_grid_holds():
+    run_order(wl.make_random_dispatch(17, T=40000, K=4, E=64, R=16, H=16, pad_fraction=0.05))
+
+
 def test_few_large_groups_duplicates_invalid_entries_and_source_rank():
     run_order(wl.make_random_dispatch(5, T=3000, K=1, E=12, R=6, H=16))
     run_order(wl.make_random_dispatch(11, T=2000, K=2, E=4, R=4, H=8, contiguous_map=True))

@@ -84,6 +84,14 @@ def test_token_counts_around_tile_edges(T, separate):
     run_dispatch(inp, max_tokens=1100, separate=separate)
 
 
+def test_more_tokens_than_one_resident_grid_holds():
+    # 40000 tokens = 157 tiles, more than the SMs of a B200: the plan takes its three-kernel route by itself
+    inp = wl.make_random_dispatch(17, T=40000, K=4, E=64, R=16, H=16, pad_fraction=0.05)
+    p, tot = run_dispatch(inp)
+    assert tot["T_nonempty"] > 39000 and tot["G"] > 1000
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",), separate=True)
+
+
 def test_top1_and_few_large_groups():
     # every token in a large group: exercises member ranking inside groups across tiles
     inp = wl.make_random_dispatch(5, T=3000, K=1, E=12, R=6, H=16)
