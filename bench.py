@@ -293,7 +293,7 @@ def allgather_sweep(mw, wl, torch) -> list:
                 b.record()
             torch.cuda.synchronize()
             us = statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3
-            moved = 2 * R * S + R * S + window * R * S        # pack read+write, deliver read + window copies
+            moved = R * S + R * S + window * R * S            # one pass: shards read, send buffer + window copies written
             out.append({"shard_bytes": S, "window_ranks": window, "p50_us": round(us, 1),
                         "gbs": round(moved / us / 1e3, 1), "l2_resident": bool(moved < (100 << 20))})
             del shards, send, recv

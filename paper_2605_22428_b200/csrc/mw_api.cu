@@ -349,6 +349,13 @@ int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int 
     a.dst_count = dst_rank_count;
     a.capacity_rows = INT64_MAX;
     int rc;
+    if (!(ctx->cfg.flags & (MW_FLAG_COPY_BULK | MW_FLAG_COPY_REG_STORE | MW_FLAG_COPY_LDST))) {
+        // one pass: every shard is read once and written to its send slot(s) and to its slot in every region of the window
+        a.mode = layout == MW_LAYOUT_MULTIWRITE ? MW_CP_AG_FUSED_MW : MW_CP_AG_FUSED_UC;
+        a.src = (const uint8_t *)shards; a.dst = (uint8_t *)recv_base; a.dst2 = (uint8_t *)send_buf;
+        a.dst_stride = stride; a.host_rows = R;
+        return mw_copy_launch(ctx, a, as_stream(stream));
+    }
     if (layout == MW_LAYOUT_MULTIWRITE) {
         a.mode = MW_CP_AG_PACK_MW;
         a.src = (const uint8_t *)shards; a.dst = (uint8_t *)send_buf; a.host_rows = R;

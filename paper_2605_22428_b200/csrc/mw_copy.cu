@@ -157,6 +157,8 @@ __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row, int mod
     case MW_CP_DISPATCH_UC: return 2 * a.ndst[row];
     case MW_CP_AG_DELIVER_MW:
     case MW_CP_AG_PACK_UC: return a.dst_count;
+    case MW_CP_AG_FUSED_MW: return a.dst_count + 1;
+    case MW_CP_AG_FUSED_UC: return 2 * a.dst_count;
     case MW_CP_PAIR_DIRECT: return a.pair_n;
     case MW_CP_PAIR_SEND: return a.pair_copies + 1;
     default: return 1;
@@ -219,6 +221,13 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
         return a.dst + (int64_t)lo * a.dst_stride + p * a.row_bytes;
     }
     case MW_CP_AG_DELIVER_MW: return a.dst + (int64_t)q * a.dst_stride + row * a.row_bytes;
+    case MW_CP_AG_FUSED_MW:
+        if (q == a.dst_count) return a.dst2 + row * a.row_bytes;
+        return a.dst + (int64_t)q * a.dst_stride + row * a.row_bytes;
+    case MW_CP_AG_FUSED_UC:
+        if (q >= a.dst_count) return a.dst + (int64_t)(q - a.dst_count) * a.dst_stride + row * a.row_bytes;
+        if (a.dst_begin + q == row) return nullptr;                      // the copy to the shard's own rank is never sent
+        return a.dst2 + (row * a.dst_count + q) * a.row_bytes;
     case MW_CP_AG_PACK_UC:
         if (a.dst_begin + q == row) return nullptr;
         return a.dst + (row * a.dst_count + q) * a.row_bytes;
@@ -767,6 +776,8 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_PAIR_FORWARD: err = rows_launch<2, MW_CP_PAIR_FORWARD>(grid, block, st, overlap, a); break;
         case MW_CP_DISPATCH_MW: err = rows_launch<1, MW_CP_DISPATCH_MW>(grid, block, st, overlap, a); break;
         case MW_CP_DISPATCH_UC: err = rows_launch<1, MW_CP_DISPATCH_UC>(grid, block, st, overlap, a); break;
+        case MW_CP_AG_FUSED_MW: err = rows_launch<1, MW_CP_AG_FUSED_MW>(grid, block, st, overlap, a); break;
+        case MW_CP_AG_FUSED_UC: err = rows_launch<1, MW_CP_AG_FUSED_UC>(grid, block, st, overlap, a); break;
         default: return MW_ERR_INVALID_ARG;
         }
     } else if (ctx->cfg.flags & MW_FLAG_COPY_LDST) {

@@ -124,7 +124,9 @@ enum mw_copy_mode {
     MW_CP_PAIR_SEND = 8,    // relayed segment of shard r to its partner's relay area (and to r itself)
     MW_CP_PAIR_FORWARD = 9, // partner forwards the relayed segment to the other members of r's domain
     MW_CP_DISPATCH_MW = 10, // pack and deliver in one pass: x[mw_row_token[j]] -> send[j] and every destination of row j
-    MW_CP_DISPATCH_UC = 11  // x[mw_row_token[j]] -> its unicast send slots and every destination of row j
+    MW_CP_DISPATCH_UC = 11, // x[mw_row_token[j]] -> its unicast send slots and every destination of row j
+    MW_CP_AG_FUSED_MW = 12, // AllGather pack and deliver in one pass: shard i -> send[i] and region(d)[i] for the window
+    MW_CP_AG_FUSED_UC = 13  // shard i -> send[i][d] (d != i) and region(d)[i] for the window
 };
 
 struct mw_copy_args {
