@@ -767,10 +767,6 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_PACK_MW: err = rows_launch<2, MW_CP_PACK_MW>(grid, block, st, overlap, a); break;
         case MW_CP_SCATTER: err = rows_launch<1, MW_CP_SCATTER>(grid, block, st, overlap, a); break;
         case MW_CP_DELIVER_UC: err = rows_launch<2, MW_CP_DELIVER_UC>(grid, block, st, overlap, a); break;
-        case MW_CP_AG_PACK_MW: err = rows_launch<2, MW_CP_AG_PACK_MW>(grid, block, st, overlap, a); break;
-        case MW_CP_AG_DELIVER_MW: err = rows_launch<1, MW_CP_AG_DELIVER_MW>(grid, block, st, overlap, a); break;
-        case MW_CP_AG_PACK_UC: err = rows_launch<1, MW_CP_AG_PACK_UC>(grid, block, st, overlap, a); break;
-        case MW_CP_AG_DELIVER_UC: err = rows_launch<2, MW_CP_AG_DELIVER_UC>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_DIRECT: err = rows_launch<1, MW_CP_PAIR_DIRECT>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_SEND: err = rows_launch<1, MW_CP_PAIR_SEND>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_FORWARD: err = rows_launch<2, MW_CP_PAIR_FORWARD>(grid, block, st, overlap, a); break;
@@ -778,7 +774,7 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_DISPATCH_UC: err = rows_launch<1, MW_CP_DISPATCH_UC>(grid, block, st, overlap, a); break;
         case MW_CP_AG_FUSED_MW: err = rows_launch<1, MW_CP_AG_FUSED_MW>(grid, block, st, overlap, a); break;
         case MW_CP_AG_FUSED_UC: err = rows_launch<1, MW_CP_AG_FUSED_UC>(grid, block, st, overlap, a); break;
-        default: return MW_ERR_INVALID_ARG;
+        default: return MW_ERR_INVALID_ARG;     // the two-launch AllGather modes only run with a MW_FLAG_COPY_* bit
         }
     } else if (ctx->cfg.flags & MW_FLAG_COPY_LDST) {
         const int64_t chunk = choose_chunk(a.row_bytes, est_rows, (int64_t)ctx->sm_count * 2 * (kLdstThreads / 32));
