@@ -333,14 +333,14 @@ def relay_measure(mw, wl, torch) -> dict:
         torch.cuda.synchronize()
         us = a.elapsed_time(b) * 1e3 / n
         assert relay.mw_relay_get_totals()["status"] == 0
-    moved = (2 * rows_send + (rows_send + H) + (H + SD)) * B           # pack, first level, second level
+    moved = ((2 * rows_send + H) + (H + SD)) * B                       # first level in one pass (x read once), second level
     return {"servers": s.R // P, "ranks_per_server": P, "src_rank": src, "hop_rows": H, "delivered_rows": SD,
             "inter_server_unicast_mb": round(tot["inter_unicast_bytes"] / 1e6, 1),
             "inter_server_multiwrite_mb": round(tot["inter_multiwrite_bytes"] / 1e6, 1),
             "inter_server_bytes_saved_pct": round(100 * (1 - tot["inter_multiwrite_bytes"] / tot["inter_unicast_bytes"]), 2),
             "direct_mb": round(tot["direct_bytes"] / 1e6, 1), "relay_forward_mb": round(tot["forward_bytes"] / 1e6, 1),
             "step_us": round(us, 1), "gbs": round(moved / us / 1e3, 1),
-            "note": "step = both plans + descriptors + pack + first-level deliver + second-level expansion"}
+            "note": "step = both plans + descriptors + first level (pack and deliver in one pass) + second-level expansion"}
 
 
 def fused_dispatch_measure(mw, wl, torch) -> dict:

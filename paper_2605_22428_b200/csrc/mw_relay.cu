@@ -41,47 +41,50 @@ __global__ void k_relay_table(const int32_t *e2r, int E, int R, int src, int P, 
 struct DescArgs {
     int T, Kd, R, src, P;
     int64_t rows_max, row_bytes;
-    const int32_t *hop_dest_rank, *hop_dest_pos, *hop_rank_offsets;
+    const int32_t *hop_rank_tokens, *hop_rank_offsets;
     const int32_t *flat_dest_rank, *flat_dest_pos, *flat_rank_offsets;
     const mw_totals *hop_totals, *flat_totals;
     int32_t *s2_ndst, *s2_rank, *s2_pos, *s2_flat;
     mw_relay_totals *totals;
 };
 
-// One thread per token: for each of its next hops, the final destinations behind that hop.
+// One thread per row of the hop area (rows of one hop are consecutive, so the plane stores of a warp are
+// coalesced): the row's token comes from the first-level plan's rank_tokens, its hop from a binary search in the
+// hop offsets, and the final destinations behind that hop from the flat plan's (rank, slot) pairs of the token.
 __global__ void __launch_bounds__(256) k_relay_desc(DescArgs a)
 {
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     long long direct = 0, inter_mw = 0, inter_uc = 0, forward = 0, hop_rows = 0, delivered = 0;
-    if (t < a.T) {
-        const int32_t *hr = a.hop_dest_rank + (int64_t)t * a.Kd, *hp = a.hop_dest_pos + (int64_t)t * a.Kd;
-        const int32_t *fr = a.flat_dest_rank + (int64_t)t * a.Kd, *fp = a.flat_dest_pos + (int64_t)t * a.Kd;
-        for (int j = 0; j < a.Kd; ++j) {
-            const int h = hr[j];
-            if (h < 0) break;
-            const int64_t q = (int64_t)a.hop_rank_offsets[h] + hp[j];          // row of the hop area
-            const bool remote = h / a.P != a.src / a.P;
-            ++hop_rows;
-            inter_mw += remote;
-            int n = 0;
-            for (int i = 0; i < a.Kd; ++i) {
-                const int r = fr[i];
-                if (r < 0) break;
-                if (next_hop(r, a.src, a.P) != h) continue;
-                a.s2_rank[(int64_t)n * a.rows_max + q] = r;
-                a.s2_pos[(int64_t)n * a.rows_max + q] = fp[i];
-                a.s2_flat[(int64_t)n * a.rows_max + q] = a.flat_rank_offsets[r] + fp[i];
-                ++n;
-                ++delivered;
-                if (remote) { ++inter_uc; forward += (r != h); }
-                else direct += (r != a.src);
-            }
-            a.s2_ndst[q] = n;
-            for (int i = n; i < a.Kd; ++i) {
-                a.s2_rank[(int64_t)i * a.rows_max + q] = -1;
-                a.s2_pos[(int64_t)i * a.rows_max + q] = -1;
-                a.s2_flat[(int64_t)i * a.rows_max + q] = -1;
-            }
+    if (q < a.hop_totals->total_dest) {
+        int lo = 0, hi = a.R;                                  // hop h: the last rank with hop_rank_offsets[h] <= q
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (a.hop_rank_offsets[mid] <= q) lo = mid; else hi = mid;
+        }
+        const int h = lo;
+        const int tok = a.hop_rank_tokens[q];
+        const int32_t *fr = a.flat_dest_rank + (int64_t)tok * a.Kd, *fp = a.flat_dest_pos + (int64_t)tok * a.Kd;
+        const bool remote = h / a.P != a.src / a.P;
+        hop_rows = 1;
+        inter_mw = remote;
+        int n = 0;
+        for (int i = 0; i < a.Kd; ++i) {
+            const int r = fr[i];
+            if (r < 0) break;
+            if (next_hop(r, a.src, a.P) != h) continue;
+            a.s2_rank[(int64_t)n * a.rows_max + q] = r;
+            a.s2_pos[(int64_t)n * a.rows_max + q] = fp[i];
+            a.s2_flat[(int64_t)n * a.rows_max + q] = a.flat_rank_offsets[r] + fp[i];
+            ++n;
+            ++delivered;
+            if (remote) { ++inter_uc; forward += (r != h); }
+            else direct += (r != a.src);
+        }
+        a.s2_ndst[q] = n;
+        for (int i = n; i < a.Kd; ++i) {
+            a.s2_rank[(int64_t)i * a.rows_max + q] = -1;
+            a.s2_pos[(int64_t)i * a.rows_max + q] = -1;
+            a.s2_flat[(int64_t)i * a.rows_max + q] = -1;
         }
     }
     // block totals -> device totals (integer sums: independent of the order of the atomics)
@@ -98,7 +101,7 @@ __global__ void __launch_bounds__(256) k_relay_desc(DescArgs a)
         if (v[4]) atomicAdd(out + 4, (unsigned long long)(v[4] * a.row_bytes));
         if (v[5]) atomicAdd(out + 5, (unsigned long long)(v[5] * a.row_bytes));
     }
-    if (t == 0) {
+    if (q == 0) {                                              // thread 0 forwards the plans' status
         const int s = a.flat_totals->status ? a.flat_totals->status : a.hop_totals->status;
         if (s) atomicCAS(&a.totals->status, 0, s);
     }
@@ -180,14 +183,16 @@ int mw_relay_plan(mw_relay *relay, const int32_t *topk_ids, const int32_t *exper
     DescArgs a;
     a.T = T; a.Kd = relay->hop->Kd; a.R = c.R; a.src = c.src_rank; a.P = relay->P;
     a.rows_max = relay->rows_max; a.row_bytes = c.row_bytes;
-    a.hop_dest_rank = relay->hop->d.dest_rank; a.hop_dest_pos = relay->hop->d.dest_pos;
+    a.hop_rank_tokens = relay->hop->d.rank_tokens;
     a.hop_rank_offsets = relay->hop->d.rank_offsets;
     a.flat_dest_rank = relay->flat->d.dest_rank; a.flat_dest_pos = relay->flat->d.dest_pos;
     a.flat_rank_offsets = relay->flat->d.rank_offsets;
     a.hop_totals = relay->hop->d.totals; a.flat_totals = relay->flat->d.totals;
     a.s2_ndst = relay->s2_ndst; a.s2_rank = relay->s2_rank; a.s2_pos = relay->s2_pos; a.s2_flat = relay->s2_flat;
     a.totals = relay->totals;
-    k_relay_desc<<<(T > 0 ? (T + 255) / 256 : 1), 256, 0, st>>>(a);
+    // one thread per possible hop row (T * Kd bounds their number); at least one block forwards the plans' status
+    const int64_t rows_bound = (int64_t)T * a.Kd;
+    k_relay_desc<<<(unsigned)(rows_bound > 0 ? (rows_bound + 255) / 256 : 1), 256, 0, st>>>(a);
     relay->hop->launches += 2;
     relay->planned = 1;
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
@@ -220,8 +225,7 @@ int mw_relay_dispatch(mw_relay *relay, const void *x, void *send_buf, int64_t se
     mw_ctx *hop = relay->hop;
     if (recv_stride_bytes && recv_capacity_rows * hop->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
     // first level: each row once per group of identical next-hop set, one copy per next hop
-    int rc = mw_pack(hop, x, MW_LAYOUT_MULTIWRITE, send_buf, send_capacity_rows, stream);
-    if (rc == MW_OK) rc = mw_deliver(hop, MW_LAYOUT_MULTIWRITE, send_buf, hop_buf, 0, hop_capacity_rows, stream);
+    int rc = mw_dispatch(hop, x, MW_LAYOUT_MULTIWRITE, send_buf, send_capacity_rows, hop_buf, 0, hop_capacity_rows, stream);
     if (rc != MW_OK) return rc;
     // second level: every hop row to the final destinations behind that hop
     mw_copy_args a;
