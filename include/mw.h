@@ -169,8 +169,8 @@ MW_API int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view);
 MW_API int mw_get_totals(mw_ctx *ctx, mw_totals *host_out, void *stream);
 
 /*
- * Pack: fill the send buffer from the hidden rows, using the latest plan (Section 5.2 step 1:
- * "loads its local message data into the pre-allocated send buffer").
+ * Pack: fill the send buffer from the hidden rows, using the latest plan (Section 5.2 step 1: every rank first
+ * copies its own data into a send buffer allocated beforehand).
  *   MW_LAYOUT_MULTIWRITE  send_buf[j] = x[mw_row_token[j]],            j < T'
  *   MW_LAYOUT_UNICAST     send_buf[rank_offsets[r] + i] = x[rank_tokens[rank_offsets[r] + i]]
  *   x         device, [T, row_bytes], 16-byte aligned
@@ -296,7 +296,7 @@ MW_API int mw_expert_index(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *
                     int32_t *expert_token, int32_t *expert_slot, void *stream);
 
 /*
- * Paired-relay AllGather with segment split (Section 3.1 "paired relaying", Section 5.2): cfg.R = 2n
+ * Paired-relay AllGather with segment split (the paired relaying of Section 3.1; Section 5.2): cfg.R = 2n
  * ranks on a full mesh form two domains, [0, n) and [n, 2n); rank r is paired with (r + n) mod 2n.
  * Each domain gathers its own n shards: afterwards the receive region of every rank holds the shards
  * of its domain in rank order.  Bytes [0, direct_bytes) of a shard go on the direct links to the other
@@ -345,8 +345,8 @@ MW_API int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int
  *
  * The R ranks form servers of ranks_per_server consecutive ranks; the source is rank cfg.src_rank
  * (it must be a member of the domain).  A destination in the source's own server is its own next
- * hop; every other server's next hop is the rank with the source's index inside that server (the
- * "same-index NPU"), which forwards the row to the destinations inside its server.  First level:
+ * hop; every other server's next hop is the rank with the source's index inside that server (Section 3.2),
+ * which forwards the row to the destinations inside its server.  First level:
  * an ordinary MultiWrite plan / pack / deliver over next-hop sets into a hop area (one region per
  * next hop).  Second level: every row of the hop area is written to the final destinations whose
  * next hop it is, at the slots of the flat plan, so the final receive regions are byte-identical
