@@ -332,7 +332,7 @@ int mwo_allgather(const uint8_t *shards, int32_t R, int64_t shard_bytes, int lay
  * Ranks are grouped into servers of ranks_per_server consecutive ranks.  The source (src_rank, a
  * member of the domain) writes directly to destinations inside its own server; for every other
  * server that holds at least one destination of a token it sends ONE copy to the rank with its own
- * index inside that server (the "same-index NPU"), which then replicates the row to the destinations
+ * index inside that server (Section 3.2), which then replicates the row to the destinations
  * inside its server (Section 3.2; Section 4.1 "Local forwarding table": one copy per distinct next hop;
  * Section 4.3.3: M is partitioned by next hop).
  */
