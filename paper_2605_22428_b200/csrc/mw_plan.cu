@@ -472,12 +472,6 @@ __device__ bool grid_barrier_wait(unsigned int *counter, unsigned int target, bo
     return s_alive != 0;
 }
 
-__device__ __forceinline__ bool grid_barrier(unsigned int *counter, unsigned int target, bool alive, int *status)
-{
-    grid_barrier_arrive(counter);
-    return grid_barrier_wait(counter, target, alive, status);
-}
-
 template <int WT>
 __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
 {
@@ -627,7 +621,44 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     __syncthreads();
     look_back(0, a.R);
     __syncthreads();
-    if (active) {
+    bool alive = grid_barrier_wait(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
+
+    // ---- phase B2: leaders and group sizes are final; every tile publishes its two totals ----
+    int leader = -1, gcount = 0, lead_excl = 0, gc_excl = 0;
+    int64_t SD_last = 0, self_copies = 0;          // thread 0 of the last tile
+    if (alive) {
+        if (nd > 0) { leader = __ldcg(a.d.slot_leader + slot); gcount = __ldcg(a.d.slot_count + slot); }
+        const bool is_leader = nd > 0 && leader == t;
+        if (active) a.d.token_leader[t] = leader;
+        int lead_total, gc_total;
+        lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
+        gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
+        // group id and offset relative to the tile, stored at the leader; the sums over earlier tiles are added
+        // by whoever reads them, after the barrier (no second look-back chain)
+        if (is_leader) { a.d.gid_at[t] = lead_excl; a.d.goff_at[t] = gc_excl; }
+        if (tid == 0) a.d.tile_agg[tile] = ((unsigned long long)(uint32_t)gc_total << 32) | (uint32_t)lead_total;
+        if (tile == a.ntiles - 1) {
+            // this tile's inclusive prefix is the grand total of every rank counter
+            int carry = 0;
+            for (int r0 = 0; r0 < a.R; r0 += MW_TILE) {
+                const int r = r0 + tid;
+                const int v = r < a.R ? base[r] + cnt[r] : 0;
+                int total;
+                const int excl = block_excl_scan(v, warp_sums, total);
+                if (r < a.R) a.d.rank_offsets[r] = carry + excl;
+                carry += total;
+            }
+            if (tid == 0) {
+                a.d.rank_offsets[a.R] = carry;
+                SD_last = carry;
+                self_copies = a.src_rank >= 0 ? base[a.src_rank] + cnt[a.src_rank] : 0;
+            }
+        }
+    }
+    // The (rank, slot) pairs of every token are only read by later kernels: they are stored while the second
+    // barrier is in flight (arrive, store, wait), off the critical path.
+    grid_barrier_arrive(a.d.gbar);
+    if (alive && active) {
         int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
         if (a.Kd == 8) {
             // the usual top-8: the token's eight (rank, slot) pairs leave as four 16-byte stores instead of sixteen
@@ -666,41 +697,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
         }
     }
-    bool alive = grid_barrier_wait(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
-
-    // ---- phase B2: leaders and group sizes are final; every tile publishes its two totals ----
-    int leader = -1, gcount = 0, lead_excl = 0, gc_excl = 0;
-    int64_t SD_last = 0, self_copies = 0;          // thread 0 of the last tile
-    if (alive) {
-        if (nd > 0) { leader = __ldcg(a.d.slot_leader + slot); gcount = __ldcg(a.d.slot_count + slot); }
-        const bool is_leader = nd > 0 && leader == t;
-        if (active) a.d.token_leader[t] = leader;
-        int lead_total, gc_total;
-        lead_excl = block_excl_scan(is_leader ? 1 : 0, warp_sums, lead_total);
-        gc_excl = block_excl_scan(is_leader ? gcount : 0, warp_sums, gc_total);
-        // group id and offset relative to the tile, stored at the leader; the sums over earlier tiles are added
-        // by whoever reads them, after the barrier (no second look-back chain)
-        if (is_leader) { a.d.gid_at[t] = lead_excl; a.d.goff_at[t] = gc_excl; }
-        if (tid == 0) a.d.tile_agg[tile] = ((unsigned long long)(uint32_t)gc_total << 32) | (uint32_t)lead_total;
-        if (tile == a.ntiles - 1) {
-            // this tile's inclusive prefix is the grand total of every rank counter
-            int carry = 0;
-            for (int r0 = 0; r0 < a.R; r0 += MW_TILE) {
-                const int r = r0 + tid;
-                const int v = r < a.R ? base[r] + cnt[r] : 0;
-                int total;
-                const int excl = block_excl_scan(v, warp_sums, total);
-                if (r < a.R) a.d.rank_offsets[r] = carry + excl;
-                carry += total;
-            }
-            if (tid == 0) {
-                a.d.rank_offsets[a.R] = carry;
-                SD_last = carry;
-                self_copies = a.src_rank >= 0 ? base[a.src_rank] + cnt[a.src_rank] : 0;
-            }
-        }
-    }
-    alive = grid_barrier(a.d.gbar, a.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
+    alive = grid_barrier_wait(a.d.gbar, a.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
     if (!alive) {
         if (tid == 0) set_status(&a.d.totals->status, MW_ERR_TIMEOUT);
         return;
