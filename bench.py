@@ -387,6 +387,53 @@ def fused_dispatch_measure(mw, wl, torch) -> dict:
     return out
 
 
+def large_ep_measure(mw, wl, torch) -> dict:
+    """The other large-batch shape (R = 128, T = 8192, Zipf-skewed experts): the same three calls as the headline step."""
+    inp = wl.make_dispatch("large_ep")
+    s = inp.shape
+    B, T = s.row_bytes, s.T
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    xh = torch.from_numpy(inp.x.view(np.int16))
+    with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+        ctx.mw_plan(ids, e2r, T)
+        tot = ctx.mw_get_totals()
+        Tn, SD = tot["T_nonempty"], tot["total_dest"]
+        sets = [(xh.cuda(), torch.empty(Tn * B, dtype=torch.uint8, device="cuda"),
+                 torch.empty(SD * B, dtype=torch.uint8, device="cuda")) for _ in range(2)]      # 2 x 1.17 GB > L2
+
+        def step(i):
+            x, send, recv = sets[i % 2]
+            ctx.mw_plan(ids, e2r, T)
+            ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+            ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
+
+        def copies(i):
+            x, send, recv = sets[i % 2]
+            ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+            ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
+
+        out = {}
+        for name, fn, n in (("step_us", step, 200), ("pack_plus_deliver_us", copies, 200)):
+            for i in range(6):
+                fn(i)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(n):
+                fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            out[name] = round(a.elapsed_time(b) * 1e3 / n, 1)
+        assert ctx.mw_get_totals()["status"] == 0
+    nbytes = (3 * Tn + SD) * B
+    out.update({"rows_packed": Tn, "rows_delivered": SD, "groups": tot["G"], "algorithmic_bytes_per_step": nbytes,
+                "step_gbs": round(nbytes / out["step_us"] / 1e3, 1),
+                "pack_plus_deliver_gbs": round(nbytes / out["pack_plus_deliver_us"] / 1e3, 1),
+                "pack_plus_deliver_fraction_of_nominal_8TBs": round(nbytes / out["pack_plus_deliver_us"] / 1e3 / 8000.0, 4),
+                "tokens_per_s": round(T / out["step_us"] * 1e6, 1)})
+    return out
+
+
 def order_measure(mw, wl, torch) -> dict:
     """Group-major receive order (Sections 4.3.1, 4.3.2) and expert index (Section 2.3.2) on the headline workload."""
     inp = wl.make_dispatch(WORKLOAD, payload=False)
@@ -671,6 +718,7 @@ def run_cuda(args):
             line["combine_dsv3_prefill"] = combine_measure(mw, wl, torch)
             line["dispatch_fused"] = fused_dispatch_measure(mw, wl, torch)
             line["receiver_order"] = order_measure(mw, wl, torch)
+            line["large_ep"] = large_ep_measure(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:
