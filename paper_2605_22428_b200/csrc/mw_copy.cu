@@ -642,8 +642,16 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
     grid_launch_dependents();
     grid_dependency_wait();
     const int tid = threadIdx.x;
+    // Deliver walks the send rows from the last to the first and writes with streaming (evict-first) stores.
+    // The rows come out of the pack launch in ascending order, so the most recently packed ones are still in
+    // L2; taking them first, with stores that do not displace them, turns most send-row reads into L2 hits and
+    // leaves DRAM an almost pure write stream.  Measured on B200, deliver right after pack: 4096 rows of
+    // 14336 bytes (59 MB of send rows) 85 -> 74 us; 8192 rows (117 MB, about the size of L2) 164 -> 154 us.
+    // With send rows that are not in L2 the streaming stores cost 3 to 4 % instead.
+    constexpr bool kAfterPack = MODE == MW_CP_SCATTER;
+    const unsigned blk = kAfterPack ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
     // 32-bit on purpose: the division is on the way to the first load
-    const int row = blockIdx.x / a.chunks_per_row, piece = blockIdx.x % a.chunks_per_row;
+    const int row = blk / a.chunks_per_row, piece = blk % a.chunks_per_row;
     // what decides whether the block has work is loaded together and looked at afterwards: one round trip
     // (all of it lies inside the plan's arrays for any row below the launch bound)
     const int status = (a.totals && a.rows_from != 0) ? a.totals->status : MW_OK;
@@ -675,7 +683,10 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
                 if (!d) continue;
 #pragma unroll
                 for (int k = 0; k < V; ++k)
-                    if (off + k * step < a.row_bytes) *(uint4 *)(d + off + k * step) = v[k];
+                    if (off + k * step < a.row_bytes) {
+                        if constexpr (kAfterPack) __stcs((uint4 *)(d + off + k * step), v[k]);
+                        else *(uint4 *)(d + off + k * step) = v[k];
+                    }
             }
         }
     }
