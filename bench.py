@@ -246,7 +246,7 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
             ctx.mw_plan_dispatch(ids, e2r, s.T, x, mw.MW_LAYOUT_MULTIWRITE, send, Tn, recv, 0, SD)
 
         for name, fn in (("plan", plan), ("pack_deliver", dispatch), ("chain", chain), ("one_call", one_call)):
-            for _ in range(50):
+            for _ in range(min(50, launches)):
                 fn()
             evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
             torch.cuda.synchronize()
@@ -257,10 +257,39 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
             torch.cuda.synchronize()
             us = [a.elapsed_time(b) * 1e3 for a, b in evs]
             out[name] = {"p50_us": round(percentile(us, 0.5), 2), "p99_us": round(percentile(us, 0.99), 2)}
+        # the single-launch call keeps no host-side state, so it can be replayed from a CUDA graph: no host launch cost
+        torch.cuda.synchronize()
+        graph, chained, n_chain = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph(), 20
+        with torch.cuda.graph(graph):
+            one_call()
+        with torch.cuda.graph(chained):
+            for _ in range(n_chain):
+                one_call()
+        for _ in range(20):
+            graph.replay()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+        torch.cuda.synchronize()
+        for a, b in evs:
+            a.record()
+            graph.replay()
+            b.record()
+        torch.cuda.synchronize()
+        us = [a.elapsed_time(b) * 1e3 for a, b in evs]
+        out["one_call_graph"] = {"p50_us": round(percentile(us, 0.5), 2), "p99_us": round(percentile(us, 0.99), 2)}
+        evs = evs[:min(50, launches)]
+        for a, b in evs:
+            a.record()
+            chained.replay()
+            b.record()
+        torch.cuda.synchronize()
+        us = [a.elapsed_time(b) * 1e3 / n_chain for a, b in evs]
+        out["one_call_graph_chained"] = {"p50_us": round(percentile(us, 0.5), 2), "calls_per_graph": n_chain}
+        assert ctx.mw_get_totals()["status"] == 0
     out["launches"] = launches
     out["note"] = ("L2-resident working set (0.9 MB in, 7.3 MB out): judged on latency, not on HBM fraction; chain = "
                    "mw_plan + mw_dispatch (2 launches: mw_dispatch packs and delivers in one pass), one_call = mw_plan_dispatch (1 launch); each figure includes "
-                   "the host's launch cost through the Python binding")
+                   "the host's launch cost through the Python binding, except one_call_graph (the same call replayed from a "
+                   "CUDA graph, one call per graph) and one_call_graph_chained (20 calls per graph, time per call)")
     return out
 
 
@@ -738,7 +767,16 @@ def main():
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="MW_FLAG_* bits for the timed context")
     ap.add_argument("--kernels-only", action="store_true",
                     help="only the device-timed steps (for profiler runs): no end-to-end leg, extras or CPU baseline")
+    ap.add_argument("--decode-only", type=int, default=0, metavar="LAUNCHES",
+                    help="only the decode-shape latency measurement with this many launches per figure (for profiler runs)")
     args = ap.parse_args()
+    if args.decode_only > 0 and args.impl == "cuda":
+        import torch
+        from paper_2605_22428_b200 import binding as mw
+        from paper_2605_22428_b200 import workloads as wl
+        torch.cuda.set_device(0)
+        print(json.dumps({"decode_only": True, "decode": decode_latency(mw, wl, torch, args.decode_only)}))
+        return 0
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")
     return run_reference(args) if args.impl == "reference" else run_cuda(args)

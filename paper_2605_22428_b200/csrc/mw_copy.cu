@@ -635,7 +635,7 @@ __host__ __device__ constexpr bool mode_is_one_to_one(int mode)
            mode == MW_CP_PAIR_FORWARD;
 }
 
-template <int V, int MODE>
+template <int V, int MODE, bool kAfterPack = false>
 __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constant__ mw_copy_args a)
 {
     __shared__ uint8_t *dst_s[kRowsDstBatch];
@@ -647,8 +647,8 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
     // L2; taking them first, with stores that do not displace them, turns most send-row reads into L2 hits and
     // leaves DRAM an almost pure write stream.  Measured on B200, deliver right after pack: 4096 rows of
     // 14336 bytes (59 MB of send rows) 85 -> 74 us; 8192 rows (117 MB, about the size of L2) 164 -> 154 us.
-    // With send rows that are not in L2 the streaming stores cost 3 to 4 % instead.
-    constexpr bool kAfterPack = MODE == MW_CP_SCATTER;
+    // With send rows that are not in L2 the streaming stores cost 3 to 4 % instead, so only the deliver from a
+    // MultiWrite send buffer is launched with kAfterPack (the unicast pack scatters rows of x, which come from DRAM).
     const unsigned blk = kAfterPack ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
     // 32-bit on purpose: the division is on the way to the first load
     const int row = blk / a.chunks_per_row, piece = blk % a.chunks_per_row;
@@ -693,10 +693,10 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
 }
 
 // One instantiation per mode, so that the mode switches of the work list fold away.
-template <int V, int MODE>
+template <int V, int MODE, bool AFTER_PACK = false>
 cudaError_t rows_launch(dim3 grid, dim3 block, cudaStream_t st, bool overlap, const mw_copy_args &a)
 {
-    return mw_launch(k_copy_rows<V, MODE>, grid, block, 0, st, overlap, a);
+    return mw_launch(k_copy_rows<V, MODE, AFTER_PACK>, grid, block, 0, st, overlap, a);
 }
 
 struct CopyShape { int warps; int stages; int64_t chunk; int batch; };
@@ -776,7 +776,11 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         const dim3 block(threads);
         switch (a.mode) {
         case MW_CP_PACK_MW: err = rows_launch<2, MW_CP_PACK_MW>(grid, block, st, overlap, a); break;
-        case MW_CP_SCATTER: err = rows_launch<1, MW_CP_SCATTER>(grid, block, st, overlap, a); break;
+        case MW_CP_SCATTER:
+            // no source index: the rows are a send buffer, packed just before
+            err = a.src_index ? rows_launch<1, MW_CP_SCATTER>(grid, block, st, overlap, a)
+                              : rows_launch<1, MW_CP_SCATTER, true>(grid, block, st, overlap, a);
+            break;
         case MW_CP_DELIVER_UC: err = rows_launch<2, MW_CP_DELIVER_UC>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_DIRECT: err = rows_launch<1, MW_CP_PAIR_DIRECT>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_SEND: err = rows_launch<1, MW_CP_PAIR_SEND>(grid, block, st, overlap, a); break;

@@ -231,6 +231,42 @@ def test_one_call_groups_padding_invalid_ids_and_source_rank():
     run_dispatch(big_k, one_call=True)
 
 
+def test_one_call_replays_from_a_cuda_graph():
+    """The single-launch path keeps no host-side state, so a captured call can be replayed: the same graph is run
+    on two different batches written into the same device buffers and checked against the oracle both times."""
+    torch = torch_mod()
+    a, b = wl.make_dispatch("decode"), wl.make_dispatch("decode", 100)
+    s = a.shape
+    T, B = a.T, s.row_bytes
+    ids_d = torch.from_numpy(a.topk_ids).cuda()
+    e2r_d = torch.from_numpy(a.expert_to_rank).cuda()
+    x_d = torch.from_numpy(a.x.view(np.int16)).cuda()
+    plans = [mwo.plan(i.topk_ids, i.expert_to_rank, s.R, B) for i in (a, b)]
+    Tn = max(p.totals["T_nonempty"] for p in plans)
+    SD = max(p.totals["total_dest"] for p in plans)
+    send, recv = Guarded(Tn * B), Guarded(SD * B)
+    with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+        ctx.mw_plan_dispatch(ids_d, e2r_d, T, x_d.data_ptr(), mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn, recv.ptr(), 0, SD)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            ctx.mw_plan_dispatch(ids_d, e2r_d, T, x_d.data_ptr(), mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn, recv.ptr(), 0, SD)
+        for inp, p in ((a, plans[0]), (b, plans[1]), (a, plans[0])):
+            ids_d.copy_(torch.from_numpy(inp.topk_ids))
+            x_d.copy_(torch.from_numpy(inp.x.view(np.int16)))
+            send.body.fill_(SENTINEL)
+            recv.body.fill_(SENTINEL)
+            graph.replay()
+            torch.cuda.synchronize()
+            assert_plan_equal(ctx.plan_arrays(T), p, ctx.mw_get_totals())
+            want_send = mwo.pack_mw(p, inp.x)
+            n_send, n_recv = p.totals["T_nonempty"] * B, p.totals["total_dest"] * B
+            assert np.array_equal(send.host()[:n_send].reshape(-1, B), want_send)
+            assert np.array_equal(recv.host()[:n_recv], mwo.deliver_mw(p, want_send, 0, SENTINEL))
+            assert (send.host()[n_send:] == SENTINEL).all() and (recv.host()[n_recv:] == SENTINEL).all()
+            assert send.guards_intact() and recv.guards_intact()
+
+
 def test_one_call_capacity_overflow_is_reported_and_contained():
     torch = torch_mod()
     inp = wl.make_random_dispatch(21, T=200, K=3, E=32, R=8, H=16, contiguous_map=True)
