@@ -514,11 +514,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                     const bool ok = r[j] >= 0 && r[j] < a.R;
                     bad |= (id[j] >= 0 && id[j] < a.E && !ok);
                     valid += ok;
-                    if (ok) {
+                    const uint64_t rank_bit = ok ? 1ull << (r[j] & 63) : 0ull;
 #pragma unroll
-                        for (int w = 0; w < WT; ++w)
-                            if ((r[j] >> 6) == w) m[w] |= 1ull << (r[j] & 63);              // OR = per-rank dedup
-                    }
+                    for (int w = 0; w < WT; ++w) m[w] |= rank_bit & equal_mask64(r[j] >> 6, w);   // OR = per-rank dedup
                 }
             }
             uint64_t h = 0x2545f4914f6cdd1dull;
@@ -530,7 +528,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             if (a.src_rank >= 0 && nd == 1) {
 #pragma unroll
                 for (int w = 0; w < WT; ++w)
-                    if ((a.src_rank >> 6) == w) self_only = (m[w] >> (a.src_rank & 63)) & 1;
+                    self_only |= (int)((m[w] & equal_mask64(a.src_rank >> 6, w)) >> (a.src_rank & 63)) & 1;
             }
             if (nd > 0) {
                 if (WT == 1 && a.Kd < 64) {
@@ -606,9 +604,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     const uint32_t bit = 1u << (tid & 31);
     grid_barrier_arrive(a.d.gbar);  // this tile's bitmaps are in the table (also orders the clearing of the bit matrix)
     if (nd > 0) {
-#pragma unroll
-        for (int w = 0; w < WT; ++w)
-            for (uint64_t word = m[w]; word; word &= word - 1)
+#pragma unroll 1
+        for (int w = 0; w < a.W; ++w)
+            for (uint64_t word = bitmap_word(m, w); word; word &= word - 1)
                 atomicOr(bits + (size_t)(w * 64 + __ffsll((long long)word) - 1) * 8 + wi, bit);
     }
     __syncthreads();
@@ -667,9 +665,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             for (int i = 0; i < 8; ++i) { rr[i] = -1; pp[i] = -1; }
             if (nd > 0) {
                 int i = 0;
-#pragma unroll
-                for (int w = 0; w < WT; ++w)
-                    for (uint64_t word = m[w]; word; word &= word - 1) {
+#pragma unroll 1
+                for (int w = 0; w < a.W; ++w)
+                    for (uint64_t word = bitmap_word(m, w); word; word &= word - 1) {
                         const int r = w * 64 + __ffsll((long long)word) - 1;
                         const int p = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
 #pragma unroll
@@ -685,9 +683,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
         } else {
             int i = 0;
             if (nd > 0) {
-#pragma unroll
-                for (int w = 0; w < WT; ++w)
-                    for (uint64_t word = m[w]; word; word &= word - 1) {
+#pragma unroll 1
+                for (int w = 0; w < a.W; ++w)
+                    for (uint64_t word = bitmap_word(m, w); word; word &= word - 1) {
                         const int r = w * 64 + __ffsll((long long)word) - 1;
                         dr[i] = r;
                         dp[i] = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
@@ -765,9 +763,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     }
     {
         int i = 0;
-#pragma unroll
-        for (int w = 0; w < WT; ++w)
-            for (uint64_t word = m[w]; word; word &= word - 1) {
+#pragma unroll 1
+        for (int w = 0; w < a.W; ++w)
+            for (uint64_t word = bitmap_word(m, w); word; word &= word - 1) {
                 const int r = w * 64 + __ffsll((long long)word) - 1;
                 const int p = base[r] + (int)pre[r * 8 + wi] + __popc(bits[r * 8 + wi] & (bit - 1));
                 a.d.row_dest_rank[(int64_t)i * a.Tm + row] = r;

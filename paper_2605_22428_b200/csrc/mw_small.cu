@@ -2,12 +2,19 @@
 //
 // With a few dozen tokens the three-launch chain (plan, pack, deliver) is dominated by launch gaps and
 // by the plan's chain of global-memory round trips, the cost the paper reports for its small batches
-// (Section 6.3: replication overhead outweighs the savings at batch 64).  Here every block of a
-// persistent grid recomputes the whole plan in its own shared memory (the inputs are 2 KB) -- same
-// rules, same results as the plan kernels, no grid-wide synchronisation -- and then moves its share of
-// the rows: each row chunk is read once from x into registers and written to its slot of the MultiWrite
-// send buffer and to every destination region.  Block 0 also writes the plan metadata, so the context
-// is left exactly as after mw_plan + mw_dispatch.
+// (Section 6.3: replication overhead outweighs the savings at batch 64).  Here every block of the grid
+// recomputes the whole plan in its own shared memory (the inputs are 2 KB) -- same rules, same results
+// as the plan kernels, no grid-wide synchronisation -- and then moves its share of the rows: each row
+// chunk is read once from x into registers and written to its slot of the MultiWrite send buffer and to
+// every destination region.  A few blocks move no rows and write the plan metadata instead, so the
+// context is left exactly as after mw_plan + mw_dispatch.
+//
+// The kernel is latency-bound (a batch of 64 tokens occupies two warps), so the work of every phase is
+// spread over all threads of the block: whatever exists once per (token, expert slot) -- rank lookup,
+// bitmap bit, slot inside the destination region, descriptors -- is done by one thread per pair, and
+// only the group table and the per-token scalars are done by one thread per token.  Two expert slots of
+// a token that name the same rank compute and store identical values; nothing below counts them twice.
+// The kernel keeps no state on the host or in global scratch, so a captured launch can be replayed.
 #include "mw_internal.cuh"
 
 namespace {
@@ -15,8 +22,10 @@ namespace {
 constexpr int kSmallThreads = 256;     // = largest T
 constexpr int kSmallSlots = 512;       // bitmap table in shared memory (load <= 1/2)
 constexpr int kSmallMaxKd = 16;
-constexpr int kSmallMaxW = 4;
+constexpr int kSmallMaxW = 4;          // R <= 256: the three prefix sums fit one packed block scan
 constexpr int kSmallChunk = 2048;      // bytes of a row moved by one warp at a time (4 x 16 bytes per lane)
+constexpr int kSmallWriters = 4;       // blocks that write plan metadata instead of moving rows
+constexpr int kSmallMinGrid = 16;      // smaller grids: block 0 writes everything and also moves rows
 
 struct SmallArgs {
     const int32_t *ids, *e2r;
@@ -24,7 +33,11 @@ struct SmallArgs {
     uint8_t *send, *recv;
     int T, K, E, R, W, Kd, src_rank, Tm;
     int64_t row_bytes, send_capacity_rows, recv_stride, recv_capacity_rows;
-    mw_dev d;
+    // plan arrays the metadata blocks fill
+    uint64_t *token_mask, *group_mask;
+    int32_t *token_ndest, *token_group, *token_mw_row, *mw_row_token, *group_offsets, *rank_offsets, *rank_tokens;
+    int32_t *dest_rank, *dest_pos, *token_leader, *row_ndest, *row_dest_rank, *row_dest_pos, *row_dest_flat;
+    mw_totals *totals;
 };
 
 __device__ __forceinline__ uint64_t mix64s(uint64_t h, uint64_t v)
@@ -35,18 +48,17 @@ __device__ __forceinline__ uint64_t mix64s(uint64_t h, uint64_t v)
 }
 
 // Exclusive prefix sum over the 256 threads of the block; `total` is returned to every thread.
-__device__ __forceinline__ int scan256(int v, int *warp_sums, int &total)
+__device__ __forceinline__ uint32_t scan256(uint32_t v, uint32_t *warp_sums, uint32_t &total)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int incl = v;
+    uint32_t incl = v;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { int n = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += n; }
-    __syncthreads();
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += n; }
     if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
-    int before = 0, sum = 0;
+    uint32_t before = 0, sum = 0;
 #pragma unroll
-    for (int w = 0; w < kSmallThreads / 32; ++w) { const int s = warp_sums[w]; if (w < warp) before += s; sum += s; }
+    for (int w = 0; w < kSmallThreads / 32; ++w) { const uint32_t s = warp_sums[w]; if (w < warp) before += s; sum += s; }
     total = sum;
     return before + incl - v;
 }
@@ -57,186 +69,196 @@ __device__ __forceinline__ uint4 ld16(const uint8_t *p)
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-__device__ __forceinline__ void st16(uint8_t *p, const uint4 &v)
+
+// Rank named by expert slot p = t * K + k, or -1 (padding or invalid).  ids and the table are inputs of the
+// launch and never written by it, so the second look at them (descriptor phase) is served by L1.
+__device__ __forceinline__ int slot_rank(const SmallArgs &a, int p, int &id_out)
 {
-    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+    const int id = __ldg(a.ids + p);
+    id_out = id;
+    if (id < 0 || id >= a.E) return -1;
+    const int r = __ldg(a.e2r + id);
+    return (r >= 0 && r < a.R) ? r : -1;
 }
 
-template <int WT>
 __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_constant__ SmallArgs a)
 {
     extern __shared__ __align__(16) uint8_t ssm[];
     // shared-memory layout (sizes depend on R, W, Kd)
-    uint64_t *masks_s = (uint64_t *)ssm;                                   // [256, W]
-    unsigned long long *hkey = (unsigned long long *)(masks_s + kSmallThreads * a.W);   // [512]
-    int *hlead = (int *)(hkey + kSmallSlots);                              // [512]
-    int *hcnt = hlead + kSmallSlots;                                       // [512]
-    uint32_t *bits = (uint32_t *)(hcnt + kSmallSlots);                     // [R, 9] (padded rows)
-    int *pre = (int *)(bits + a.R * 9);                                    // [R, 9]
-    int *cnt = pre + a.R * 9;                                              // [R]
-    int *ro = cnt + a.R;                                                   // [R + 1]
-    int *leader_s = ro + a.R + 1;                                          // [256]
-    int *gid_s = leader_s + kSmallThreads;                                 // [256] group id, at the leader's index
+    uint64_t *mask64 = (uint64_t *)ssm;                                    // [256, W] bitmap of token t
+    uint32_t *mask32 = (uint32_t *)ssm;                                    //          the same words as 32-bit halves
+    unsigned long long *hkey = (unsigned long long *)(mask64 + kSmallThreads * a.W);   // [512] (hash tag, first claimant)
+    int *hlead = (int *)(hkey + kSmallSlots);                              // [512] smallest token with that bitmap
+    int *hcnt = hlead + kSmallSlots;                                       // [512] tokens with that bitmap
+    int *hrun = hcnt + kSmallSlots;                                        // [512] members counted so far (rank inside a group)
+    uint32_t *bits = (uint32_t *)(hrun + kSmallSlots);                     // [R, 9] bit t of row r: token t targets rank r (padded rows)
+    int *pre = (int *)(bits + a.R * 9);                                    // [R, 9] tokens before each 32-token word that target r
+    int *ro = pre + a.R * 9;                                               // [R + 1] region starts
+    int *nd_s = ro + a.R + 1;                                              // [256] destinations of token t
+    int *gid_s = nd_s + kSmallThreads;                                     // [256] group id, at the leader's index
     int *goff_s = gid_s + kSmallThreads;                                   // [256] group offset, at the leader's index
-    int *row_token_s = goff_s + kSmallThreads;                             // [256] token of send row j
+    int *tok_row_s = goff_s + kSmallThreads;                               // [256] send row of token t, -1 if none
+    int *row_token_s = tok_row_s + kSmallThreads;                          // [256] token of send row j
     int *row_nd_s = row_token_s + kSmallThreads;                           // [256] destinations of send row j
-    int *row_flat_s = row_nd_s + kSmallThreads;                            // [256, Kd] destination rows (or rank<<16|slot when strided)
-    __shared__ int warp_sums[kSmallThreads / 32];
+    int *row_flat_s = row_nd_s + kSmallThreads;                            // [256, Kd] destination rows (rank<<16|slot when strided)
+    __shared__ uint32_t warp_sums[kSmallThreads / 32];
     __shared__ int s_acc[3];
 
-    const int tid = threadIdx.x, t = tid;
+    const int tid = threadIdx.x, t = tid, lane = tid & 31, warp = tid >> 5;
     const bool active = t < a.T;
-    grid_launch_dependents();
-    grid_dependency_wait();        // the previous dispatch may still read the plan arrays block 0 rewrites
+    const int pairs = a.T * a.K;
+    // which part of the metadata this block writes (-1: none), and its place among the blocks that move rows
+    const int writers = (int)gridDim.x >= kSmallMinGrid ? kSmallWriters : 1;
+    const int my_part = (int)blockIdx.x < writers ? (int)blockIdx.x : -1;
+    auto writes = [&](int part) { return my_part >= 0 && part % writers == my_part; };
+    const int movers = writers == 1 ? (int)gridDim.x : (int)gridDim.x - writers;
+    const int mover = writers == 1 ? (int)blockIdx.x : (int)blockIdx.x - writers;
 
-    // ---- bitmaps ----
-    uint64_t m[WT];
-#pragma unroll
-    for (int w = 0; w < WT; ++w) m[w] = 0;
-    int nd = 0, valid = 0, bad = 0, self_only = 0;
-    uint64_t h = 0x2545f4914f6cdd1dull;
-    if (active) {
-        const int32_t *my = a.ids + (int64_t)t * a.K;
-        for (int k0 = 0; k0 < a.K; k0 += 8) {
-            int id[8], r[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) id[j] = (k0 + j < a.K) ? my[k0 + j] : -1;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const bool ok = id[j] >= 0 && id[j] < a.E;
-                bad |= (id[j] != -1 && !ok);
-                r[j] = ok ? a.e2r[id[j]] : -1;
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const bool ok = r[j] >= 0 && r[j] < a.R;
-                bad |= (id[j] >= 0 && id[j] < a.E && !ok);
-                valid += ok;
-                if (ok) {
-#pragma unroll
-                    for (int w = 0; w < WT; ++w)
-                        if ((r[j] >> 6) == w) m[w] |= 1ull << (r[j] & 63);          // OR = per-rank dedup
-                }
-            }
-        }
-#pragma unroll
-        for (int w = 0; w < WT; ++w)
-            if (w < a.W) { masks_s[tid * a.W + w] = m[w]; nd += __popcll(m[w]); h = mix64s(h, m[w]); }
-        if (a.src_rank >= 0 && nd == 1) {
-#pragma unroll
-            for (int w = 0; w < WT; ++w)
-                if ((a.src_rank >> 6) == w) self_only = (m[w] >> (a.src_rank & 63)) & 1;
-        }
-    }
-    for (int i = tid; i < kSmallSlots; i += kSmallThreads) { hkey[i] = ~0ull; hlead[i] = 0x7fffffff; hcnt[i] = 0; }
+    // ---- clear the tables (no global memory involved: overlaps the tail of the previous kernel) ----
+    grid_launch_dependents();
+    for (int i = tid; i < kSmallThreads * a.W; i += kSmallThreads) mask64[i] = 0;
+    for (int i = tid; i < kSmallSlots; i += kSmallThreads) { hkey[i] = ~0ull; hlead[i] = 0x7fffffff; hcnt[i] = 0; hrun[i] = 0; }
     for (int i = tid; i < a.R * 9; i += kSmallThreads) bits[i] = 0;
     if (tid < 3) s_acc[tid] = 0;
+    grid_dependency_wait();        // the previous dispatch may still read the plan arrays this launch rewrites
     __syncthreads();
-    valid = __reduce_add_sync(0xffffffffu, valid);
-    self_only = __reduce_add_sync(0xffffffffu, self_only);
-    bad = __reduce_or_sync(0xffffffffu, (unsigned)bad);
-    if ((tid & 31) == 0) {
-        if (valid) atomicAdd(s_acc + 0, valid);
-        if (self_only) atomicAdd(s_acc + 1, self_only);
-        if (bad) s_acc[2] = 1;
-    }
 
-    // ---- groups: table keyed by bitmap, leader = smallest token index ----
-    int slot = -1;
-    const int wi = tid >> 5;
-    const uint32_t bit = 1u << (tid & 31);
-    if (nd > 0) {
-        const uint32_t tag = (uint32_t)(h >> 32);
-        const unsigned long long mine = ((unsigned long long)tag << 32) | (uint32_t)t;
-        slot = (int)(h & (kSmallSlots - 1));
-        for (int probes = 0; probes < kSmallSlots; ++probes) {
-            const unsigned long long cur = atomicCAS(hkey + slot, ~0ull, mine);
-            if (cur == ~0ull) break;
-            if ((uint32_t)(cur >> 32) == tag) {
-                const uint64_t *om = masks_s + (size_t)(uint32_t)cur * a.W;
-                bool same = true;
-#pragma unroll
-                for (int w = 0; w < WT; ++w)
-                    if (w < a.W) same &= (om[w] == m[w]);
-                if (same) break;
-            }
-            slot = (slot + 1) & (kSmallSlots - 1);
+    // ---- one thread per expert slot: rank lookup, bitmap bit (Section 4.1: bit r set <=> rank r is a target;
+    //      OR = several experts on one rank count once), token bit in the rank's row ----
+    {
+        int valid = 0, bad = 0;
+        for (int p = tid; p < pairs; p += kSmallThreads) {
+            int id;
+            const int r = slot_rank(a, p, id);
+            bad |= (id != -1 && r < 0);
+            if (r < 0) continue;
+            ++valid;
+            const int tk = p / a.K;
+            atomicOr(mask32 + tk * 2 * a.W + (r >> 5), 1u << (r & 31));
+            atomicOr(bits + r * 9 + (tk >> 5), 1u << (tk & 31));
         }
-        atomicMin(hlead + slot, t);
-        atomicAdd(hcnt + slot, 1);
-#pragma unroll
-        for (int w = 0; w < WT; ++w)
-            for (uint64_t word = m[w]; word; word &= word - 1)
-                atomicOr(bits + (size_t)(w * 64 + __ffsll((long long)word) - 1) * 9 + wi, bit);
+        valid = __reduce_add_sync(0xffffffffu, valid);
+        bad = __reduce_or_sync(0xffffffffu, (unsigned)bad);
+        if (lane == 0) {
+            if (valid) atomicAdd(s_acc + 0, valid);
+            if (bad) s_acc[2] = 1;
+        }
     }
     __syncthreads();
+
+    // ---- one thread per token: groups (table keyed by bitmap, leader = smallest token index);
+    //      one thread per rank: tokens of each 32-token word that target it ----
+    int nd = 0, slot = -1;
+    if (active) {
+        uint64_t h = 0x2545f4914f6cdd1dull;
+        for (int w = 0; w < a.W; ++w) { const uint64_t m = mask64[t * a.W + w]; nd += __popcll(m); h = mix64s(h, m); }
+        if (a.src_rank >= 0 && nd == 1 && ((mask64[t * a.W + (a.src_rank >> 6)] >> (a.src_rank & 63)) & 1)) atomicAdd(s_acc + 1, 1);
+        if (nd > 0) {
+            const uint32_t tag = (uint32_t)(h >> 32);
+            const unsigned long long mine = ((unsigned long long)tag << 32) | (uint32_t)t;
+            slot = (int)(h & (kSmallSlots - 1));
+            for (int probes = 0; probes < kSmallSlots; ++probes) {
+                const unsigned long long cur = atomicCAS(hkey + slot, ~0ull, mine);
+                if (cur == ~0ull) break;
+                if ((uint32_t)(cur >> 32) == tag) {
+                    const uint64_t *om = mask64 + (size_t)(uint32_t)cur * a.W;
+                    bool same = true;
+                    for (int w = 0; w < a.W; ++w) same &= (om[w] == mask64[t * a.W + w]);
+                    if (same) break;
+                }
+                slot = (slot + 1) & (kSmallSlots - 1);
+            }
+            atomicMin(hlead + slot, t);
+            atomicAdd(hcnt + slot, 1);
+        }
+    }
+    nd_s[tid] = nd;
+    int my_cnt = 0;                // tokens that target rank `tid`
+    if (tid < a.R) {
+#pragma unroll
+        for (int w8 = 0; w8 < 8; ++w8) { pre[tid * 9 + w8] = my_cnt; my_cnt += __popc(bits[tid * 9 + w8]); }
+    }
+    __syncthreads();
+
+    // ---- group ids, group offsets and region starts: three exclusive prefix sums in one packed scan
+    //      (leaders <= 256: 9 bits, members <= 256: 9 bits, destinations <= 256 * 16: 13 bits) ----
     const int leader = nd > 0 ? hlead[slot] : -1;
     const int gcount = nd > 0 ? hcnt[slot] : 0;
-    leader_s[tid] = leader;
     const bool is_leader = nd > 0 && leader == t;
-    for (int r = tid; r < a.R; r += kSmallThreads) {
-        int run = 0;
-#pragma unroll
-        for (int w8 = 0; w8 < 8; ++w8) { pre[r * 9 + w8] = run; run += __popc(bits[r * 9 + w8]); }
-        cnt[r] = run;
-    }
-    int G, Tn, SD;
-    const int gid = scan256(is_leader ? 1 : 0, warp_sums, G);
-    const int goff_mine = scan256(is_leader ? gcount : 0, warp_sums, Tn);
-    if (is_leader) { gid_s[tid] = gid; goff_s[tid] = goff_mine; }
-    {
-        int carry = 0;
-        for (int r0 = 0; r0 < a.R; r0 += kSmallThreads) {
-            const int r = r0 + tid;
-            int total;
-            const int excl = scan256(r < a.R ? cnt[r] : 0, warp_sums, total);
-            if (r < a.R) ro[r] = carry + excl;
-            carry += total;
-        }
-        SD = carry;
-        if (tid == 0) ro[a.R] = carry;
-    }
-    __syncthreads();
+    uint32_t total;
+    const uint32_t excl = scan256((is_leader ? 1u | ((uint32_t)gcount << 9) : 0u) | ((uint32_t)my_cnt << 18), warp_sums, total);
+    const int G = (int)(total & 511u), Tn = (int)((total >> 9) & 511u), SD = (int)(total >> 18);
+    const int goff_mine = (int)((excl >> 9) & 511u);
+    if (is_leader) { gid_s[tid] = (int)(excl & 511u); goff_s[tid] = goff_mine; }
+    if (tid < a.R) ro[tid] = (int)(excl >> 18);
+    if (tid == 0) ro[a.R] = SD;
 
-    // ---- send rows and destination slots ----
-    int row = -1, g = -1;
+    // ---- rank inside the group, in token order.  Only when some group has more than one member: the warps
+    //      take turns, and in each the first member of a group claims places for all its members of that warp ----
+    int within = 0;
+    if (G != Tn) {
+        const int key = (nd > 0 && gcount > 1) ? slot : -1 - lane;       // negative keys are unique: groups of one
+        const unsigned same = __match_any_sync(0xffffffffu, key);
+        const int first = __ffs(same) - 1;
+        for (int turn = 0; turn < kSmallThreads / 32; ++turn) {
+            if (warp == turn) {
+                int base = 0;
+                if (key >= 0 && lane == first) base = atomicAdd(hrun + slot, __popc(same));
+                within = __shfl_sync(0xffffffffu, base, first) + __popc(same & ((1u << lane) - 1u));
+            }
+            __syncthreads();
+        }
+    } else {
+        __syncthreads();
+    }
+
+    // ---- one thread per token: send row ----
+    int g = -1, row = -1, overflow = 0;
     if (nd > 0) {
-        int within = 0;
-        if (gcount > 1)
-            for (int u = leader; u < t; ++u) within += (leader_s[u] == leader);
         g = gid_s[leader];
         row = goff_s[leader] + within;
         row_token_s[row] = t;
         row_nd_s[row] = nd;
-        int i = 0;
-#pragma unroll
-        for (int w = 0; w < WT; ++w)
-            for (uint64_t word = m[w]; word; word &= word - 1) {
-                const int r = w * 64 + __ffsll((long long)word) - 1;
-                const int pos = pre[r * 9 + wi] + __popc(bits[r * 9 + wi] & (bit - 1));
-                row_flat_s[row * a.Kd + i] = a.recv_stride ? ((r << 16) | pos) : ro[r] + pos;
-                ++i;
-            }
+        overflow = row >= a.send_capacity_rows;
+    }
+    tok_row_s[tid] = row;
+    __syncthreads();
+
+    // ---- one thread per expert slot: place among the token's destinations (= set bits below r), slot inside
+    //      the region (= earlier tokens that target r), descriptors ----
+    for (int p = tid; p < pairs; p += kSmallThreads) {
+        int id;
+        const int r = slot_rank(a, p, id);
+        if (r < 0) continue;
+        const int tk = p / a.K, wi = tk >> 5;
+        const uint64_t *m = mask64 + tk * a.W;
+        int i = __popcll(m[r >> 6] & ((1ull << (r & 63)) - 1ull));
+        for (int w = 0; w < (r >> 6); ++w) i += __popcll(m[w]);
+        const int pos = pre[r * 9 + wi] + __popc(bits[r * 9 + wi] & ((1u << (tk & 31)) - 1u));
+        const int flat = ro[r] + pos, rowk = tok_row_s[tk];
+        row_flat_s[rowk * a.Kd + i] = a.recv_stride ? ((r << 16) | pos) : flat;
+        overflow |= (a.recv_stride ? pos : flat) >= a.recv_capacity_rows;
+        if (writes(2)) {
+            a.dest_rank[tk * a.Kd + i] = r;
+            a.dest_pos[tk * a.Kd + i] = pos;
+            a.rank_tokens[flat] = tk;
+        }
+        if (writes(3)) {
+            a.row_dest_rank[(int64_t)i * a.Tm + rowk] = r;
+            a.row_dest_pos[(int64_t)i * a.Tm + rowk] = pos;
+            a.row_dest_flat[(int64_t)i * a.Tm + rowk] = flat;
+        }
     }
     __syncthreads();
 
-    // ---- block 0 leaves the plan metadata exactly as the plan kernels would ----
-    if (blockIdx.x == 0) {
-        // rows that do not fit their buffer are skipped by whichever block meets them; the status is block 0's to write
-        int overflow = 0;
-        if (nd > 0) {
-            overflow |= row >= a.send_capacity_rows;
-            for (int i = 0; i < nd; ++i) {
-                const int f = row_flat_s[row * a.Kd + i];
-                overflow |= (a.recv_stride ? (f & 0xffff) : f) >= a.recv_capacity_rows;
-            }
-        }
+    // ---- the metadata blocks leave the plan arrays exactly as the plan kernels would ----
+    if (writes(0)) {
+        // rows that do not fit their buffer are skipped by whichever block meets them; the status is written here
         overflow = __syncthreads_or(overflow);
-        for (int r = tid; r <= a.R; r += kSmallThreads) a.d.rank_offsets[r] = ro[r];
+        for (int r = tid; r <= a.R; r += kSmallThreads) a.rank_offsets[r] = ro[r];
         if (tid == 0) {
-            const int64_t self_copies = a.src_rank >= 0 ? cnt[a.src_rank] : 0;
+            const int64_t self_copies = a.src_rank >= 0 ? ro[a.src_rank + 1] - ro[a.src_rank] : 0;
             const int64_t sent_rows = (int64_t)Tn - s_acc[1];
-            a.d.group_offsets[G] = Tn;
             mw_totals tt;
             tt.T_nonempty = Tn; tt.G = G; tt.total_dest = SD;
             tt.mw_bytes = sent_rows * a.row_bytes;
@@ -246,64 +268,55 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
             tt.meta_bytes = a.R <= 64 ? 0 : sent_rows * ((a.row_bytes + 4095) / 4096) * (int64_t)(8 * a.W);
             tt.status = s_acc[2] ? MW_ERR_BAD_INDEX : overflow ? MW_ERR_CAPACITY : MW_OK;
             tt.reserved = 0;
-            *a.d.totals = tt;
+            *a.totals = tt;
         }
+        // tails
         for (int u = tid; u <= a.T; u += kSmallThreads) {
-            if (u > G) a.d.group_offsets[u] = -1;
+            if (u > G) a.group_offsets[u] = -1;
+            if (u == G) a.group_offsets[u] = Tn;
             if (u < a.T) {
-                if (u >= Tn) a.d.mw_row_token[u] = -1;
-                for (int i = 0; i < a.Kd; ++i)
-                    if (u * a.Kd + i >= SD) a.d.rank_tokens[u * a.Kd + i] = -1;
+                if (u >= Tn) a.mw_row_token[u] = -1;
                 if (u >= G)
-                    for (int w = 0; w < a.W; ++w) a.d.group_mask[(int64_t)u * a.W + w] = 0;
+                    for (int w = 0; w < a.W; ++w) a.group_mask[(int64_t)u * a.W + w] = 0;
             }
         }
-        if (active) {
-            for (int w = 0; w < a.W; ++w) a.d.token_mask[(int64_t)t * a.W + w] = masks_s[tid * a.W + w];
-            a.d.token_ndest[t] = nd;
-            a.d.token_group[t] = g;
-            a.d.token_mw_row[t] = row;
-            int32_t *dr = a.d.dest_rank + (int64_t)t * a.Kd, *dp = a.d.dest_pos + (int64_t)t * a.Kd;
-            int i = 0;
-            if (nd > 0) {
-                a.d.mw_row_token[row] = t;
-                a.d.row_ndest[row] = nd;
-                a.d.token_leader[t] = leader;
-                if (is_leader) {
-                    a.d.group_offsets[g] = goff_s[tid];
-                    for (int w = 0; w < a.W; ++w) a.d.group_mask[(int64_t)g * a.W + w] = masks_s[tid * a.W + w];
-                }
-#pragma unroll
-                for (int w = 0; w < WT; ++w)
-                    for (uint64_t word = m[w]; word; word &= word - 1) {
-                        const int r = w * 64 + __ffsll((long long)word) - 1;
-                        const int pos = pre[r * 9 + wi] + __popc(bits[r * 9 + wi] & (bit - 1));
-                        dr[i] = r;
-                        dp[i] = pos;
-                        a.d.rank_tokens[ro[r] + pos] = t;
-                        a.d.row_dest_rank[(int64_t)i * a.Tm + row] = r;
-                        a.d.row_dest_pos[(int64_t)i * a.Tm + row] = pos;
-                        a.d.row_dest_flat[(int64_t)i * a.Tm + row] = ro[r] + pos;
-                        ++i;
-                    }
-                for (int q = i; q < a.Kd; ++q) {
-                    a.d.row_dest_rank[(int64_t)q * a.Tm + row] = -1;
-                    a.d.row_dest_pos[(int64_t)q * a.Tm + row] = -1;
-                    a.d.row_dest_flat[(int64_t)q * a.Tm + row] = -1;
-                }
-            } else {
-                a.d.token_leader[t] = -1;
+        for (int q = SD + tid; q < a.T * a.Kd; q += kSmallThreads) a.rank_tokens[q] = -1;
+    }
+    if (writes(1) && active) {
+        for (int w = 0; w < a.W; ++w) a.token_mask[(int64_t)t * a.W + w] = mask64[t * a.W + w];
+        a.token_ndest[t] = nd;
+        a.token_group[t] = g;
+        a.token_mw_row[t] = row;
+        a.token_leader[t] = leader;
+        if (nd > 0) {
+            a.mw_row_token[row] = t;
+            a.row_ndest[row] = nd;
+            if (is_leader) {
+                a.group_offsets[g] = goff_mine;
+                for (int w = 0; w < a.W; ++w) a.group_mask[(int64_t)g * a.W + w] = mask64[t * a.W + w];
             }
-            for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
         }
     }
+    if (writes(2) || writes(3)) {
+        // unused entries: -1
+        const bool lists = writes(2), planes = writes(3);
+        for (int q = tid; q < a.T * a.Kd; q += kSmallThreads) {
+            const int tk = q / a.Kd, i = q % a.Kd, n = nd_s[tk];
+            if (i < n) continue;
+            if (lists) { a.dest_rank[q] = -1; a.dest_pos[q] = -1; }
+            if (planes && n > 0) {
+                const int64_t at = (int64_t)i * a.Tm + tok_row_s[tk];
+                a.row_dest_rank[at] = -1; a.row_dest_pos[at] = -1; a.row_dest_flat[at] = -1;
+            }
+        }
+    }
+    if (mover < 0) return;
 
-    // ---- rows: every warp of the grid takes (send row, chunk) items round robin ----
-    const int lane = tid & 31;
+    // ---- rows: every warp of the moving blocks takes (send row, chunk) items round robin ----
     const int chunks = (int)((a.row_bytes + kSmallChunk - 1) / kSmallChunk);
     const int items = Tn * chunks;
-    const int warps = gridDim.x * (kSmallThreads / 32);
-    for (int item = (tid >> 5) * gridDim.x + blockIdx.x; item < items; item += warps) {
+    const int warps = movers * (kSmallThreads / 32);
+    for (int item = warp * movers + mover; item < items; item += warps) {
         const int j = item / chunks;
         const int64_t off = (int64_t)(item % chunks) * kSmallChunk;
         const int nvec = (int)(min((int64_t)kSmallChunk, a.row_bytes - off) >> 4);
@@ -332,7 +345,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
             d += off + lane * 16;
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (u * 32 + lane < nvec) st16(d + u * 512, v[u]);
+                if (u * 32 + lane < nvec) *(uint4 *)(d + u * 512) = v[u];
         }
     }
 }
@@ -340,7 +353,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
 size_t small_smem_bytes(const mw_ctx *ctx)
 {
     const size_t R = (size_t)ctx->cfg.R, W = (size_t)ctx->W, Kd = (size_t)ctx->Kd;
-    return kSmallThreads * W * 8 + kSmallSlots * 16 + R * 9 * 8 + (2 * R + 1) * 4 + 5 * kSmallThreads * 4 + kSmallThreads * Kd * 4 + 64;
+    return kSmallThreads * W * 8 + kSmallSlots * 20 + R * 9 * 8 + (R + 1) * 4 + 6 * kSmallThreads * 4 + kSmallThreads * Kd * 4 + 64;
 }
 
 }  // namespace
@@ -357,8 +370,8 @@ int mw_small_setup(mw_ctx *ctx)
 {
     const size_t need = small_smem_bytes(ctx);
     if (ctx->W > kSmallMaxW || ctx->Kd > kSmallMaxKd || need + 1024 > (size_t)ctx->max_smem_optin) return MW_OK;   // path not available
-    void (*fn)(SmallArgs) = ctx->W <= 1 ? k_dispatch_small<1> : ctx->W <= 2 ? k_dispatch_small<2> : k_dispatch_small<4>;
-    if (need > 48 * 1024 && cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)
+    if (need > 48 * 1024 &&
+        cudaFuncSetAttribute(k_dispatch_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)
         return MW_ERR_CUDA;
     return MW_OK;
 }
@@ -376,9 +389,14 @@ int mw_small_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_
     a.send_capacity_rows = send_capacity_rows;
     a.recv_stride = recv_stride_bytes;
     a.recv_capacity_rows = recv_capacity_rows;
-    a.d = ctx->d;
-    void (*fn)(SmallArgs) = ctx->W <= 1 ? k_dispatch_small<1> : ctx->W <= 2 ? k_dispatch_small<2> : k_dispatch_small<4>;
-    const cudaError_t e = mw_launch(fn, dim3(ctx->sm_count), dim3(kSmallThreads), small_smem_bytes(ctx), st,
+    const mw_dev &d = ctx->d;
+    a.token_mask = d.token_mask; a.group_mask = d.group_mask;
+    a.token_ndest = d.token_ndest; a.token_group = d.token_group; a.token_mw_row = d.token_mw_row;
+    a.mw_row_token = d.mw_row_token; a.group_offsets = d.group_offsets; a.rank_offsets = d.rank_offsets;
+    a.rank_tokens = d.rank_tokens; a.dest_rank = d.dest_rank; a.dest_pos = d.dest_pos; a.token_leader = d.token_leader;
+    a.row_ndest = d.row_ndest; a.row_dest_rank = d.row_dest_rank; a.row_dest_pos = d.row_dest_pos;
+    a.row_dest_flat = d.row_dest_flat; a.totals = d.totals;
+    const cudaError_t e = mw_launch(k_dispatch_small, dim3(ctx->sm_count), dim3(kSmallThreads), small_smem_bytes(ctx), st,
                                     !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP), a);
     ctx->launches += 1;
     ctx->planned_T = T;
