@@ -432,6 +432,12 @@ def large_ep_measure(mw, wl, torch) -> dict:
 
         def step(i):
             x, send, recv = sets[i % 2]
+            ctx.mw_plan_prefetch(ids, e2r, T, x)
+            ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+            ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
+
+        def step_plain(i):
+            x, send, recv = sets[i % 2]
             ctx.mw_plan(ids, e2r, T)
             ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
             ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
@@ -442,7 +448,7 @@ def large_ep_measure(mw, wl, torch) -> dict:
             ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
 
         out = {}
-        for name, fn, n in (("step_us", step, 200), ("pack_plus_deliver_us", copies, 200)):
+        for name, fn, n in (("step_us", step, 200), ("step_without_prefetch_us", step_plain, 200), ("pack_plus_deliver_us", copies, 200)):
             for i in range(6):
                 fn(i)
             torch.cuda.synchronize()
@@ -628,7 +634,10 @@ def run_cuda(args):
         x, send, recv = sets[i % nsets]
         if evs:
             evs[0].record()
-        ctx.mw_plan(ids, e2r, T)
+        if args.no_prefetch:
+            ctx.mw_plan(ids, e2r, T)
+        else:
+            ctx.mw_plan_prefetch(ids, e2r, T, x)      # the same plan; idle SMs bring x into L2 meanwhile
         if evs:
             evs[1].record()
         ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
@@ -767,6 +776,8 @@ def main():
     ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="MW_FLAG_* bits for the timed context")
     ap.add_argument("--kernels-only", action="store_true",
                     help="only the device-timed steps (for profiler runs): no end-to-end leg, extras or CPU baseline")
+    ap.add_argument("--no-prefetch", action="store_true",
+                    help="plan with mw_plan instead of mw_plan_prefetch (hidden rows not brought into L2 while planning)")
     ap.add_argument("--decode-only", type=int, default=0, metavar="LAUNCHES",
                     help="only the decode-shape latency measurement with this many launches per figure (for profiler runs)")
     args = ap.parse_args()

@@ -162,6 +162,16 @@ MW_API int mw_destroy(mw_ctx *ctx);
 MW_API int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
             mw_plan_view *view, void *stream);
 
+/*
+ * mw_plan with one more argument: the hidden rows x (device, [T, row_bytes], 16-byte aligned; may be NULL when T is 0) that the pack step
+ * will load into the send buffer next (Section 5.2 step 1).  Same plan, same results.  Planning is a chain of
+ * dependent steps on a few SMs and leaves the memory system idle, so the launch carries extra blocks that ask
+ * the L2 cache for the first rows of x (up to half the cache) meanwhile; mw_pack / mw_dispatch then find them
+ * there.  x is only read.  It must not be written by work that runs concurrently with the plan.
+ */
+MW_API int mw_plan_prefetch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
+                     const void *x, mw_plan_view *view, void *stream);
+
 /* Fills `view` with the workspace pointers of the context and the T of its latest plan (no device work). */
 MW_API int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view);
 

@@ -33,7 +33,7 @@ MW_FLAG_COPY_BULK = 0x40
 
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
-EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
+EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_plan_prefetch", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
            "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_group_major", "mw_deliver_group_major", "mw_expert_index",
            "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
            "mw_strerror", "mw_pair_balanced_direct_bytes") + RELAY_EXPORTS
@@ -111,6 +111,7 @@ def lib():
         L.mw_create.argtypes = [C.POINTER(vp), C.POINTER(mw_config)]
         L.mw_destroy.argtypes = [vp]
         L.mw_plan.argtypes = [vp, vp, vp, i32, C.POINTER(mw_plan_view), vp]
+        L.mw_plan_prefetch.argtypes = [vp, vp, vp, i32, vp, C.POINTER(mw_plan_view), vp]
         L.mw_get_plan_view.argtypes = [vp, C.POINTER(mw_plan_view)]
         L.mw_get_totals.argtypes = [vp, C.POINTER(mw_totals), vp]
         L.mw_pack.argtypes = [vp, vp, C.c_int, vp, i64, vp]
@@ -140,7 +141,7 @@ def lib():
             getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:18]:
+        for name in EXPORTS[:19]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -242,6 +243,15 @@ class Context:
         rc = lib().mw_plan(self._h, _ptr(topk_ids), _ptr(expert_to_rank), T, C.byref(view), _stream(stream))
         if check and rc != MW_OK:
             raise MwError(rc, "mw_plan")
+        self.view = view
+        return rc
+
+    def mw_plan_prefetch(self, topk_ids, expert_to_rank, T: int | None, x, stream=None, check: bool = True) -> int:
+        T = int(topk_ids.shape[0]) if T is None else T
+        view = mw_plan_view()
+        rc = lib().mw_plan_prefetch(self._h, _ptr(topk_ids), _ptr(expert_to_rank), T, _ptr(x), C.byref(view), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_plan_prefetch")
         self.view = view
         return rc
 

@@ -135,6 +135,7 @@ int mw_create(mw_ctx **out, const mw_config *cfg)
     c->planned_T = -1;
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
+    cudaDeviceGetAttribute(&c->l2_bytes, cudaDevAttrL2CacheSize, cfg->device);
     cudaDeviceGetAttribute(&c->coop_ok, cudaDevAttrCooperativeLaunch, cfg->device);
 
     const size_t bytes = carve(c, nullptr);
@@ -167,9 +168,12 @@ int mw_destroy(mw_ctx *ctx)
     return e == cudaSuccess ? MW_OK : MW_ERR_CUDA;
 }
 
-int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, mw_plan_view *view, void *stream)
+namespace {
+int plan_with_rows(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *rows,
+                   mw_plan_view *view, void *stream)
 {
     if (!ctx || !expert_to_rank || T < 0 || T > ctx->cfg.max_tokens || (T > 0 && !topk_ids)) return MW_ERR_INVALID_ARG;
+    if (rows && !aligned16(rows)) return MW_ERR_ALIGNMENT;
     if (view) {
         const mw_dev &d = ctx->d;
         view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
@@ -178,7 +182,20 @@ int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank,
         view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
         view->T = T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
     }
-    return mw_plan_launch(ctx, topk_ids, expert_to_rank, T, as_stream(stream));
+    return mw_plan_launch(ctx, topk_ids, expert_to_rank, T, rows, as_stream(stream));
+}
+}  // namespace
+
+int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, mw_plan_view *view, void *stream)
+{
+    return plan_with_rows(ctx, topk_ids, expert_to_rank, T, nullptr, view, stream);
+}
+
+int mw_plan_prefetch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x,
+                     mw_plan_view *view, void *stream)
+{
+    if (!x && T > 0) return MW_ERR_INVALID_ARG;
+    return plan_with_rows(ctx, topk_ids, expert_to_rank, T, x, view, stream);
 }
 
 int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view)
@@ -303,7 +320,7 @@ int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert
     if (!aligned16(x) || !aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
     if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
     if (!mw_small_applies(ctx, T, layout)) {
-        const int rc = mw_plan(ctx, topk_ids, expert_to_rank, T, view, stream);
+        const int rc = mw_plan_prefetch(ctx, topk_ids, expert_to_rank, T, x, view, stream);
         if (rc != MW_OK) return rc;
         return mw_dispatch(ctx, x, layout, send_buf, send_capacity_rows, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
     }

@@ -58,6 +58,7 @@ struct mw_ctx {
     int W, Kd, HS, NC, max_tiles;
     int sm_count;
     int max_smem_optin;
+    int l2_bytes;
     mw_dev d;
     void *slab;
     uint32_t epoch;         // plans issued so far (tile records carry it, so they need no clearing)
@@ -119,7 +120,8 @@ __device__ __forceinline__ uint64_t bitmap_word(const uint64_t (&m)[WT], int w)
 #endif
 
 // ---- plan (mw_plan.cu) ----
-int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t st);
+// `rows` (may be null): the hidden rows [T, row_bytes] the pack step will read; they are brought into L2 while the plan runs
+int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *rows, cudaStream_t st);
 int mw_plan_smem_setup(mw_ctx *ctx);
 
 // ---- single-launch small-batch path (mw_small.cu) ----

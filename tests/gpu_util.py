@@ -57,7 +57,7 @@ def assert_plan_equal(got: dict, p: mwo.Plan, totals: dict):
 
 def run_dispatch(inp, *, layouts=(mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST), strides=("compact", "strided"),
                  flags: int = 0, src_rank: int = -1, max_tokens: int | None = None, check_payload: bool = True,
-                 repeats: int = 1, one_call: bool = False, separate: bool = False):
+                 repeats: int = 1, one_call: bool = False, separate: bool = False, prefetch: bool = False):
     """Plans and dispatches `inp` on the GPU, checks everything against the oracle, returns (plan, totals)."""
     torch = torch_mod()
     s = inp.shape
@@ -66,9 +66,14 @@ def run_dispatch(inp, *, layouts=(mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST)
     e2r_d = torch.from_numpy(inp.expert_to_rank).cuda()
     p = mwo.plan(inp.topk_ids, inp.expert_to_rank, s.R, B, src_rank)
     assert p.ret == 0
+    x_early = torch.from_numpy(inp.x.view(np.int16)).cuda() if prefetch else None
     with mw.Context(s.R, s.E, s.K, max_tokens or max(T, 1), B, src_rank=src_rank, flags=flags) as ctx:
         for _ in range(repeats):
-            ctx.mw_plan(ids_d, e2r_d, T)
+            if prefetch:
+                # the same plan; the launch also asks L2 for the hidden rows
+                ctx.mw_plan_prefetch(ids_d, e2r_d, T, x_early)
+            else:
+                ctx.mw_plan(ids_d, e2r_d, T)
             totals = ctx.mw_get_totals()
             got = ctx.plan_arrays(T)
             assert_plan_equal(got, p, totals)

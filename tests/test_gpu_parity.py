@@ -199,6 +199,34 @@ def test_nan_and_negative_zero_payload_round_trips():
     run_dispatch(inp)
 
 
+# ---- planning with the hidden rows prefetched into L2 -------------------------------------------------
+@pytest.mark.parametrize("cfg", [0, 1, 2, 3])
+def test_plan_prefetch_gives_the_same_plan_and_payload(cfg):
+    # full size: the large_ep rows (117 MB) exceed the half of L2 the prefetch is limited to
+    run_dispatch(wl.make_dispatch(cfg), layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact",), separate=True, prefetch=True,
+                 repeats=2)
+
+
+@pytest.mark.parametrize("T", [0, 1, 255, 257, 1025])
+def test_plan_prefetch_token_counts(T):
+    inp = wl.make_random_dispatch(T + 3, T=T, K=3, E=40, R=10, H=40, pad_fraction=0.1)
+    run_dispatch(inp, max_tokens=1100, prefetch=True)
+
+
+def test_plan_prefetch_argument_errors():
+    torch = torch_mod()
+    inp = wl.make_random_dispatch(5, T=64, K=2, E=8, R=4, H=16)
+    ids = torch.from_numpy(inp.topk_ids).cuda()
+    e2r = torch.from_numpy(inp.expert_to_rank).cuda()
+    x = torch.from_numpy(inp.x.view(np.int16)).cuda()
+    with mw.Context(4, 8, 2, 64, 32) as ctx:
+        assert ctx.mw_plan_prefetch(ids, e2r, 64, None, check=False) == mw.MW_ERR_INVALID_ARG
+        assert ctx.mw_plan_prefetch(ids, e2r, 64, x.data_ptr() + 8, check=False) == mw.MW_ERR_ALIGNMENT
+        assert ctx.mw_plan_prefetch(ids, e2r, 65, x, check=False) == mw.MW_ERR_INVALID_ARG
+        assert ctx.mw_plan_prefetch(ids, e2r, 64, x, check=False) == mw.MW_OK
+        torch.cuda.synchronize()
+
+
 # ---- plan + dispatch in one call (single-launch path for small batches) ----------------------------
 @pytest.mark.parametrize("cfg,H", [("decode", None), ("tiny", None), ("decode", 72)])
 def test_one_call_small_batches_match(cfg, H):
