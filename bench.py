@@ -395,8 +395,12 @@ def fused_dispatch_measure(mw, wl, torch) -> dict:
             ctx.mw_plan(ids, e2r, T)
             dispatch(i)
 
+        def step_prefetch(i):
+            ctx.mw_plan_prefetch(ids, e2r, T, sets[i % 3][0])      # x comes out of L2; the receive slots are streamed
+            dispatch(i)
+
         out = {}
-        for name, fn, n in (("dispatch_us", dispatch, 200), ("step_us", step, 400)):
+        for name, fn, n in (("dispatch_us", dispatch, 200), ("step_us", step, 400), ("step_prefetch_us", step_prefetch, 400)):
             for i in range(6):
                 fn(i)
             torch.cuda.synchronize()

@@ -295,6 +295,7 @@ int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t 
     mw_copy_args a = base_args(ctx);
     a.mode = layout == MW_LAYOUT_MULTIWRITE ? MW_CP_DISPATCH_MW : MW_CP_DISPATCH_UC;
     a.src = (const uint8_t *)x;
+    a.src_in_l2 = ctx->prefetched == x && layout == MW_LAYOUT_MULTIWRITE;
     a.src_index = ctx->d.mw_row_token;
     a.dst = (uint8_t *)recv_base;
     a.dst_stride = recv_stride_bytes;

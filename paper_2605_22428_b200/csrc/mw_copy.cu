@@ -649,7 +649,7 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
     // 14336 bytes (59 MB of send rows) 85 -> 74 us; 8192 rows (117 MB, about the size of L2) 164 -> 154 us.
     // With send rows that are not in L2 the streaming stores cost 3 to 4 % instead, so only the deliver from a
     // MultiWrite send buffer is launched with kAfterPack (the unicast pack scatters rows of x, which come from DRAM).
-    const unsigned blk = kAfterPack ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
+    const unsigned blk = (kAfterPack && MODE == MW_CP_SCATTER) ? gridDim.x - 1 - blockIdx.x : blockIdx.x;
     // 32-bit on purpose: the division is on the way to the first load
     const int row = blk / a.chunks_per_row, piece = blk % a.chunks_per_row;
     // what decides whether the block has work is loaded together and looked at afterwards: one round trip
@@ -684,7 +684,8 @@ __global__ void __launch_bounds__(kRowsMaxVecs) k_copy_rows(const __grid_constan
 #pragma unroll
                 for (int k = 0; k < V; ++k)
                     if (off + k * step < a.row_bytes) {
-                        if constexpr (kAfterPack) __stcs((uint4 *)(d + off + k * step), v[k]);
+                        // one pass from prefetched rows: the send slot (destination 0) is kept, the receive slots stream
+                        if (kAfterPack && (MODE != MW_CP_DISPATCH_MW || qb + q > 0)) __stcs((uint4 *)(d + off + k * step), v[k]);
                         else *(uint4 *)(d + off + k * step) = v[k];
                     }
             }
@@ -785,7 +786,10 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_PAIR_DIRECT: err = rows_launch<1, MW_CP_PAIR_DIRECT>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_SEND: err = rows_launch<1, MW_CP_PAIR_SEND>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_FORWARD: err = rows_launch<2, MW_CP_PAIR_FORWARD>(grid, block, st, overlap, a); break;
-        case MW_CP_DISPATCH_MW: err = rows_launch<1, MW_CP_DISPATCH_MW>(grid, block, st, overlap, a); break;
+        case MW_CP_DISPATCH_MW:
+            err = a.src_in_l2 ? rows_launch<1, MW_CP_DISPATCH_MW, true>(grid, block, st, overlap, a)
+                              : rows_launch<1, MW_CP_DISPATCH_MW>(grid, block, st, overlap, a);
+            break;
         case MW_CP_DISPATCH_UC: err = rows_launch<1, MW_CP_DISPATCH_UC>(grid, block, st, overlap, a); break;
         case MW_CP_AG_FUSED_MW: err = rows_launch<1, MW_CP_AG_FUSED_MW>(grid, block, st, overlap, a); break;
         case MW_CP_AG_FUSED_UC: err = rows_launch<1, MW_CP_AG_FUSED_UC>(grid, block, st, overlap, a); break;

@@ -66,6 +66,7 @@ struct mw_ctx {
     uint32_t gbar_arrivals; // grid-barrier arrivals made by all previous fused plans
     int coop_ok;            // device supports cooperative launch
     int32_t planned_T;      // T of the latest plan, -1 before the first
+    const void *prefetched; // rows the latest plan launch brought into L2 (null: none)
     uint32_t gm_epoch;      // epoch of the plan the group-major arrays were made from (0: none)
     int64_t launches;
     // host staging (MW_FLAG_HOST_STAGING)
@@ -170,6 +171,7 @@ struct mw_copy_args {
     int stages;                // bulk-copy pipeline depth per warp
     int batch;                 // consecutive items claimed per work ticket
     int keep_in_l2;            // destination rows are read again soon: do not mark them evict-first
+    int src_in_l2;             // fused dispatch: the source rows were prefetched into L2 by the plan launch
     int loose_bound;           // host_rows may be far above the row count: take the persistent grid, which pays nothing for absent rows
     unsigned int *work_ctr;    // [2] ticket counter, finished-warp counter (both zero between launches)
     int Kd, R, dst_begin, dst_count;

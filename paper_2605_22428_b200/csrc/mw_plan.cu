@@ -841,6 +841,7 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     ctx->planned_T = T;
     // rows to bring into L2 meanwhile: the first half-L2 of them (the pack step reads them in ascending order)
     a.pf_base = (const uint8_t *)rows;
+    ctx->prefetched = nullptr;
     a.pf_bytes = rows ? (int64_t)T * ctx->cfg.row_bytes : 0;
     if (a.pf_bytes > ctx->l2_bytes / 2) a.pf_bytes = (ctx->l2_bytes / 2) & ~(int64_t)15;
     if (blocks <= ctx->sm_count && blocks <= MW_TILE && !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS)) {
@@ -862,6 +863,7 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
         } else {
             // with rows to prefetch, one more block for every SM the tiles leave free
             const int extra = a.pf_bytes > 0 ? ctx->sm_count - blocks : 0;
+            if (extra > 0 && a.pf_bytes == (int64_t)T * ctx->cfg.row_bytes) ctx->prefetched = rows;     // all of them fit
             e = mw_launch(fn, dim3(blocks + extra), dim3(MW_TILE), tile_smem_bytes(ctx), st, false, a);
         }
         if (e == cudaSuccess) {
@@ -870,6 +872,7 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
             return MW_OK;
         }
         cudaGetLastError();   // the launch was refused: take the multi-pass route
+        ctx->prefetched = nullptr;
     }
     k_plan_mask<<<blocks, MW_TILE, 0, st>>>(a);
     k_plan_tile<<<blocks, MW_TILE, tile_smem_bytes(ctx), st>>>(a);
