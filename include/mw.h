@@ -221,7 +221,10 @@ MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, i
  * to outweigh the savings) the three kernels are replaced by a single launch in which every
  * block recomputes the plan in shared memory and then moves its share of the rows; larger
  * batches, the unicast layout and contexts created with a plan or copy variant flag take the
- * ordinary three-kernel route.
+ * ordinary three-kernel route (planning through mw_plan_prefetch).
+ * The single launch keeps no state on the host, so a call captured into a CUDA graph may be replayed
+ * (new ids and rows in the same buffers).  mw_plan and mw_plan_prefetch may not: the look-back epoch
+ * and the barrier targets of their kernel are launch arguments that advance with every call.
  */
 MW_API int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
                             const void *x, int layout, void *send_buf, int64_t send_capacity_rows, void *recv_base,

@@ -4,18 +4,21 @@
 // Section 4.1 steps 3-5 and Section 4.3.3, the relay replicating a payload to every destination
 // named by its bitmap.)
 //
-// A work item is (row, chunk of at most 7168 bytes).  A persistent grid of one block per SM runs
-// one pipeline per warp; warps claim items through a ticket counter (work is claimed, not dealt).
+// k_copy_rows (the default): an ordinary grid with one block per (row, piece of at most 512 16-byte vectors);
+//                 a thread loads its vectors once and stores them to every destination of the row.  The deliver
+//                 from a MultiWrite send buffer walks the rows from the last to the first and streams its stores,
+//                 so that the send rows the pack launch just wrote are read from L2.
+// Behind flags, and for the relay's second level: a persistent grid of one block per SM, one pipeline per warp,
+// work item = (row, chunk of at most 7168 bytes), claimed through a ticket counter.
 //   k_copy_bulk   bulk asynchronous copies global -> shared (completion counted on an mbarrier),
 //                 several stages deep, then one shared -> global bulk copy per destination, issued
-//                 by different lanes.  A handful of instructions per row, the copy engines move the
-//                 bytes, and a row is read from memory exactly once.  The default.
+//                 by different lanes (MW_FLAG_COPY_BULK).
 //   k_copy_stage  same loads; the staged chunk is read once into registers and written to every
 //                 destination with 16-byte stores (MW_FLAG_COPY_REG_STORE).
 //   k_copy_ldst   no staging: 16-byte loads and stores through registers, static split
 //                 (MW_FLAG_COPY_LDST).
-// Measured on B200 (4096 rows of 14336 bytes, 7.7 copies each) the three differ by a few per cent;
-// all sit near 5.9 TB/s, about 90 % of what a plain device-to-device copy reaches.
+// Measured on B200 (4096 rows of 14336 bytes, 7.7 copies each): deliver 75 us with k_copy_rows after a pack
+// launch (6.8 TB/s), 88 us with k_copy_bulk.
 #include "mw_internal.cuh"
 
 namespace {
