@@ -473,6 +473,56 @@ def large_ep_measure(mw, wl, torch) -> dict:
     return out
 
 
+def two_stream_measure(mw, wl, torch) -> dict:
+    """The headline step with consecutive batches alternating between two contexts on two streams, so that the plan of
+    one batch (a latency chain on a few SMs) runs under the deliver of the previous one.  An orchestration the caller
+    chooses; the headline figure is the single-stream step."""
+    inp = wl.make_dispatch(WORKLOAD)
+    s = inp.shape
+    B, T = s.row_bytes, s.T
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    xh = torch.from_numpy(inp.x.view(np.int16))
+    ctxs = [mw.Context(s.R, s.E, s.K, T, B) for _ in range(2)]
+    try:
+        ctxs[0].mw_plan(ids, e2r, T)
+        tot = ctxs[0].mw_get_totals()
+        Tn, SD = tot["T_nonempty"], tot["total_dest"]
+        sets = [(xh.cuda(), torch.empty(Tn * B, dtype=torch.uint8, device="cuda"),
+                 torch.empty(SD * B, dtype=torch.uint8, device="cuda")) for _ in range(4)]
+        streams = [torch.cuda.Stream() for _ in range(2)]
+        main = torch.cuda.current_stream()
+
+        def step(i):
+            c, st = ctxs[i % 2], streams[i % 2]
+            x, send, recv = sets[i % 4]
+            c.mw_plan_prefetch(ids, e2r, T, x, stream=st)
+            c.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn, stream=st)
+            c.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD, stream=st)
+
+        for i in range(8):
+            step(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 400
+        a.record()
+        for st in streams:
+            st.wait_stream(main)
+        for i in range(n):
+            step(i)
+        for st in streams:
+            main.wait_stream(st)
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) * 1e3 / n
+        assert all(c.mw_get_totals()["status"] == 0 for c in ctxs)
+    finally:
+        for c in ctxs:
+            c.close()
+    nbytes = (3 * Tn + SD) * B
+    return {"step_us": round(us, 1), "step_gbs": round(nbytes / us / 1e3, 1), "tokens_per_s": round(T / us * 1e6, 1),
+            "note": "two contexts, two streams, batches alternate; time per step over 400 steps"}
+
+
 def order_measure(mw, wl, torch) -> dict:
     """Group-major receive order (Sections 4.3.1, 4.3.2) and expert index (Section 2.3.2) on the headline workload."""
     inp = wl.make_dispatch(WORKLOAD, payload=False)
@@ -761,6 +811,7 @@ def run_cuda(args):
             line["dispatch_fused"] = fused_dispatch_measure(mw, wl, torch)
             line["receiver_order"] = order_measure(mw, wl, torch)
             line["large_ep"] = large_ep_measure(mw, wl, torch)
+            line["two_streams"] = two_stream_measure(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:
