@@ -473,6 +473,69 @@ def large_ep_measure(mw, wl, torch) -> dict:
     return out
 
 
+def mid_batch_measure(mw, wl, torch) -> list:
+    """Batches between the decode shape and the prefill shape (the paper's batch 128 to 2k, Section 6.3), routing of the
+    headline workload: mw_plan_dispatch (one launch up to 1024 tokens) replayed from a CUDA graph, against the three
+    calls of the headline step launched one by one."""
+    out = []
+    for T in (128, 512, 1024, 2048):
+        inp = wl.make_dispatch(WORKLOAD, T=T)
+        s = inp.shape
+        B = s.row_bytes
+        ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+        xh = torch.from_numpy(inp.x.view(np.int16))
+        with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+            ctx.mw_plan(ids, e2r, T)
+            tot = ctx.mw_get_totals()
+            Tn, SD = tot["T_nonempty"], tot["total_dest"]
+            own = (2 * Tn + SD) * B
+            nset = max(3, int((300 << 20) // own) + 1)
+            sets = [(xh.cuda(), torch.empty(Tn * B, dtype=torch.uint8, device="cuda"),
+                     torch.empty(SD * B, dtype=torch.uint8, device="cuda")) for _ in range(nset)]
+
+            def one(i):
+                x, send, recv = sets[i % nset]
+                ctx.mw_plan_dispatch(ids, e2r, T, x, mw.MW_LAYOUT_MULTIWRITE, send, Tn, recv, 0, SD)
+
+            def three(i):
+                x, send, recv = sets[i % nset]
+                ctx.mw_plan_prefetch(ids, e2r, T, x)
+                ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+                ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
+
+            row = {"T": T, "own_bytes": own}
+            for i in range(2 * nset):
+                three(i)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(200):
+                three(i)
+            b.record()
+            torch.cuda.synchronize()
+            row["three_calls_us"] = round(a.elapsed_time(b) * 1e3 / 200, 1)
+            if T <= 1024:           # the single launch keeps no host-side state and can be replayed
+                one(0)
+                torch.cuda.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    for i in range(4 * nset):
+                        one(i)
+                for _ in range(3):
+                    graph.replay()
+                torch.cuda.synchronize()
+                a.record()
+                for _ in range(10):
+                    graph.replay()
+                b.record()
+                torch.cuda.synchronize()
+                row["one_call_graph_us"] = round(a.elapsed_time(b) * 1e3 / (40 * nset), 1)
+                row["one_call_gbs"] = round(own / row["one_call_graph_us"] / 1e3, 1)
+            assert ctx.mw_get_totals()["status"] == 0
+            out.append(row)
+    return out
+
+
 def two_stream_measure(mw, wl, torch) -> dict:
     """The headline step with consecutive batches alternating between two contexts on two streams, so that the plan of
     one batch (a latency chain on a few SMs) runs under the deliver of the previous one.  An orchestration the caller
@@ -812,6 +875,7 @@ def run_cuda(args):
             line["receiver_order"] = order_measure(mw, wl, torch)
             line["large_ep"] = large_ep_measure(mw, wl, torch)
             line["two_streams"] = two_stream_measure(mw, wl, torch)
+            line["mid_batches"] = mid_batch_measure(mw, wl, torch)
         line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
         line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
     if rank == 0:

@@ -216,10 +216,11 @@ MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, i
 
 /*
  * mw_plan followed by mw_dispatch in one call (same arguments, same results, the context is left
- * in the same state).  For small batches in the MultiWrite layout (T <= 256, R <= 256, min(K, R)
- * <= 16: the decode-sized batches of Section 6.3, where the paper finds the replication overhead
- * to outweigh the savings) the three kernels are replaced by a single launch in which every
- * block recomputes the plan in shared memory and then moves its share of the rows; larger
+ * in the same state).  For small batches in the MultiWrite layout (T <= 1024, R <= 256, min(K, R)
+ * <= 16: the batch sizes of Section 6.3, from the decode-sized ones, where the paper finds the
+ * replication overhead to outweigh the savings, up to its batch of 1k) the three kernels are
+ * replaced by a single launch in which every block recomputes the plan in shared memory and then
+ * moves its share of the rows (256 threads per block up to 128 tokens, 1024 beyond); larger
  * batches, the unicast layout and contexts created with a plan or copy variant flag take the
  * ordinary three-kernel route (planning through mw_plan_prefetch).
  * The single launch keeps no state on the host, so a call captured into a CUDA graph may be replayed

@@ -1,4 +1,5 @@
-// Single-launch plan + pack + deliver for small batches (decode-sized: T <= 256 tokens).
+// Single-launch plan + pack + deliver for small batches (T <= 1024 tokens: 256 threads per block for the
+// decode-sized ones, 1024 threads beyond 128 tokens).
 //
 // With a few dozen tokens the three-launch chain (plan, pack, deliver) is dominated by launch gaps and
 // by the plan's chain of global-memory round trips, the cost the paper reports for its small batches
@@ -17,10 +18,13 @@
 // The kernel keeps no state on the host or in global scratch, so a captured launch can be replayed.
 #include "mw_internal.cuh"
 
+#include <type_traits>
+
 namespace {
 
-constexpr int kSmallThreads = 256;     // = largest T
-constexpr int kSmallSlots = 512;       // bitmap table in shared memory (load <= 1/2)
+constexpr int kSmallThreads = 256;     // threads = largest T of the narrow variant (decode-sized batches)
+constexpr int kMidThreads = 1024;      // threads = largest T of the wide variant (batches of up to 1024 tokens)
+constexpr int kSmallNarrowBest = 128;  // up to this many tokens the 256-thread variant is the faster one
 constexpr int kSmallMaxKd = 16;
 constexpr int kSmallMaxW = 4;          // R <= 256: the three prefix sums fit one packed block scan
 constexpr int kSmallChunk = 2048;      // bytes of a row moved by one warp at a time (4 x 16 bytes per lane)
@@ -47,19 +51,23 @@ __device__ __forceinline__ uint64_t mix64s(uint64_t h, uint64_t v)
     return h;
 }
 
-// Exclusive prefix sum over the 256 threads of the block; `total` is returned to every thread.
-__device__ __forceinline__ uint32_t scan256(uint32_t v, uint32_t *warp_sums, uint32_t &total)
+// Exclusive prefix sum over the NT threads of the block; `total` is returned to every thread.  V is a packed word:
+// 32 bits hold the three sums of a 256-token batch, the 1024-token batch needs 64.
+template <int NT, class V>
+__device__ __forceinline__ V block_scan(V v, V *warp_sums, V &total)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t incl = v;
+    V incl = v;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += n; }
+    for (int o = 1; o < 32; o <<= 1) { const V n = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += n; }
     if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
-    uint32_t before = 0, sum = 0;
+    const V ws = lane < NT / 32 ? warp_sums[lane] : (V)0;
+    V wincl = ws;
 #pragma unroll
-    for (int w = 0; w < kSmallThreads / 32; ++w) { const uint32_t s = warp_sums[w]; if (w < warp) before += s; sum += s; }
-    total = sum;
+    for (int o = 1; o < NT / 32; o <<= 1) { const V n = __shfl_up_sync(0xffffffffu, wincl, o); if (lane >= o) wincl += n; }
+    total = __shfl_sync(0xffffffffu, wincl, NT / 32 - 1);
+    const V before = __shfl_sync(0xffffffffu, wincl - ws, warp);
     return before + incl - v;
 }
 
@@ -81,27 +89,35 @@ __device__ __forceinline__ int slot_rank(const SmallArgs &a, int p, int &id_out)
     return (r >= 0 && r < a.R) ? r : -1;
 }
 
-__global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_constant__ SmallArgs a)
+template <int NT>
+__global__ void __launch_bounds__(NT) k_dispatch_small(const __grid_constant__ SmallArgs a)
 {
+    constexpr int kSlots = 2 * NT;            // bitmap table in shared memory (load <= 1/2)
+    constexpr int kWords = NT / 32;           // 32-token words per rank row of the bit matrix
+    constexpr int kRow = kWords + 1;          // padded row
+    // packed scan word: leaders | members << kB1 | destinations << kB2 (NT = 256: 9 + 9 + 13 bits; 1024: 11 + 11 + 15)
+    using Packed = typename std::conditional<NT == 256, uint32_t, uint64_t>::type;
+    constexpr int kB1 = NT == 256 ? 9 : 11, kB2 = 2 * kB1;
+    constexpr Packed kM1 = ((Packed)1 << kB1) - 1;
     extern __shared__ __align__(16) uint8_t ssm[];
     // shared-memory layout (sizes depend on R, W, Kd)
-    uint64_t *mask64 = (uint64_t *)ssm;                                    // [256, W] bitmap of token t
+    uint64_t *mask64 = (uint64_t *)ssm;                                    // [NT, W] bitmap of token t
     uint32_t *mask32 = (uint32_t *)ssm;                                    //          the same words as 32-bit halves
-    unsigned long long *hkey = (unsigned long long *)(mask64 + kSmallThreads * a.W);   // [512] (hash tag, first claimant)
-    int *hlead = (int *)(hkey + kSmallSlots);                              // [512] smallest token with that bitmap
-    int *hcnt = hlead + kSmallSlots;                                       // [512] tokens with that bitmap
-    int *hrun = hcnt + kSmallSlots;                                        // [512] members counted so far (rank inside a group)
-    uint32_t *bits = (uint32_t *)(hrun + kSmallSlots);                     // [R, 9] bit t of row r: token t targets rank r (padded rows)
-    int *pre = (int *)(bits + a.R * 9);                                    // [R, 9] tokens before each 32-token word that target r
-    int *ro = pre + a.R * 9;                                               // [R + 1] region starts
-    int *nd_s = ro + a.R + 1;                                              // [256] destinations of token t
-    int *gid_s = nd_s + kSmallThreads;                                     // [256] group id, at the leader's index
-    int *goff_s = gid_s + kSmallThreads;                                   // [256] group offset, at the leader's index
-    int *tok_row_s = goff_s + kSmallThreads;                               // [256] send row of token t, -1 if none
-    int *row_token_s = tok_row_s + kSmallThreads;                          // [256] token of send row j
-    int *row_nd_s = row_token_s + kSmallThreads;                           // [256] destinations of send row j
-    int *row_flat_s = row_nd_s + kSmallThreads;                            // [256, Kd] destination rows (rank<<16|slot when strided)
-    __shared__ uint32_t warp_sums[kSmallThreads / 32];
+    unsigned long long *hkey = (unsigned long long *)(mask64 + NT * a.W);   // [2 NT] (hash tag, first claimant)
+    int *hlead = (int *)(hkey + kSlots);                              // [2 NT] smallest token with that bitmap
+    int *hcnt = hlead + kSlots;                                       // [2 NT] tokens with that bitmap
+    int *hrun = hcnt + kSlots;                                        // [2 NT] members counted so far (rank inside a group)
+    uint32_t *bits = (uint32_t *)(hrun + kSlots);                     // [R, NT/32 + 1] bit t of row r: token t targets rank r (padded rows)
+    int *pre = (int *)(bits + a.R * kRow);                                    // [R, NT/32 + 1] tokens before each 32-token word that target r
+    int *ro = pre + a.R * kRow;                                               // [R + 1] region starts
+    int *nd_s = ro + a.R + 1;                                              // [NT] destinations of token t
+    int *gid_s = nd_s + NT;                                     // [NT] group id, at the leader's index
+    int *goff_s = gid_s + NT;                                   // [NT] group offset, at the leader's index
+    int *tok_row_s = goff_s + NT;                               // [NT] send row of token t, -1 if none
+    int *row_token_s = tok_row_s + NT;                          // [NT] token of send row j
+    int *row_nd_s = row_token_s + NT;                           // [NT] destinations of send row j
+    int *row_flat_s = row_nd_s + NT;                            // [NT, Kd] destination rows (rank<<16|slot when strided)
+    __shared__ Packed warp_sums[32];
     __shared__ int s_acc[3];
 
     const int tid = threadIdx.x, t = tid, lane = tid & 31, warp = tid >> 5;
@@ -116,9 +132,9 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
 
     // ---- clear the tables (no global memory involved: overlaps the tail of the previous kernel) ----
     grid_launch_dependents();
-    for (int i = tid; i < kSmallThreads * a.W; i += kSmallThreads) mask64[i] = 0;
-    for (int i = tid; i < kSmallSlots; i += kSmallThreads) { hkey[i] = ~0ull; hlead[i] = 0x7fffffff; hcnt[i] = 0; hrun[i] = 0; }
-    for (int i = tid; i < a.R * 9; i += kSmallThreads) bits[i] = 0;
+    for (int i = tid; i < NT * a.W; i += NT) mask64[i] = 0;
+    for (int i = tid; i < kSlots; i += NT) { hkey[i] = ~0ull; hlead[i] = 0x7fffffff; hcnt[i] = 0; hrun[i] = 0; }
+    for (int i = tid; i < a.R * kRow; i += NT) bits[i] = 0;
     if (tid < 3) s_acc[tid] = 0;
     grid_dependency_wait();        // the previous dispatch may still read the plan arrays this launch rewrites
     __syncthreads();
@@ -127,7 +143,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
     //      OR = several experts on one rank count once), token bit in the rank's row ----
     {
         int valid = 0, bad = 0;
-        for (int p = tid; p < pairs; p += kSmallThreads) {
+        for (int p = tid; p < pairs; p += NT) {
             int id;
             const int r = slot_rank(a, p, id);
             bad |= (id != -1 && r < 0);
@@ -135,7 +151,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
             ++valid;
             const int tk = p / a.K;
             atomicOr(mask32 + tk * 2 * a.W + (r >> 5), 1u << (r & 31));
-            atomicOr(bits + r * 9 + (tk >> 5), 1u << (tk & 31));
+            atomicOr(bits + r * kRow + (tk >> 5), 1u << (tk & 31));
         }
         valid = __reduce_add_sync(0xffffffffu, valid);
         bad = __reduce_or_sync(0xffffffffu, (unsigned)bad);
@@ -156,8 +172,8 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
         if (nd > 0) {
             const uint32_t tag = (uint32_t)(h >> 32);
             const unsigned long long mine = ((unsigned long long)tag << 32) | (uint32_t)t;
-            slot = (int)(h & (kSmallSlots - 1));
-            for (int probes = 0; probes < kSmallSlots; ++probes) {
+            slot = (int)(h & (kSlots - 1));
+            for (int probes = 0; probes < kSlots; ++probes) {
                 const unsigned long long cur = atomicCAS(hkey + slot, ~0ull, mine);
                 if (cur == ~0ull) break;
                 if ((uint32_t)(cur >> 32) == tag) {
@@ -166,7 +182,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
                     for (int w = 0; w < a.W; ++w) same &= (om[w] == mask64[t * a.W + w]);
                     if (same) break;
                 }
-                slot = (slot + 1) & (kSmallSlots - 1);
+                slot = (slot + 1) & (kSlots - 1);
             }
             atomicMin(hlead + slot, t);
             atomicAdd(hcnt + slot, 1);
@@ -176,21 +192,22 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
     int my_cnt = 0;                // tokens that target rank `tid`
     if (tid < a.R) {
 #pragma unroll
-        for (int w8 = 0; w8 < 8; ++w8) { pre[tid * 9 + w8] = my_cnt; my_cnt += __popc(bits[tid * 9 + w8]); }
+        for (int w8 = 0; w8 < kWords; ++w8) { pre[tid * kRow + w8] = my_cnt; my_cnt += __popc(bits[tid * kRow + w8]); }
     }
     __syncthreads();
 
     // ---- group ids, group offsets and region starts: three exclusive prefix sums in one packed scan
-    //      (leaders <= 256: 9 bits, members <= 256: 9 bits, destinations <= 256 * 16: 13 bits) ----
+    //      (leaders <= NT, members <= NT, destinations <= 16 NT) ----
     const int leader = nd > 0 ? hlead[slot] : -1;
     const int gcount = nd > 0 ? hcnt[slot] : 0;
     const bool is_leader = nd > 0 && leader == t;
-    uint32_t total;
-    const uint32_t excl = scan256((is_leader ? 1u | ((uint32_t)gcount << 9) : 0u) | ((uint32_t)my_cnt << 18), warp_sums, total);
-    const int G = (int)(total & 511u), Tn = (int)((total >> 9) & 511u), SD = (int)(total >> 18);
-    const int goff_mine = (int)((excl >> 9) & 511u);
-    if (is_leader) { gid_s[tid] = (int)(excl & 511u); goff_s[tid] = goff_mine; }
-    if (tid < a.R) ro[tid] = (int)(excl >> 18);
+    Packed total;
+    const Packed excl = block_scan<NT, Packed>((is_leader ? (Packed)1 | ((Packed)gcount << kB1) : (Packed)0) | ((Packed)my_cnt << kB2),
+                                               warp_sums, total);
+    const int G = (int)(total & kM1), Tn = (int)((total >> kB1) & kM1), SD = (int)(total >> kB2);
+    const int goff_mine = (int)((excl >> kB1) & kM1);
+    if (is_leader) { gid_s[tid] = (int)(excl & kM1); goff_s[tid] = goff_mine; }
+    if (tid < a.R) ro[tid] = (int)(excl >> kB2);
     if (tid == 0) ro[a.R] = SD;
 
     // ---- rank inside the group, in token order.  Only when some group has more than one member: the warps
@@ -200,7 +217,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
         const int key = (nd > 0 && gcount > 1) ? slot : -1 - lane;       // negative keys are unique: groups of one
         const unsigned same = __match_any_sync(0xffffffffu, key);
         const int first = __ffs(same) - 1;
-        for (int turn = 0; turn < kSmallThreads / 32; ++turn) {
+        for (int turn = 0; turn < NT / 32; ++turn) {
             if (warp == turn) {
                 int base = 0;
                 if (key >= 0 && lane == first) base = atomicAdd(hrun + slot, __popc(same));
@@ -226,7 +243,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
 
     // ---- one thread per expert slot: place among the token's destinations (= set bits below r), slot inside
     //      the region (= earlier tokens that target r), descriptors ----
-    for (int p = tid; p < pairs; p += kSmallThreads) {
+    for (int p = tid; p < pairs; p += NT) {
         int id;
         const int r = slot_rank(a, p, id);
         if (r < 0) continue;
@@ -234,7 +251,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
         const uint64_t *m = mask64 + tk * a.W;
         int i = __popcll(m[r >> 6] & ((1ull << (r & 63)) - 1ull));
         for (int w = 0; w < (r >> 6); ++w) i += __popcll(m[w]);
-        const int pos = pre[r * 9 + wi] + __popc(bits[r * 9 + wi] & ((1u << (tk & 31)) - 1u));
+        const int pos = pre[r * kRow + wi] + __popc(bits[r * kRow + wi] & ((1u << (tk & 31)) - 1u));
         const int flat = ro[r] + pos, rowk = tok_row_s[tk];
         row_flat_s[rowk * a.Kd + i] = a.recv_stride ? ((r << 16) | pos) : flat;
         overflow |= (a.recv_stride ? pos : flat) >= a.recv_capacity_rows;
@@ -255,7 +272,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
     if (writes(0)) {
         // rows that do not fit their buffer are skipped by whichever block meets them; the status is written here
         overflow = __syncthreads_or(overflow);
-        for (int r = tid; r <= a.R; r += kSmallThreads) a.rank_offsets[r] = ro[r];
+        for (int r = tid; r <= a.R; r += NT) a.rank_offsets[r] = ro[r];
         if (tid == 0) {
             const int64_t self_copies = a.src_rank >= 0 ? ro[a.src_rank + 1] - ro[a.src_rank] : 0;
             const int64_t sent_rows = (int64_t)Tn - s_acc[1];
@@ -271,7 +288,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
             *a.totals = tt;
         }
         // tails
-        for (int u = tid; u <= a.T; u += kSmallThreads) {
+        for (int u = tid; u <= a.T; u += NT) {
             if (u > G) a.group_offsets[u] = -1;
             if (u == G) a.group_offsets[u] = Tn;
             if (u < a.T) {
@@ -280,7 +297,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
                     for (int w = 0; w < a.W; ++w) a.group_mask[(int64_t)u * a.W + w] = 0;
             }
         }
-        for (int q = SD + tid; q < a.T * a.Kd; q += kSmallThreads) a.rank_tokens[q] = -1;
+        for (int q = SD + tid; q < a.T * a.Kd; q += NT) a.rank_tokens[q] = -1;
     }
     if (writes(1) && active) {
         for (int w = 0; w < a.W; ++w) a.token_mask[(int64_t)t * a.W + w] = mask64[t * a.W + w];
@@ -300,7 +317,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
     if (writes(2) || writes(3)) {
         // unused entries: -1
         const bool lists = writes(2), planes = writes(3);
-        for (int q = tid; q < a.T * a.Kd; q += kSmallThreads) {
+        for (int q = tid; q < a.T * a.Kd; q += NT) {
             const int tk = q / a.Kd, i = q % a.Kd, n = nd_s[tk];
             if (i < n) continue;
             if (lists) { a.dest_rank[q] = -1; a.dest_pos[q] = -1; }
@@ -315,7 +332,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
     // ---- rows: every warp of the moving blocks takes (send row, chunk) items round robin ----
     const int chunks = (int)((a.row_bytes + kSmallChunk - 1) / kSmallChunk);
     const int items = Tn * chunks;
-    const int warps = movers * (kSmallThreads / 32);
+    const int warps = movers * (NT / 32);
     for (int item = warp * movers + mover; item < items; item += warps) {
         const int j = item / chunks;
         const int64_t off = (int64_t)(item % chunks) * kSmallChunk;
@@ -350,10 +367,15 @@ __global__ void __launch_bounds__(kSmallThreads) k_dispatch_small(const __grid_c
     }
 }
 
-size_t small_smem_bytes(const mw_ctx *ctx)
+size_t small_smem_bytes(const mw_ctx *ctx, int NT)
 {
-    const size_t R = (size_t)ctx->cfg.R, W = (size_t)ctx->W, Kd = (size_t)ctx->Kd;
-    return kSmallThreads * W * 8 + kSmallSlots * 20 + R * 9 * 8 + (R + 1) * 4 + 6 * kSmallThreads * 4 + kSmallThreads * Kd * 4 + 64;
+    const size_t R = (size_t)ctx->cfg.R, W = (size_t)ctx->W, Kd = (size_t)ctx->Kd, N = (size_t)NT;
+    return N * W * 8 + 2 * N * 20 + R * (N / 32 + 1) * 8 + (R + 1) * 4 + 6 * N * 4 + N * Kd * 4 + 64;
+}
+
+bool small_fits(const mw_ctx *ctx, int NT)
+{
+    return ctx->W <= kSmallMaxW && ctx->Kd <= kSmallMaxKd && small_smem_bytes(ctx, NT) + 1024 <= (size_t)ctx->max_smem_optin;
 }
 
 }  // namespace
@@ -361,17 +383,20 @@ size_t small_smem_bytes(const mw_ctx *ctx)
 // True if the single-launch path can serve this context and batch.
 bool mw_small_applies(const mw_ctx *ctx, int32_t T, int layout)
 {
-    return T <= kSmallThreads && layout == MW_LAYOUT_MULTIWRITE && ctx->W <= kSmallMaxW && ctx->Kd <= kSmallMaxKd &&
+    return layout == MW_LAYOUT_MULTIWRITE &&
            !(ctx->cfg.flags & (MW_FLAG_PLAN_MULTIPASS | MW_FLAG_PLAN_COOPERATIVE | MW_FLAG_COPY_LDST | MW_FLAG_COPY_REG_STORE)) &&
-           small_smem_bytes(ctx) + 1024 <= (size_t)ctx->max_smem_optin;
+           ((T <= kSmallThreads && small_fits(ctx, kSmallThreads)) || (T <= kMidThreads && small_fits(ctx, kMidThreads)));
 }
 
 int mw_small_setup(mw_ctx *ctx)
 {
-    const size_t need = small_smem_bytes(ctx);
-    if (ctx->W > kSmallMaxW || ctx->Kd > kSmallMaxKd || need + 1024 > (size_t)ctx->max_smem_optin) return MW_OK;   // path not available
-    if (need > 48 * 1024 &&
-        cudaFuncSetAttribute(k_dispatch_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)
+    if (small_fits(ctx, kSmallThreads) && small_smem_bytes(ctx, kSmallThreads) > 48 * 1024 &&
+        cudaFuncSetAttribute(k_dispatch_small<kSmallThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)small_smem_bytes(ctx, kSmallThreads)) != cudaSuccess)
+        return MW_ERR_CUDA;
+    if (small_fits(ctx, kMidThreads) && small_smem_bytes(ctx, kMidThreads) > 48 * 1024 &&
+        cudaFuncSetAttribute(k_dispatch_small<kMidThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)small_smem_bytes(ctx, kMidThreads)) != cudaSuccess)
         return MW_ERR_CUDA;
     return MW_OK;
 }
@@ -396,8 +421,14 @@ int mw_small_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_
     a.rank_tokens = d.rank_tokens; a.dest_rank = d.dest_rank; a.dest_pos = d.dest_pos; a.token_leader = d.token_leader;
     a.row_ndest = d.row_ndest; a.row_dest_rank = d.row_dest_rank; a.row_dest_pos = d.row_dest_pos;
     a.row_dest_flat = d.row_dest_flat; a.totals = d.totals;
-    const cudaError_t e = mw_launch(k_dispatch_small, dim3(ctx->sm_count), dim3(kSmallThreads), small_smem_bytes(ctx), st,
-                                    !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP), a);
+    // Measured on B200 (plan part alone, 64 ranks, top-8; microseconds per call back to back, 256 / 1024 threads):
+    // 64 tokens 4.9 / 5.3, 128 tokens 6.0 / 6.0, 192 tokens 8.4 / 6.9, 256 tokens 10.2 / 8.4.
+    const bool narrow = T <= kSmallThreads && small_fits(ctx, kSmallThreads) && (T <= kSmallNarrowBest || !small_fits(ctx, kMidThreads));
+    const cudaError_t e = !narrow
+        ? mw_launch(k_dispatch_small<kMidThreads>, dim3(ctx->sm_count), dim3(kMidThreads), small_smem_bytes(ctx, kMidThreads), st,
+                    !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP), a)
+        : mw_launch(k_dispatch_small<kSmallThreads>, dim3(ctx->sm_count), dim3(kSmallThreads), small_smem_bytes(ctx, kSmallThreads), st,
+                    !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP), a);
     ctx->launches += 1;
     ctx->planned_T = T;
     ctx->epoch += 2;          // a new plan (keeps the parity the tiled plan's double-buffered accumulators rely on)

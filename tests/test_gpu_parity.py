@@ -234,11 +234,23 @@ def test_one_call_small_batches_match(cfg, H):
     run_dispatch(wl.make_dispatch(cfg, 100, H=H), one_call=True)
 
 
-@pytest.mark.parametrize("T", [0, 1, 31, 255, 256, 257, 600])
+@pytest.mark.parametrize("T", [0, 1, 31, 128, 129, 255, 256, 257, 600, 1023, 1024, 1025, 1500])
 def test_one_call_token_counts(T):
-    # up to 256 tokens the single launch is taken, beyond that the three-kernel route: same results
+    # up to 128 tokens the single launch with 256 threads per block, up to 1024 tokens the one with 1024 threads,
+    # beyond that the three-kernel route: same results
     inp = wl.make_random_dispatch(T + 11, T=T, K=3, E=40, R=10, H=40, pad_fraction=0.1)
-    run_dispatch(inp, one_call=True, max_tokens=700)
+    run_dispatch(inp, one_call=True, max_tokens=1600)
+
+
+@pytest.mark.parametrize("cfg,T,H", [("dsv3_prefill", 1024, 72), ("dsv3_prefill", 700, None), ("large_ep", 1000, 40), ("decode", 1024, 24)])
+def test_one_call_wide_variant_on_the_configurations_routing(cfg, T, H):
+    # one bitmap word (64 ranks), two (128) and four (256); 700 tokens of full-size rows
+    run_dispatch(wl.make_dispatch(cfg, 100, T=T, H=H), one_call=True)
+
+
+def test_one_call_wide_variant_groups_and_sixteen_destinations():
+    run_dispatch(wl.make_random_dispatch(21, T=1000, K=2, E=8, R=4, H=16), one_call=True)                 # few groups of hundreds
+    run_dispatch(wl.make_random_dispatch(22, T=900, K=16, E=64, R=32, H=16, pad_fraction=0.2), one_call=True, src_rank=5)
 
 
 def test_one_call_groups_padding_invalid_ids_and_source_rank():
