@@ -433,6 +433,24 @@ def test_allgather_parity(layout, R, S, begin, count, strided, flags):
     assert send.guards_intact() and recv.guards_intact()
 
 
+def test_allgather_largest_shard_of_the_sweep():
+    """64 ranks x 64 MB shards (4 GB of shards), the top of the size sweep; one destination region is materialised."""
+    torch = torch_mod()
+    R, S = 64, 64 << 20
+    sh = wl.make_allgather_shards(R, S, seed=4)
+    want_send, want_recv, want_tot, ret = mwo.allgather(sh, mw.MW_LAYOUT_MULTIWRITE, 5, 1, 0, SENTINEL)
+    assert ret == 0
+    sh_d = torch.from_numpy(sh).cuda()
+    send, recv = Guarded(len(want_send)), Guarded(len(want_recv))
+    with mw.Context(R, 8, 2, 16, 32) as ctx:
+        rc, tot = ctx.mw_allgather_pack(sh_d, S, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), recv.ptr(), 0, 5, 1)
+        torch.cuda.synchronize()
+    assert tot == want_tot
+    assert torch.equal(send.body.cpu(), torch.from_numpy(want_send))
+    assert torch.equal(recv.body.cpu(), torch.from_numpy(want_recv))
+    assert send.guards_intact() and recv.guards_intact()
+
+
 # ---- the host-buffer entry point ---------------------------------------------------------------------
 @pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
 def test_dispatch_from_host_buffers(layout):
