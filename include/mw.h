@@ -207,6 +207,20 @@ MW_API int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_
                int64_t recv_capacity_rows, void *stream);
 
 /*
+ * mw_deliver with every receive region named by its own base address, the form the paper gives its interface
+ * (Section 4.3.2: used like a standard write, but accepts an array of remote buffer addresses instead of one;
+ * Section 4.3.1: the payload is written into buffer B_i at every destination D_i).
+ *   recv_ptrs           device, array of R addresses (8-byte aligned array); entry r is the start of region(r),
+ *                       16-byte aligned, room for recv_capacity_rows rows.  Entries of ranks that receive nothing
+ *                       are not looked at.  The addresses are read on the device: a null or misaligned entry of a
+ *                       rank that does receive rows sets MW_ERR_INVALID_ARG / MW_ERR_ALIGNMENT in the accounting
+ *                       status (mw_get_totals) and that region is not written.
+ * Same rows in the same order as mw_deliver.
+ */
+MW_API int mw_deliver_ptrs(mw_ctx *ctx, int layout, const void *send_buf, void *const *recv_ptrs,
+                    int64_t recv_capacity_rows, void *stream);
+
+/*
  * The whole data movement of one dispatch, with the results of mw_pack followed by mw_deliver (same send buffer,
  * same receive regions, bit for bit) but in one pass: every hidden row is read once and written to its send
  * slot(s) and to all its receive slots.  With a MW_FLAG_COPY_* bit set it is the two calls in sequence.

@@ -33,7 +33,7 @@ MW_FLAG_COPY_BULK = 0x40
 
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
-EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_plan_prefetch", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_dispatch", "mw_plan_dispatch",
+EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_plan_prefetch", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_deliver_ptrs", "mw_dispatch", "mw_plan_dispatch",
            "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_group_major", "mw_deliver_group_major", "mw_expert_index",
            "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
            "mw_strerror", "mw_pair_balanced_direct_bytes") + RELAY_EXPORTS
@@ -116,6 +116,7 @@ def lib():
         L.mw_get_totals.argtypes = [vp, C.POINTER(mw_totals), vp]
         L.mw_pack.argtypes = [vp, vp, C.c_int, vp, i64, vp]
         L.mw_deliver.argtypes = [vp, C.c_int, vp, vp, i64, i64, vp]
+        L.mw_deliver_ptrs.argtypes = [vp, C.c_int, vp, vp, i64, vp]
         L.mw_dispatch.argtypes = [vp, vp, C.c_int, vp, i64, vp, i64, i64, vp]
         L.mw_plan_dispatch.argtypes = [vp, vp, vp, i32, vp, C.c_int, vp, i64, vp, i64, i64, C.POINTER(mw_plan_view), vp]
         L.mw_allgather_pack.argtypes = [vp, vp, i64, C.c_int, vp, vp, i64, i32, i32, C.POINTER(mw_totals), vp]
@@ -141,7 +142,7 @@ def lib():
             getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:19]:
+        for name in EXPORTS[:20]:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -274,6 +275,13 @@ class Context:
                               _stream(stream))
         if check and rc != MW_OK:
             raise MwError(rc, "mw_deliver")
+        return rc
+
+    def mw_deliver_ptrs(self, layout: int, send_buf, recv_ptrs, recv_capacity_rows: int, stream=None, check: bool = True) -> int:
+        """recv_ptrs: device int64 tensor (or address) holding the R region base addresses."""
+        rc = lib().mw_deliver_ptrs(self._h, layout, _ptr(send_buf), _ptr(recv_ptrs), recv_capacity_rows, _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_deliver_ptrs")
         return rc
 
     def mw_dispatch(self, x, layout: int, send_buf, send_capacity_rows: int, recv, recv_stride_bytes: int,

@@ -278,6 +278,32 @@ int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_base, i
     return mw_copy_launch(ctx, a, as_stream(stream));
 }
 
+int mw_deliver_ptrs(mw_ctx *ctx, int layout, const void *send_buf, void *const *recv_ptrs, int64_t recv_capacity_rows,
+                    void *stream)
+{
+    if (!ctx || !send_buf || !recv_ptrs || recv_capacity_rows < 0 || check_layout(layout)) return MW_ERR_INVALID_ARG;
+    if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
+    if (!aligned16(send_buf) || ((uintptr_t)recv_ptrs & 7u)) return MW_ERR_ALIGNMENT;
+    mw_copy_args a = base_args(ctx);
+    a.src = (const uint8_t *)send_buf;
+    a.dst_ptrs = (uint8_t *const *)recv_ptrs;
+    a.capacity_rows = recv_capacity_rows;
+    if (layout == MW_LAYOUT_MULTIWRITE) {
+        a.mode = MW_CP_SCATTER;
+        a.rows_from = 1;
+        a.ndst = ctx->d.row_ndest;
+        a.d_rank = ctx->d.row_dest_rank;
+        a.d_pos = ctx->d.row_dest_pos;
+        a.d_flat = ctx->d.row_dest_flat;
+        a.host_rows = ctx->planned_T;
+    } else {
+        a.mode = MW_CP_DELIVER_UC;
+        a.rows_from = 2;
+        a.host_rows = (int64_t)ctx->planned_T * ctx->Kd;
+    }
+    return mw_copy_launch(ctx, a, as_stream(stream));
+}
+
 int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows,
                 void *recv_base, int64_t recv_stride_bytes, int64_t recv_capacity_rows, void *stream)
 {

@@ -171,8 +171,25 @@ __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row, int mod
 __device__ __forceinline__ int n_dst(const mw_copy_args &a, int64_t row) { return n_dst(a, row, a.mode); }
 
 // Receive slot of destination q of send row `row` (plan descriptors in plane layout).
+// Region r given by its own base address (Section 4.3.2: a write that takes an array of remote buffer addresses).
+// The addresses live in device memory, so they are checked here: a null or misaligned one is reported, nothing is written.
+__device__ __forceinline__ uint8_t *region_base(const mw_copy_args &a, int r)
+{
+    uint8_t *base = a.dst_ptrs[r];
+    if (!base) { flag_error(a, MW_ERR_INVALID_ARG); return nullptr; }
+    if ((uintptr_t)base & 15u) { flag_error(a, MW_ERR_ALIGNMENT); return nullptr; }
+    return base;
+}
+
 __device__ __forceinline__ uint8_t *scatter_dst(const mw_copy_args &a, int64_t row, int q)
 {
+    if (a.dst_ptrs) {
+        const int r = a.d_rank[q * a.d_stride + row], p = a.d_pos[q * a.d_stride + row];
+        if (r < 0) return nullptr;
+        if (p >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+        uint8_t *base = region_base(a, r);
+        return base ? base + (int64_t)p * a.row_bytes : nullptr;
+    }
     if (a.dst_stride) {
         const int r = a.d_rank[q * a.d_stride + row], p = a.d_pos[q * a.d_stride + row];
         if (r < 0) return nullptr;
@@ -209,7 +226,7 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
         return a.dst2 + at * a.row_bytes;
     }
     case MW_CP_DELIVER_UC: {
-        if (!a.dst_stride) {
+        if (!a.dst_stride && !a.dst_ptrs) {
             if (row >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
             return a.dst + row * a.row_bytes;
         }
@@ -221,6 +238,10 @@ __device__ __forceinline__ uint8_t *dst_row(const mw_copy_args &a, int64_t row, 
         }
         const int64_t p = row - a.rank_offsets[lo];
         if (p >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+        if (a.dst_ptrs) {
+            uint8_t *base = region_base(a, lo);
+            return base ? base + p * a.row_bytes : nullptr;
+        }
         return a.dst + (int64_t)lo * a.dst_stride + p * a.row_bytes;
     }
     case MW_CP_AG_DELIVER_MW: return a.dst + (int64_t)q * a.dst_stride + row * a.row_bytes;
@@ -281,7 +302,7 @@ __device__ __forceinline__ RawDesc fetch_raw(const mw_copy_args &a, int64_t row,
     if (a.mode == MW_CP_SCATTER) {
         d.n = a.ndst[row];
         if (lane < a.Kd) {
-            if (a.dst_stride) { d.x = a.d_rank[lane * a.d_stride + row]; d.y = a.d_pos[lane * a.d_stride + row]; }
+            if (a.dst_stride || a.dst_ptrs) { d.x = a.d_rank[lane * a.d_stride + row]; d.y = a.d_pos[lane * a.d_stride + row]; }
             else d.x = a.d_flat[lane * a.d_stride + row];
         }
     }
@@ -295,6 +316,11 @@ __device__ __forceinline__ uint8_t *resolve_dst(const mw_copy_args &a, int64_t r
     case MW_CP_SCATTER: {
         *nd = d.n;
         if (lane >= d.n || d.x < 0) return nullptr;
+        if (a.dst_ptrs) {
+            if (d.y >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
+            uint8_t *base = region_base(a, d.x);
+            return base ? base + (int64_t)d.y * a.row_bytes : nullptr;
+        }
         if (a.dst_stride) {
             if (d.y >= a.capacity_rows) { flag_error(a, MW_ERR_CAPACITY); return nullptr; }
             return a.dst + (int64_t)d.x * a.dst_stride + (int64_t)d.y * a.row_bytes;

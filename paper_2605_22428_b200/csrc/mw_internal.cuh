@@ -158,6 +158,7 @@ struct mw_copy_args {
     const uint8_t *src;        // source rows (x, send buffer or shards)
     const uint8_t *src2;       // AllGather unicast deliver: the shards (own copy is local)
     uint8_t *dst;              // destination base
+    uint8_t *const *dst_ptrs;  // deliver: device array [R] of region base addresses (then dst and dst_stride are unused), or null
     uint8_t *dst2;             // paired AllGather, relayed segment: the receive area (own copy), dst being the relay area;
                                // fused dispatch: the send buffer
     int64_t row_bytes;         // bytes per row (B, or the shard size)

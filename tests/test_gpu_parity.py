@@ -409,6 +409,74 @@ def test_host_side_argument_errors():
     assert mw.strerror(mw.MW_ERR_TIMEOUT) and mw.strerror(12345) == "unknown error code"
 
 
+# ---- deliver into regions named by an array of addresses (Section 4.3.2) ------------------------------------
+@pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
+@pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
+def test_deliver_to_an_array_of_region_addresses(layout, flags):
+    torch = torch_mod()
+    for inp in (wl.make_random_dispatch(61, T=700, K=4, E=32, R=16, H=24, pad_fraction=0.1), wl.make_dispatch("dsv3_prefill", 100, T=1500, H=264)):
+        s = inp.shape
+        B, R = s.row_bytes, s.R
+        p = mwo.plan(inp.topk_ids, inp.expert_to_rank, R, B)
+        counts = np.diff(p.rank_offsets)
+        cap = int(counts.max()) + 1
+        send_want = mwo.pack_mw(p, inp.x) if layout == mw.MW_LAYOUT_MULTIWRITE else mwo.pack_uc(p, inp.x)
+        strided = (mwo.deliver_mw if layout == mw.MW_LAYOUT_MULTIWRITE else mwo.deliver_uc)(p, send_want, cap * B, SENTINEL)
+        # regions scattered over one buffer in a shuffled order with uneven 16-byte gaps
+        rng = np.random.default_rng(5)
+        order, offs, at = rng.permutation(R), np.zeros(R, np.int64), 0
+        for r in order:
+            at += 16 * int(rng.integers(0, 9))
+            offs[r] = at
+            at += cap * B
+        area = Guarded(at + 64)
+        want = np.full(at + 64, SENTINEL, np.uint8)
+        for r in range(R):
+            want[offs[r]:offs[r] + counts[r] * B] = strided[r * cap * B:r * cap * B + counts[r] * B]
+        ptrs = torch.from_numpy(offs + area.ptr()).cuda()
+        ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+        x = torch.from_numpy(inp.x.view(np.int16)).cuda()
+        send = Guarded(len(send_want.reshape(-1)))
+        with mw.Context(R, s.E, s.K, inp.T, B, flags=flags) as ctx:
+            ctx.mw_plan(ids, e2r, inp.T)
+            ctx.mw_pack(x, layout, send.ptr(), len(send_want))
+            ctx.mw_deliver_ptrs(layout, send.ptr(), ptrs, cap)
+            assert ctx.mw_get_totals()["status"] == 0
+            assert np.array_equal(area.host(), want)
+            assert area.guards_intact() and send.guards_intact()
+
+
+def test_deliver_ptrs_reports_bad_addresses_and_capacity():
+    torch = torch_mod()
+    inp = wl.make_random_dispatch(62, T=300, K=3, E=12, R=6, H=8)
+    s = inp.shape
+    B, R = s.row_bytes, s.R
+    p = mwo.plan(inp.topk_ids, inp.expert_to_rank, R, B)
+    cap = int(np.diff(p.rank_offsets).max())
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    x = torch.from_numpy(inp.x.view(np.int16)).cuda()
+    area = Guarded(R * cap * B)
+    good = np.arange(R, dtype=np.int64) * cap * B + area.ptr()
+    with mw.Context(R, s.E, s.K, inp.T, B) as ctx:
+        send = torch.empty(p.totals["T_nonempty"] * B, dtype=torch.uint8, device="cuda")
+        for bad, code in ((0, mw.MW_ERR_INVALID_ARG), (good[2] + 8, mw.MW_ERR_ALIGNMENT)):
+            ptrs = good.copy()
+            ptrs[2] = bad
+            ctx.mw_plan(ids, e2r, inp.T)
+            ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, p.totals["T_nonempty"])
+            ctx.mw_deliver_ptrs(mw.MW_LAYOUT_MULTIWRITE, send, torch.from_numpy(ptrs).cuda(), cap)
+            assert ctx.mw_get_totals()["status"] == code
+            got = area.host().reshape(R, cap * B)
+            assert (got[2] == SENTINEL).all()                     # the region with the bad address is left alone
+            area.body.fill_(SENTINEL)
+        ctx.mw_plan(ids, e2r, inp.T)
+        ctx.mw_deliver_ptrs(mw.MW_LAYOUT_MULTIWRITE, send, torch.from_numpy(good).cuda(), cap - 1)
+        assert ctx.mw_get_totals()["status"] == mw.MW_ERR_CAPACITY
+        assert area.guards_intact()
+        assert ctx.mw_deliver_ptrs(mw.MW_LAYOUT_MULTIWRITE, send, None, cap, check=False) == mw.MW_ERR_INVALID_ARG
+        assert ctx.mw_deliver_ptrs(7, send, torch.from_numpy(good).cuda(), cap, check=False) == mw.MW_ERR_INVALID_ARG
+
+
 # ---- AllGather ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
 @pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
