@@ -156,24 +156,34 @@ def strerror(code: int) -> str:
     return lib().mw_strerror(int(code)).decode()
 
 
-def _ptr(t) -> C.c_void_p:
-    """Device (or host) address of a torch tensor / numpy array / integer address / None."""
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array / integer address / None, as a plain integer
+    (ctypes converts it; building a c_void_p object per argument doubles the cost of a call)."""
     if t is None:
-        return C.c_void_p(0)
+        return None
     if isinstance(t, int):
-        return C.c_void_p(t)
+        return t
     if hasattr(t, "data_ptr"):
-        return C.c_void_p(t.data_ptr())
-    return C.c_void_p(t.ctypes.data)
+        return t.data_ptr()
+    return t.ctypes.data
 
 
-def _stream(stream) -> C.c_void_p:
+_raw_stream = None
+
+
+def _stream(stream):
+    """cudaStream_t of a torch stream / integer handle / None (= torch's current stream), as a plain integer."""
+    global _raw_stream
     if stream is None:
         import torch
-        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        if _raw_stream is None:
+            # the raw handle without building a Stream object (a microsecond per call); falls back to the public API
+            fast = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+            _raw_stream = fast if fast is not None else (lambda dev: torch.cuda.current_stream(dev).cuda_stream)
+        return _raw_stream(torch.cuda.current_device()) or None
     if isinstance(stream, int):
-        return C.c_void_p(stream)
-    return C.c_void_p(stream.cuda_stream)
+        return stream or None
+    return stream.cuda_stream or None
 
 
 MW_STATIC_MAX_TOKENS = 16384
