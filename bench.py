@@ -286,7 +286,7 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
         out["one_call_graph_chained"] = {"p50_us": round(percentile(us, 0.5), 2), "calls_per_graph": n_chain}
         assert ctx.mw_get_totals()["status"] == 0
     out["launches"] = launches
-    out["note"] = ("L2-resident working set (0.9 MB in, 7.3 MB out): judged on latency, not on HBM fraction; chain = "
+    out["note"] = ("L2-resident working set (0.9 MB in, 7.3 MB out): a latency figure, not an HBM fraction; chain = "
                    "mw_plan + mw_dispatch (2 launches: mw_dispatch packs and delivers in one pass), one_call = mw_plan_dispatch (1 launch); each figure includes "
                    "the host's launch cost through the Python binding, except one_call_graph (the same call replayed from a "
                    "CUDA graph, one call per graph) and one_call_graph_chained (20 calls per graph, time per call)")
