@@ -840,6 +840,7 @@ def run_cuda(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": WORKLOAD, "R": s.R, "E": s.E, "K": s.K, "T": T, "row_bytes": B, "layout": "multiwrite",
                    "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "step": ("mw_plan" if args.no_prefetch else "mw_plan_prefetch") + " + mw_pack + mw_deliver (three kernel launches)",
                    "l2": f"cycles over {nsets} buffer sets of {(2 * Tn + SD) * B / 1e6:.0f} MB each (larger than the 126 MB L2)",
                    "rows_packed": Tn, "rows_delivered": SD, "groups": tot["G"],
                    "algorithmic_bytes_per_step": alg["step"]},
