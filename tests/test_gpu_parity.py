@@ -199,6 +199,13 @@ def test_nan_and_negative_zero_payload_round_trips():
     run_dispatch(inp)
 
 
+def test_large_batch_with_many_empty_tokens():
+    """9000 tokens of 8 KB rows (a send buffer beyond half of L2), more than half of the expert slots padding: the
+    number of send rows is far below the host-side bound the launches are sized from."""
+    inp = wl.make_random_dispatch(77, T=9000, K=4, E=64, R=32, H=4096, pad_fraction=0.55)
+    run_dispatch(inp, layouts=(mw.MW_LAYOUT_MULTIWRITE,), strides=("compact", "strided"))
+
+
 # ---- planning with the hidden rows prefetched into L2 -------------------------------------------------
 @pytest.mark.parametrize("cfg", [0, 1, 2, 3])
 def test_plan_prefetch_gives_the_same_plan_and_payload(cfg):
