@@ -30,6 +30,21 @@ def test_library_builds_and_exports_every_declared_symbol():
     assert sorted(names) == sorted(mw.EXPORTS)
 
 
+def test_header_is_plain_c_and_struct_layouts_match_the_binding(tmp_path):
+    """include/mw.h must compile as C99 on its own (no C++, no CUDA or torch types), and the structs the binding
+    mirrors with ctypes must have the sizes the C compiler gives them."""
+    import subprocess
+    header = os.path.join(ROOT, "include", "mw.h")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-fsyntax-only", "-x", "c", header])
+    src = tmp_path / "sizes.c"
+    src.write_text('#include <stdio.h>\n#include "mw.h"\nint main(void) { printf("%zu %zu %zu\\n", sizeof(mw_config), '
+                   'sizeof(mw_totals), sizeof(mw_plan_view)); return 0; }\n')
+    exe = tmp_path / "sizes"
+    subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    got = [int(v) for v in subprocess.check_output([str(exe)]).split()]
+    assert got == [ctypes.sizeof(mw.mw_config), ctypes.sizeof(mw.mw_totals), ctypes.sizeof(mw.mw_plan_view)]
+
+
 def test_error_strings_and_struct_sizes():
     assert mw.strerror(mw.MW_OK) == "ok"
     for code in range(-7, 0):
