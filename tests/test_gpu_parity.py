@@ -484,6 +484,25 @@ def test_deliver_ptrs_reports_bad_addresses_and_capacity():
         assert ctx.mw_deliver_ptrs(7, send, torch.from_numpy(good).cuda(), cap, check=False) == mw.MW_ERR_INVALID_ARG
 
 
+# ---- seeded sweep over shapes -------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(30))
+def test_random_shapes(seed):
+    """Shapes drawn from a seeded generator (ranks across the bitmap-word boundaries, top-k from 1 to 12, batches across
+    the tile, small-batch and wide-variant limits, padding, repeated ids, a source inside the domain), each through one of
+    the call chains: three calls, three calls with the prefetching plan, or the single call."""
+    rng = np.random.default_rng(9000 + seed)
+    R = int(rng.choice([1, 2, 7, 16, 63, 64, 65, 100, 128, 129, 200, 256, 300]))
+    E = R * int(rng.integers(1, 4))
+    K = int(rng.integers(1, 13))
+    T = int(rng.choice([0, 1, 33, 127, 128, 129, 256, 257, 700, 1024, 1025, 1300]))
+    H = int(rng.choice([8, 24, 40, 520]))
+    inp = wl.make_random_dispatch(seed, T=T, K=K, E=E, R=R, H=H, pad_fraction=float(rng.choice([0.0, 0.1, 0.5])),
+                                  distinct=bool(rng.integers(0, 2)))
+    src = int(rng.integers(0, R)) if rng.integers(0, 3) == 0 else -1
+    chain = seed % 3
+    run_dispatch(inp, src_rank=src, max_tokens=1400, one_call=chain == 0, prefetch=chain == 1, separate=bool(seed % 2))
+
+
 # ---- AllGather ---------------------------------------------------------------------------------------
 @pytest.mark.parametrize("flags", [0, mw.MW_FLAG_COPY_BULK])
 @pytest.mark.parametrize("layout", [mw.MW_LAYOUT_MULTIWRITE, mw.MW_LAYOUT_UNICAST])
