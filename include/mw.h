@@ -439,12 +439,15 @@ MW_API int mw_relay_contexts(mw_relay *relay, mw_ctx **hop_ctx, mw_ctx **flat_ct
  *   token_group_size  device, int32 [T]: number of tokens with that bitmap, 0 if empty
  *   status            device, int32 [1]: MW_OK, or MW_ERR_BAD_INDEX if an id or table entry was
  *                     out of range (such slots are ignored)
- * Inputs as for mw_plan: topk_ids device int32 [T, K], expert_to_rank device int32 [E].
+ * Inputs as for mw_plan: topk_ids device int32 [T, K], expert_to_rank device int32 [E].  With T = 0 only
+ * `status` is written and every other pointer may be NULL.
  *
  * Limits and rules
  *   - T <= MW_STATIC_MAX_TOKENS; a larger T returns MW_ERR_CAPACITY and launches nothing.
  *   - The first call on each device looks up the device address of the array (one CUDA runtime
- *     query, no allocation); make that first call before starting any stream capture.
+ *     query, no allocation); make that first call before starting any stream capture.  The address
+ *     is remembered per device ordinal for the life of the process: it does not survive a
+ *     cudaDeviceReset of that device, after which this entry point must not be used again.
  *   - All calls on a device share the one array, which still holds the previous call's contents;
  *     every call therefore begins by emptying the table on `stream`.  Two calls whose GPU work
  *     overlaps (different streams, or different host threads without ordering) race on the array

@@ -487,8 +487,8 @@ int64_t mwo_balanced_direct_bytes(int64_t shard_bytes, int32_t n, int layout)
 }
 
 /*
- * Combine: the reverse of dispatch (Section 2.3.2: "returns computation results from experts back to
- * their original senders"; it carries no redundant data, so MultiWrite does not change it).
+ * Combine: the reverse of dispatch (Section 2.3.2: the expert outputs travel back to the ranks that sent
+ * the tokens; the step carries no redundant data, so MultiWrite does not change it).
  *
  * Reading taken: every destination rank r of token t returns one row z[r][dest_pos(t, r)] of bf16
  * values (its local experts' contribution), in the slot the dispatch delivered the token to; the source
@@ -546,6 +546,41 @@ void mwo_combine(const uint8_t *z_base, int64_t z_stride_bytes, const float *wei
                 any = 1;
             }
             out[c] = any ? double_to_bf16(acc) : 0;
+        }
+    }
+}
+
+/*
+ * The same combine with the precision of the accelerator path stated operation by operation (the paper
+ * fixes none; Section 2.3.2 only names the step): the sum is carried in IEEE binary32, starting from +0,
+ * one fused multiply-add  acc = fma(w[t, i], z, acc)  per destination in ascending rank order (the product
+ * is not rounded on its own), and the binary32 sum is rounded once to bf16 (nearest even).  fmaf() of C99
+ * is correctly rounded, so every step below is exactly defined and the result is unique bit for bit.
+ * mwo_combine (binary64 sum) stays the accuracy reference: the two differ by at most the accumulated
+ * binary32 rounding errors plus one bf16 unit in the last place.
+ */
+void mwo_combine_f32(const uint8_t *z_base, int64_t z_stride_bytes, const float *weights, int32_t T, int32_t R, int32_t K,
+                     int64_t row_bytes, const int32_t *dest_rank, const int32_t *dest_pos, const int32_t *rank_offsets,
+                     uint8_t *y)
+{
+    const int Kd = K < R ? K : R;
+    const int64_t H = row_bytes / 2;
+    for (int32_t t = 0; t < T; ++t) {
+        uint16_t *out = (uint16_t *)(y + (int64_t)t * row_bytes);
+        for (int64_t c = 0; c < H; ++c) {
+            float acc = 0.0f;
+            int any = 0;
+            for (int i = 0; i < Kd; ++i) {
+                const int32_t r = dest_rank[(int64_t)t * Kd + i];
+                if (r < 0) break;
+                const uint8_t *row = region((uint8_t *)z_base, z_stride_bytes, rank_offsets, r, row_bytes) +
+                                     (int64_t)dest_pos[(int64_t)t * Kd + i] * row_bytes;
+                const float w = weights ? weights[(int64_t)t * Kd + i] : 1.0f;
+                const float z = (float)bf16_to_double(((const uint16_t *)row)[c]);      /* exact: bf16 is a subset of binary32 */
+                acc = fmaf(w, z, acc);
+                any = 1;
+            }
+            out[c] = any ? double_to_bf16((double)acc) : 0;                             /* binary32 -> binary64 is exact: one rounding */
         }
     }
 }

@@ -40,7 +40,7 @@ def build(force: bool = False) -> str:
     stale = force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
     if stale:
         tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -208,13 +208,16 @@ def relay(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: i
     return hp, fp, send, hop_buf, recv, tot.as_dict()
 
 
-def combine(p: Plan, z: np.ndarray, weights: np.ndarray | None = None, z_stride_bytes: int = 0) -> np.ndarray:
-    """y uint16 [T, H] (bf16 bits).  z: the receive area (uint8), laid out like the dispatch's."""
+def combine(p: Plan, z: np.ndarray, weights: np.ndarray | None = None, z_stride_bytes: int = 0,
+            precision: str = "f64") -> np.ndarray:
+    """y uint16 [T, H] (bf16 bits).  z: the receive area (uint8), laid out like the dispatch's.
+    precision "f64": binary64 sum, one rounding; "f32": binary32 fused multiply-adds in rank order, one rounding."""
     zz = np.ascontiguousarray(z).view(np.uint8).reshape(-1)
     y = np.zeros((p.T, p.row_bytes // 2), np.uint16)
     w = None if weights is None else np.ascontiguousarray(weights, dtype=np.float32)
-    lib().mwo_combine.restype = None
-    lib().mwo_combine(_p(zz), C.c_int64(z_stride_bytes), _p(w) if w is not None else C.c_void_p(0), C.c_int32(p.T),
+    fn = {"f64": lib().mwo_combine, "f32": lib().mwo_combine_f32}[precision]
+    fn.restype = None
+    fn(_p(zz), C.c_int64(z_stride_bytes), _p(w) if w is not None else C.c_void_p(0), C.c_int32(p.T),
                       C.c_int32(p.R), C.c_int32(p.K), C.c_int64(p.row_bytes), _p(p.dest_rank), _p(p.dest_pos),
                       _p(p.rank_offsets), _p(y))
     return y

@@ -56,17 +56,19 @@ __global__ void __launch_bounds__(256) k_static_mask(StaticScratch *s, const int
     uint64_t *m = token_mask + (int64_t)t * W;
     int nd = 0, bad = 0;
     uint64_t h = 0x2545f4914f6cdd1dull;
+    // the token's words in token_mask are private to this thread: cleared, then one pass over the expert slots
+    // (every id and table entry is loaded once, whatever W is), then read back for the count and the hash
+    for (int w = 0; w < W; ++w) m[w] = 0;
+    for (int k = 0; k < K; ++k) {
+        const int id = my[k];
+        if (id == -1) continue;
+        if (id < 0 || id >= E) { bad = 1; continue; }
+        const int r = e2r[id];
+        if (r < 0 || r >= R) { bad = 1; continue; }
+        m[r >> 6] |= 1ull << (r & 63);
+    }
     for (int w = 0; w < W; ++w) {
-        uint64_t word = 0;
-        for (int k = 0; k < K; ++k) {
-            const int id = my[k];
-            if (id == -1) continue;
-            if (id < 0 || id >= E) { bad = 1; continue; }
-            const int r = e2r[id];
-            if (r < 0 || r >= R) { bad = 1; continue; }
-            if ((r >> 6) == w) word |= 1ull << (r & 63);
-        }
-        m[w] = word;
+        const uint64_t word = m[w];
         nd += __popcll(word);
         h = mix64(h, word);
     }
@@ -123,8 +125,8 @@ extern "C" int mw_group_tokens_static(const int32_t *topk_ids, const int32_t *ex
                                       int32_t E, int32_t R, uint64_t *token_mask, int32_t *token_ndest,
                                       int32_t *token_leader, int32_t *token_group_size, int32_t *status, void *stream)
 {
-    if (T < 0 || K < 1 || K > MW_MAX_TOPK || E < 1 || R < 1 || R > MW_MAX_RANKS || !expert_to_rank || !status ||
-        (T > 0 && (!topk_ids || !token_mask || !token_ndest || !token_leader || !token_group_size)))
+    if (T < 0 || K < 1 || K > MW_MAX_TOPK || E < 1 || R < 1 || R > MW_MAX_RANKS || !status ||
+        (T > 0 && (!topk_ids || !expert_to_rank || !token_mask || !token_ndest || !token_leader || !token_group_size)))
         return MW_ERR_INVALID_ARG;
     if (T > MW_STATIC_MAX_TOKENS) return MW_ERR_CAPACITY;   // the fixed scratch holds at most this many tokens
     StaticScratch *s = nullptr;

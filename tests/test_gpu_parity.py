@@ -509,7 +509,8 @@ def test_random_shapes(seed):
 @pytest.mark.parametrize("R,S,begin,count,strided", [
     (8, 48, 0, 8, False), (5, 4112, 1, 3, True), (64, 4096, 0, 64, False), (64, 16384, 0, 64, False),
     (64, 65536, 0, 64, True), (64, 1 << 18, 0, 64, False), (64, 1 << 20, 16, 16, False),
-    (64, 4 << 20, 60, 4, False), (64, 16 << 20, 63, 1, False), (1, 64, 0, 1, False), (3, 16, 2, 0, False)])
+    (64, 4 << 20, 60, 4, False), (64, 16 << 20, 63, 1, False), (1, 64, 0, 1, False), (3, 16, 2, 0, False),
+    (128, 4096, 0, 128, False), (65, 4112, 60, 5, True), (1024, 4096, 1000, 3, False)])   # beyond 64 ranks the bitmap costs payload bytes
 def test_allgather_parity(layout, R, S, begin, count, strided, flags):
     torch = torch_mod()
     sh = wl.make_allgather_shards(R, S, seed=4)

@@ -61,6 +61,14 @@ def test_relay_dsv3_shape_eight_servers():
     assert tot["direct_bytes"] + tot["inter_unicast_bytes"] <= tot["delivered_rows"] * inp.shape.row_bytes
 
 
+def test_relay_dsv3_shape_full_size_rows():
+    # the same routing with the full 14336-byte rows (the shape the benchmark times): 8 servers of 8 ranks
+    inp = wl.make_dispatch("dsv3_prefill")
+    assert inp.shape.row_bytes == 14336
+    tot = run_relay(inp, 8, 0)
+    assert tot["hop_rows"] < tot["delivered_rows"]
+
+
 def test_relay_small_batches_and_invalid_ids():
     inp = wl.make_random_dispatch(3, T=40, K=4, E=32, R=16, H=16, pad_fraction=0.3)
     ids = inp.topk_ids.copy()

@@ -27,6 +27,10 @@ MUTATIONS = {
                                                              "if (i == 0) slot = dest_pos[(int64_t)t * Kd + i];"),
     "expert index counts experts with a bad table entry": ("        if (r < 0 || r >= R) continue;\n        for (int32_t t = 0; t < T; ++t) {\n            int hit = 0;",
                                                            "        for (int32_t t = 0; t < T; ++t) {\n            int hit = 0;"),
+    "binary32 combine rounds the product on its own": ("acc = fmaf(w, z, acc);", "{ volatile float prod = w * z; acc = prod + acc; }"),
+    "binary32 combine walks the destinations downwards": (
+        "float acc = 0.0f;\n            int any = 0;\n            for (int i = 0; i < Kd; ++i) {\n                const int32_t r = dest_rank[(int64_t)t * Kd + i];\n                if (r < 0) break;",
+        "float acc = 0.0f;\n            int any = 0;\n            for (int i = Kd - 1; i >= 0; --i) {\n                const int32_t r = dest_rank[(int64_t)t * Kd + i];\n                if (r < 0) continue;"),
     "combine ignores the weights": ("acc += w * bf16_to_double(", "acc += bf16_to_double("),
     "combine truncates instead of rounding": ("double q = nearbyint(ldexp(a, 7 - ex));", "double q = floor(ldexp(a, 7 - ex));"),
     "combine reads the wrong slot": ("(int64_t)dest_pos[(int64_t)t * Kd + i] * row_bytes;\n                const double w",
@@ -52,6 +56,9 @@ MUTATIONS = {
     "per-expert bytes deduplicated": ("++valid_slots;", "if (!(m[r / 64] >> (r % 64) & 1)) ++valid_slots;"),
     "metadata: one word instead of W": ("(int64_t)(8 * W);", "(int64_t)(8);"),
     "self copy counted as transmitted": ("if (src_rank >= 0 && (token_mask[(int64_t)t * W + src_rank / 64] >> (src_rank % 64) & 1)) --nd;", ""),
+    "allgather metadata: one word instead of W": ("((shard_bytes + 4095) / 4096) * (8 * W);", "((shard_bytes + 4095) / 4096) * 8;"),
+    "allgather metadata: per shard, not per packet": ("(int64_t)R * ((shard_bytes + 4095) / 4096) * (8 * W);", "(int64_t)R * (8 * W);"),
+    "allgather metadata charged from the first rank on": ("totals->meta_bytes = (R <= 64 || R == 1) ? 0 :", "totals->meta_bytes = (R <= 1) ? 0 :"),
     "allgather transmits the self copy": ("if (dst_begin + d == i) continue;\n                memcpy(send_buf", "memcpy(send_buf"),
     "allgather unicast counts R copies": ("totals->unicast_bytes = (int64_t)R * (R - 1) * shard_bytes;", "totals->unicast_bytes = (int64_t)R * R * shard_bytes;"),
     "allgather shards concatenated in reverse": ("memcpy(recv_base + d * stride + (int64_t)i * shard_bytes,\n                       send_buf + (int64_t)i * shard_bytes",
@@ -73,9 +80,12 @@ def run_pins():
         pins.test_allgather_is_concatenate(layout, 5, 48, 1, 3)
         pins.test_allgather_is_concatenate(layout, 8, 64, 0, 8)
     pins.test_allgather_saved_closed_form_and_paper_example()
+    pins.test_allgather_bitmap_overhead_beyond_64_ranks()
     cpins.test_one_hot_weights_select_one_destination(False)
     cpins.test_unit_weights_sum_small_integers_exactly()
     cpins.test_rounding_is_nearest_even_with_a_single_rounding()
+    cpins.test_f32_mode_is_fused_multiply_add_in_rank_order_with_one_rounding(0, 8)
+    cpins.test_f32_mode_does_not_round_the_product_before_the_addition()
     rpins.test_paper_example_four_local_four_remote()
     rpins.test_relay_brute_force(1, 12, 3, 7, 24, 4)
     ppins.test_every_rank_gets_its_domain_in_order(0, 8, 64, 32)

@@ -400,6 +400,28 @@ def test_allgather_saved_closed_form_and_paper_example():
     assert mwo.allgather(sh, 0, 60, 8)[3] == mwo.MWO_ERR_INVALID_ARG
 
 
+def test_allgather_bitmap_overhead_beyond_64_ranks():
+    """Section 6.4: up to 64 ranks the bitmap rides in the 64-bit immediate field (no payload bytes); beyond
+    that it is carried in the payload, one bitmap of one bit per rank with every 4096-byte packet."""
+    c = load_paper_constants()
+    P = c["meta_payload_bytes"]
+    # 64 ranks: nothing; 65 ranks: two words although one bit would do (whole 64-bit words travel)
+    assert mwo.allgather(wl.make_allgather_shards(64, 64), mwo.LAYOUT_MULTIWRITE, 0, 1)[2]["meta_bytes"] == 0
+    assert mwo.allgather(wl.make_allgather_shards(65, 64), mwo.LAYOUT_MULTIWRITE, 0, 1)[2]["meta_bytes"] == 65 * 1 * 16
+    # 128 ranks, one packet per shard: 128 shards x 1 packet x 128 bits
+    sh = wl.make_allgather_shards(128, P)
+    for layout in (mwo.LAYOUT_MULTIWRITE, mwo.LAYOUT_UNICAST):
+        tot = mwo.allgather(sh, layout, 0, 1)[2]
+        assert tot["meta_bytes"] == 128 * 1 * (128 // 8)
+    # a shard one byte-vector longer than a packet needs a second bitmap
+    assert mwo.allgather(wl.make_allgather_shards(128, P + 16), mwo.LAYOUT_MULTIWRITE, 0, 1)[2]["meta_bytes"] == 128 * 2 * 16
+    # 1024 ranks: 1024 bits per 4096-byte packet = the paper's 3.13 % of the transmitted payload
+    tot = mwo.allgather(wl.make_allgather_shards(1024, P), mwo.LAYOUT_MULTIWRITE, 0, 1)[2]
+    assert tot["meta_bytes"] * 8 == 1024 * c["meta_bits_1024_ranks"]
+    assert 100 * tot["meta_bytes"] / tot["mw_bytes"] == 3.125
+    assert math.floor(100 * 3.125 + 0.5) / 100 == c["meta_overhead_percent_1024_ranks"]
+
+
 def test_large_shard_generator_marks_every_page():
     sh = wl.make_allgather_shards(3, 4 << 20)
     pages = sh.view(np.uint64).reshape(3, -1, 512)[:, :, 0]
