@@ -64,24 +64,22 @@ extern "C" {
 #define MW_ERR_CAPACITY     (-3)  /* a buffer cannot hold the rows the plan assigns to it     */
 #define MW_ERR_CUDA         (-4)  /* a CUDA runtime call failed                               */
 #define MW_ERR_BAD_INDEX    (-5)  /* expert id or expert->rank entry out of range (ignored)   */
-#define MW_ERR_TIMEOUT      (-6)  /* a bounded device-side wait gave up; the plan is invalid; */
-                                  /* destroy the context (its counters may be out of step)    */
+#define MW_ERR_TIMEOUT      (-6)  /* a bounded device-side wait gave up; the plan is invalid  */
+                                  /* and the context refuses further work until mw_reset      */
 #define MW_ERR_NO_PLAN      (-7)  /* dispatch called before any plan                          */
 
 #define MW_LAYOUT_MULTIWRITE 0    /* send buffer holds each row once (one row per group member) */
 #define MW_LAYOUT_UNICAST    1    /* send buffer holds one copy per destination                */
 
 #define MW_FLAG_HOST_STAGING   0x1u  /* allocate device staging so mw_dispatch_host can be used */
-#define MW_FLAG_PLAN_MULTIPASS 0x2u  /* always take the tiled multi-kernel plan, even for small T */
-#define MW_FLAG_COPY_LDST      0x4u  /* row copies by a persistent grid of warps with 16-byte register loads/stores */
-#define MW_FLAG_PLAN_COOPERATIVE 0x8u /* launch the fused plan through the cooperative-launch API (the   */
-                                      /* driver then guarantees that all its blocks are resident; costs   */
-                                      /* about 20 us of host time per plan); default is an ordinary launch */
+#define MW_FLAG_PLAN_MULTIPASS 0x2u  /* always take the tiled multi-kernel plan, even for small T (its tiles take   */
+                                     /* tickets, so it does not need all its blocks resident at once)               */
 #define MW_FLAG_NO_OVERLAP     0x10u /* do not let a kernel's start-up overlap the previous kernel's tail */
-#define MW_FLAG_COPY_REG_STORE 0x20u /* persistent grid, bulk loads into shared memory, 16-byte register stores */
 #define MW_FLAG_COPY_BULK      0x40u /* persistent grid, bulk (TMA) loads into shared memory and bulk stores out of it; */
-                                     /* without any MW_FLAG_COPY_* bit row copies run one block per (row, piece) with   */
-                                     /* plain 16-byte loads and stores, which measured fastest on B200                  */
+                                     /* without it row copies run one block per (row, piece) with plain 16-byte loads   */
+                                     /* and stores, which measured fastest on B200                                      */
+#define MW_FLAG_SHORT_WAITS    0x80u /* device-side waits give up after about a millisecond instead of about a second   */
+                                     /* (for latency-critical hosts that prefer an early MW_ERR_TIMEOUT, and for tests) */
 
 #define MW_MAX_RANKS   1024
 #define MW_MAX_TOPK    64
@@ -149,6 +147,18 @@ MW_API int mw_create(mw_ctx **out, const mw_config *cfg);
 MW_API int mw_destroy(mw_ctx *ctx);
 
 /*
+ * Makes a context usable again after MW_ERR_TIMEOUT.  The device-side waits of this library (a plan tile waiting
+ * for the counts of the tiles before it, a plan block waiting at a grid barrier, a copy pipeline waiting for a
+ * bulk load) are bounded; when one gives up, mw_totals.status says MW_ERR_TIMEOUT, the kernels that follow skip
+ * their work, and from the mw_get_totals that reported it every call on the context except mw_get_totals,
+ * mw_reset and mw_destroy returns MW_ERR_TIMEOUT.  (A plan can run into this when other work keeps the GPU's SMs
+ * occupied for about a second, so that its blocks cannot all become resident.)  mw_reset waits for the device,
+ * empties the scratch the plans share and rewinds the host-side counters; no plan exists afterwards (the next
+ * call must be a plan).  Nothing is reallocated.  Synchronous.
+ */
+MW_API int mw_reset(mw_ctx *ctx);
+
+/*
  * Source-side planning (Section 4.1 step 1: the source turns the destination information
  * into bitmap metadata; Section 5.1, cs_send: task decomposition).  From the router output
  * it builds bitmaps, groups, per-group and per-rank counts with exclusive prefix sums, every
@@ -171,6 +181,33 @@ MW_API int mw_plan(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
  */
 MW_API int mw_plan_prefetch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
                      const void *x, mw_plan_view *view, void *stream);
+
+/*
+ * Planning one batch ahead.  A plan is a short chain of dependent steps on a few SMs and moves almost no data, while
+ * pack and deliver are bound by memory bandwidth; the source-side preparation of the next write can therefore run
+ * while the replication of the current one is in flight (Section 5.1: cs_send prepares work requests while the
+ * relay thread copies and forwards).  The context holds two plan slots:
+ *
+ *   mw_plan_next   plans a batch into the slot the data path is NOT using, on a stream the library owns.  The plan
+ *                  starts once everything submitted to `stream` so far has completed (its inputs are ready, and the
+ *                  copy kernels that read that slot two batches ago are done) and then runs concurrently with whatever
+ *                  is submitted to `stream` afterwards.  x (optional, may be NULL) as in mw_plan_prefetch.
+ *   mw_plan_swap   makes that plan the current one: `stream` waits for it (no host synchronisation) and every call
+ *                  that "uses the latest plan" now uses it; `view` (optional) receives its arrays.  MW_ERR_NO_PLAN when
+ *                  no mw_plan_next is outstanding.  Views and plan arrays of the slot swapped out stay valid until the
+ *                  next mw_plan_next overwrites them.
+ *
+ * Steady state, batch i (one stream, one context):
+ *     mw_plan_swap(ctx, &view, s);                          the plan of batch i, issued one iteration ago
+ *     mw_plan_next(ctx, ids[i+1], e2r, T[i+1], x[i+1], s);  before the copies of batch i are submitted
+ *     mw_pack(ctx, x[i], ...s);  mw_deliver(ctx, ...s);     run while batch i+1 is being planned
+ * The inputs of a pending mw_plan_next must not be overwritten before the matching mw_plan_swap's stream work.
+ * mw_plan, mw_plan_prefetch and mw_plan_dispatch plan into the current slot and may be mixed with the pair above
+ * (plans are ordered among themselves by the library); an outstanding mw_plan_next stays outstanding.
+ */
+MW_API int mw_plan_next(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x,
+                        void *stream);
+MW_API int mw_plan_swap(mw_ctx *ctx, mw_plan_view *view, void *stream);
 
 /* Fills `view` with the workspace pointers of the context and the T of its latest plan (no device work). */
 MW_API int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view);
@@ -223,7 +260,7 @@ MW_API int mw_deliver_ptrs(mw_ctx *ctx, int layout, const void *send_buf, void *
 /*
  * The whole data movement of one dispatch, with the results of mw_pack followed by mw_deliver (same send buffer,
  * same receive regions, bit for bit) but in one pass: every hidden row is read once and written to its send
- * slot(s) and to all its receive slots.  With a MW_FLAG_COPY_* bit set it is the two calls in sequence.
+ * slot(s) and to all its receive slots.  With MW_FLAG_COPY_BULK it is the two calls in sequence.
  */
 MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows,
                 void *recv_base, int64_t recv_stride_bytes, int64_t recv_capacity_rows, void *stream);
@@ -235,7 +272,7 @@ MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, i
  * replication overhead to outweigh the savings, up to its batch of 1k) the three kernels are
  * replaced by a single launch in which every block recomputes the plan in shared memory and then
  * moves its share of the rows (256 threads per block up to 128 tokens, 1024 beyond); larger
- * batches, the unicast layout and contexts created with a plan or copy variant flag take the
+ * batches, the unicast layout and contexts created with MW_FLAG_PLAN_MULTIPASS take the
  * ordinary three-kernel route (planning through mw_plan_prefetch).
  * The single launch keeps no state on the host, so a call captured into a CUDA graph may be replayed
  * (new ids and rows in the same buffers).  mw_plan and mw_plan_prefetch may not: the look-back epoch
@@ -353,6 +390,15 @@ MW_API int mw_paired_allgather(mw_ctx *ctx, const void *shards, int64_t shard_by
  * bandwidths): shard_bytes * c / (1 + c) with c copies on the pair link, rounded down to a multiple of 16. */
 MW_API int64_t mw_pair_balanced_direct_bytes(int64_t shard_bytes, int32_t ranks_per_domain, int layout);
 
+/* The same split for links of two bandwidth classes (Section 5.2 step 1: the shard is cut by the measured bandwidth
+ * ratio): links inside a domain run at w_direct, links between the domains at w_pair (same unit, both > 0).  A direct
+ * link carries d bytes and the pair link c copies of the rest, so both finish together at
+ * d = shard_bytes * c * w_direct / (w_pair + c * w_direct), evaluated in double precision and rounded down to a
+ * multiple of 16.  Equal bandwidths give mw_pair_balanced_direct_bytes; a non-positive bandwidth or a single-rank
+ * domain returns shard_bytes (everything direct).  Host arithmetic only. */
+MW_API int64_t mw_pair_split_direct_bytes(int64_t shard_bytes, int32_t ranks_per_domain, int layout, double w_direct,
+                                          double w_pair);
+
 /*
  * One whole dispatch from host memory (plan, pack, deliver) for callers whose data lives on
  * the host: copies topk_ids, expert_to_rank and x to the device, runs mw_plan and mw_dispatch
@@ -464,6 +510,21 @@ MW_API int mw_group_tokens_static(const int32_t *topk_ids, const int32_t *expert
  * pointer of the plan view (or any device memory of the context's device) into host memory.
  */
 MW_API int mw_read_device(mw_ctx *ctx, void *host_dst, const void *device_src, int64_t bytes, void *stream);
+
+/*
+ * Test hook for the give-up paths of the bounded device-side waits (nothing faults, traps or hangs: a wait simply
+ * runs out).  The bits apply to the next launch that contains the wait and are cleared by it:
+ *   MW_TEST_SKEW_LOOKBACK   the next plan's tiles look for predecessor records of an epoch nobody writes
+ *   MW_TEST_SKEW_BARRIER    the next fused plan's grid barriers wait for one arrival more than there are blocks
+ *   MW_TEST_SKEW_BULK_LOAD  the next launch of the bulk-copy engine announces every load 16 bytes too large, so
+ *                           no pipeline stage ever completes
+ * Use with MW_FLAG_SHORT_WAITS, or each wait takes about a second to give up.  The outcome is MW_ERR_TIMEOUT in
+ * mw_totals.status; recover with mw_reset.
+ */
+#define MW_TEST_SKEW_LOOKBACK  0x1u
+#define MW_TEST_SKEW_BARRIER   0x2u
+#define MW_TEST_SKEW_BULK_LOAD 0x4u
+MW_API int mw_test_skew_waits(mw_ctx *ctx, uint32_t what);
 
 /* Number of kernels this context has launched since mw_create (for launch accounting). */
 MW_API int64_t mw_kernel_launches(const mw_ctx *ctx);

@@ -38,6 +38,7 @@
  * occurrence, ascending token order) are this implementation's reading, not the
  * paper's: parity for those choices is pinned only to the independent brute force.
  */
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -487,6 +488,27 @@ int64_t mwo_balanced_direct_bytes(int64_t shard_bytes, int32_t n, int layout)
 }
 
 /*
+ * The split for links of two bandwidth classes (Section 5.2 step 1: the shard is cut in two by the measured
+ * bandwidth ratio of the links; Section 3.1 for the traffic each link carries).  Links inside a domain run at
+ * w_direct, links between the domains (the pair link and the relay's forwarding links) at w_pair, in the same
+ * unit.  With d direct bytes a direct link is busy for d / w_direct and the pair link, which carries c copies of
+ * the rest (c = 1 for MultiWrite, n - 1 for the unicast relay), for c (s - d) / w_pair; the forwarding links carry
+ * one copy each and are never slower than the pair link.  Both finish together at
+ *     d = s c w_direct / (w_pair + c w_direct),
+ * taken in double precision and rounded down to a multiple of 16 bytes.  Equal bandwidths give the split of
+ * mwo_balanced_direct_bytes.  Non-positive bandwidths or n <= 1: everything goes direct.
+ */
+int64_t mwo_split_direct_bytes(int64_t shard_bytes, int32_t n, int layout, double w_direct, double w_pair)
+{
+    if (n <= 1 || !(w_direct > 0.0) || !(w_pair > 0.0)) return shard_bytes;
+    const double c = layout == 0 ? 1.0 : (double)(n - 1);
+    const double d = floor((double)shard_bytes * c * w_direct / (w_pair + c * w_direct));
+    int64_t bytes = (int64_t)d / 16 * 16;
+    if (bytes > shard_bytes) bytes = shard_bytes / 16 * 16;
+    return bytes;
+}
+
+/*
  * Combine: the reverse of dispatch (Section 2.3.2: the expert outputs travel back to the ranks that sent
  * the tokens; the step carries no redundant data, so MultiWrite does not change it).
  *
@@ -496,8 +518,6 @@ int64_t mwo_balanced_direct_bytes(int64_t shard_bytes, int32_t n, int layout)
  * with the sum carried in double precision here and rounded once to bf16 (round to nearest even).
  * weights == NULL means all ones.  A token without destinations gets a row of zeros.
  */
-#include <math.h>
-
 static double bf16_to_double(uint16_t b)
 {
     uint32_t u = (uint32_t)b << 16;

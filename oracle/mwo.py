@@ -277,6 +277,12 @@ def balanced_direct_bytes(shard_bytes: int, n: int, layout: int) -> int:
     return int(lib().mwo_balanced_direct_bytes(C.c_int64(shard_bytes), C.c_int32(n), C.c_int(layout)))
 
 
+def split_direct_bytes(shard_bytes: int, n: int, layout: int, w_direct: float, w_pair: float) -> int:
+    lib().mwo_split_direct_bytes.restype = C.c_int64
+    return int(lib().mwo_split_direct_bytes(C.c_int64(shard_bytes), C.c_int32(n), C.c_int(layout), C.c_double(w_direct),
+                                            C.c_double(w_pair)))
+
+
 def paired_allgather(shards: np.ndarray, direct_bytes: int, layout: int, fill: int = 0):
     """Returns (relay_buf, recv, totals, ret).  shards: uint8 [R, S], R = 2n."""
     sh = np.ascontiguousarray(shards).view(np.uint8)

@@ -25,18 +25,21 @@ MW_LAYOUT_UNICAST = 1
 
 MW_FLAG_HOST_STAGING = 0x1
 MW_FLAG_PLAN_MULTIPASS = 0x2
-MW_FLAG_COPY_LDST = 0x4
-MW_FLAG_PLAN_COOPERATIVE = 0x8
 MW_FLAG_NO_OVERLAP = 0x10
-MW_FLAG_COPY_REG_STORE = 0x20
 MW_FLAG_COPY_BULK = 0x40
+MW_FLAG_SHORT_WAITS = 0x80
+
+MW_TEST_SKEW_LOOKBACK = 0x1
+MW_TEST_SKEW_BARRIER = 0x2
+MW_TEST_SKEW_BULK_LOAD = 0x4
 
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
-EXPORTS = ("mw_create", "mw_destroy", "mw_plan", "mw_plan_prefetch", "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_deliver_ptrs", "mw_dispatch", "mw_plan_dispatch",
-           "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_group_major", "mw_deliver_group_major", "mw_expert_index",
-           "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_kernel_launches",
-           "mw_strerror", "mw_pair_balanced_direct_bytes") + RELAY_EXPORTS
+INT_EXPORTS = ("mw_create", "mw_destroy", "mw_reset", "mw_plan", "mw_plan_prefetch", "mw_plan_next", "mw_plan_swap",
+               "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_deliver_ptrs", "mw_dispatch", "mw_plan_dispatch",
+               "mw_allgather_pack", "mw_paired_allgather", "mw_combine", "mw_group_major", "mw_deliver_group_major",
+               "mw_expert_index", "mw_dispatch_host", "mw_group_tokens_static", "mw_read_device", "mw_test_skew_waits") + RELAY_EXPORTS
+EXPORTS = INT_EXPORTS + ("mw_kernel_launches", "mw_strerror", "mw_pair_balanced_direct_bytes", "mw_pair_split_direct_bytes")
 
 
 class mw_config(C.Structure):
@@ -110,6 +113,10 @@ def lib():
         vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
         L.mw_create.argtypes = [C.POINTER(vp), C.POINTER(mw_config)]
         L.mw_destroy.argtypes = [vp]
+        L.mw_reset.argtypes = [vp]
+        L.mw_test_skew_waits.argtypes = [vp, C.c_uint32]
+        L.mw_plan_next.argtypes = [vp, vp, vp, i32, vp, vp]
+        L.mw_plan_swap.argtypes = [vp, C.POINTER(mw_plan_view), vp]
         L.mw_plan.argtypes = [vp, vp, vp, i32, C.POINTER(mw_plan_view), vp]
         L.mw_plan_prefetch.argtypes = [vp, vp, vp, i32, vp, C.POINTER(mw_plan_view), vp]
         L.mw_get_plan_view.argtypes = [vp, C.POINTER(mw_plan_view)]
@@ -123,6 +130,8 @@ def lib():
         L.mw_paired_allgather.argtypes = [vp, vp, i64, i64, C.c_int, vp, vp, C.POINTER(mw_pair_totals), vp]
         L.mw_pair_balanced_direct_bytes.argtypes = [i64, i32, C.c_int]
         L.mw_pair_balanced_direct_bytes.restype = i64
+        L.mw_pair_split_direct_bytes.argtypes = [i64, i32, C.c_int, C.c_double, C.c_double]
+        L.mw_pair_split_direct_bytes.restype = i64
         L.mw_combine.argtypes = [vp, vp, i64, vp, vp, vp]
         L.mw_group_major.argtypes = [vp, C.POINTER(mw_group_major_view), vp]
         L.mw_deliver_group_major.argtypes = [vp, vp, vp, i64, i64, vp]
@@ -138,11 +147,9 @@ def lib():
         L.mw_relay_get_totals.argtypes = [vp, C.POINTER(mw_relay_totals), vp]
         L.mw_relay_dispatch.argtypes = [vp, vp, vp, i64, vp, i64, vp, i64, i64, vp]
         L.mw_relay_contexts.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
-        for name in RELAY_EXPORTS:
-            getattr(L, name).restype = C.c_int
         L.mw_strerror.argtypes = [C.c_int]
         L.mw_strerror.restype = C.c_char_p
-        for name in EXPORTS[:20]:
+        for name in INT_EXPORTS:
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -150,6 +157,10 @@ def lib():
 
 def mw_pair_balanced_direct_bytes(shard_bytes: int, ranks_per_domain: int, layout: int) -> int:
     return int(lib().mw_pair_balanced_direct_bytes(shard_bytes, ranks_per_domain, layout))
+
+
+def mw_pair_split_direct_bytes(shard_bytes: int, ranks_per_domain: int, layout: int, w_direct: float, w_pair: float) -> int:
+    return int(lib().mw_pair_split_direct_bytes(shard_bytes, ranks_per_domain, layout, w_direct, w_pair))
 
 
 def strerror(code: int) -> str:
@@ -264,6 +275,34 @@ class Context:
         if check and rc != MW_OK:
             raise MwError(rc, "mw_plan_prefetch")
         self.view = view
+        return rc
+
+    def mw_plan_next(self, topk_ids, expert_to_rank, T: int | None = None, x=None, stream=None, check: bool = True) -> int:
+        T = int(topk_ids.shape[0]) if T is None else T
+        rc = lib().mw_plan_next(self._h, _ptr(topk_ids), _ptr(expert_to_rank), T, _ptr(x), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_plan_next")
+        return rc
+
+    def mw_plan_swap(self, stream=None, check: bool = True) -> int:
+        view = mw_plan_view()
+        rc = lib().mw_plan_swap(self._h, C.byref(view), _stream(stream))
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_plan_swap")
+        if rc == MW_OK:
+            self.view = view
+        return rc
+
+    def mw_reset(self, check: bool = True) -> int:
+        rc = lib().mw_reset(self._h)
+        if check and rc != MW_OK:
+            raise MwError(rc, "mw_reset")
+        return rc
+
+    def mw_test_skew_waits(self, what: int) -> int:
+        rc = lib().mw_test_skew_waits(self._h, what)
+        if rc != MW_OK:
+            raise MwError(rc, "mw_test_skew_waits")
         return rc
 
     def mw_get_totals(self, stream=None) -> dict:

@@ -1,5 +1,6 @@
 // C ABI entry points (declared and documented in include/mw.h): argument checks, workspace
 // carving, and the launch sequences.  No step of the path runs on the host.
+#include <math.h>
 #include <new>
 #include <stdlib.h>
 #include <string.h>
@@ -22,12 +23,10 @@ struct Carver {
     }
 };
 
-// Lays the workspace out inside one slab; with base == nullptr it only measures.
-size_t carve(mw_ctx *c, uint8_t *base)
+// The arrays of one plan slot: what a plan writes for the data path to read (and its own per-token values).
+void carve_slot(mw_ctx *c, Carver &k, mw_dev &d)
 {
-    Carver k{base, 0};
     const size_t Tm = (size_t)c->cfg.max_tokens, W = (size_t)c->W, Kd = (size_t)c->Kd, R = (size_t)c->cfg.R;
-    mw_dev &d = c->d;
     d.token_mask = k.take<uint64_t>(Tm * W);
     d.token_ndest = k.take<int32_t>(Tm);
     d.token_group = k.take<int32_t>(Tm);
@@ -49,6 +48,18 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.row_dest_rank = k.take<int32_t>(Tm * Kd);
     d.row_dest_pos = k.take<int32_t>(Tm * Kd);
     d.row_dest_flat = k.take<int32_t>(Tm * Kd);
+}
+
+// Lays the workspace out inside one slab; with base == nullptr it only measures.  Two plan slots, then the arrays
+// derived from the current plan on the caller's stream, then the scratch all plans share (plans are ordered
+// among themselves, so one copy is enough); mw_reset re-initialises the scratch part only.
+size_t carve(mw_ctx *c, uint8_t *base)
+{
+    Carver k{base, 0};
+    const size_t Tm = (size_t)c->cfg.max_tokens, Kd = (size_t)c->Kd, R = (size_t)c->cfg.R;
+    mw_dev &d = c->d;
+    carve_slot(c, k, d);
+    carve_slot(c, k, c->other.d);
     d.gm_rank = k.take<int32_t>(Tm * Kd);
     d.gm_offset = k.take<int32_t>(Tm * Kd);
     d.dest_pos_gm = k.take<int32_t>(Tm * Kd);
@@ -59,6 +70,8 @@ size_t carve(mw_ctx *c, uint8_t *base)
         const size_t n = (size_t)c->max_tiles * (size_t)c->cfg.E;     // beyond 256 MB the expert index is not offered
         d.ex_tile_cnt = n * sizeof(int32_t) <= ((size_t)256 << 20) ? k.take<int32_t>(n) : nullptr;
     }
+    c->scratch_begin = base ? base + k.used : nullptr;
+    const size_t scratch_from = k.used;
     d.slot_key = k.take<unsigned long long>((size_t)c->HS);
     d.slot_leader = k.take<int32_t>((size_t)c->HS);
     d.slot_count = k.take<int32_t>((size_t)c->HS);
@@ -68,6 +81,17 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.gbar = k.take<unsigned int>(1);
     d.copy_ctr = k.take<unsigned int>(2);
     d.acc = k.take<mw_acc>(2);
+    d.gave_up = k.take<unsigned int>(1);
+    c->scratch_bytes = k.used - scratch_from;
+    {   // the second slot shares everything that is not a plan array
+        mw_dev &o = c->other.d;
+        o.gm_rank = d.gm_rank; o.gm_offset = d.gm_offset; o.dest_pos_gm = d.dest_pos_gm;
+        o.row_dest_pos_gm = d.row_dest_pos_gm; o.row_dest_flat_gm = d.row_dest_flat_gm;
+        o.gm_tile_sum = d.gm_tile_sum; o.ex_tile_cnt = d.ex_tile_cnt;
+        o.slot_key = d.slot_key; o.slot_leader = d.slot_leader; o.slot_count = d.slot_count;
+        o.tile_state = d.tile_state; o.tile_agg = d.tile_agg; o.ticket = d.ticket; o.gbar = d.gbar;
+        o.copy_ctr = d.copy_ctr; o.acc = d.acc; o.gave_up = d.gave_up;
+    }
     if (c->cfg.flags & MW_FLAG_HOST_STAGING) {
         const size_t B = (size_t)c->cfg.row_bytes;
         c->st_ids = k.take<int32_t>(Tm * (size_t)c->cfg.K);
@@ -103,6 +127,62 @@ mw_copy_args base_args(mw_ctx *ctx)
     return a;
 }
 
+void fill_view(const mw_ctx *ctx, int32_t T, mw_plan_view *view)
+{
+    const mw_dev &d = ctx->d;
+    view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
+    view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
+    view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
+    view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
+    view->T = T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
+}
+
+// Exchanges the current plan slot with the other one (host-side bookkeeping only).
+void swap_slots(mw_ctx *ctx)
+{
+    const mw_slot cur = {ctx->d, ctx->planned_T, ctx->prefetched, ctx->plan_epoch};
+    ctx->d = ctx->other.d; ctx->planned_T = ctx->other.planned_T; ctx->prefetched = ctx->other.prefetched;
+    ctx->plan_epoch = ctx->other.plan_epoch;
+    ctx->other = cur;
+}
+
+// Brings the scratch that all plans share (bitmap table, look-back records, counters, accumulators) and the
+// host-side running counts back to their initial state.  The device must be idle as far as this context goes.
+int init_scratch(mw_ctx *c)
+{
+    if (cudaMemset(c->scratch_begin, 0, c->scratch_bytes) != cudaSuccess) return MW_ERR_CUDA;
+    k_fill_i32<<<64, 256>>>((int32_t *)c->d.slot_key, 2 * (int64_t)c->HS, -1);   // all ones = empty slot
+    k_fill_i32<<<64, 256>>>(c->d.slot_leader, c->HS, 0x7fffffff);                 // no leader
+    if (cudaDeviceSynchronize() != cudaSuccess) return MW_ERR_CUDA;
+    c->epoch = 0; c->tickets_used = 0; c->gbar_arrivals = 0;
+    c->planned_T = -1; c->prefetched = nullptr; c->plan_epoch = 0;
+    c->other.planned_T = -1; c->other.prefetched = nullptr; c->other.plan_epoch = 0;
+    c->next_pending = 0; c->plans_on_side_stream = 0; c->gm_epoch = 0;
+    c->test_skew = 0; c->poisoned = 0;
+    return MW_OK;
+}
+
+void release(mw_ctx *c)
+{
+    if (c->ev_submitted) cudaEventDestroy(c->ev_submitted);
+    if (c->ev_planned) cudaEventDestroy(c->ev_planned);
+    if (c->plan_stream) cudaStreamDestroy(c->plan_stream);
+    if (c->slab) cudaFree(c->slab);
+    cudaGetLastError();
+    delete c;
+}
+
+// A plan launch touches the shared scratch, so it must not overtake the previous plan.  Plans issued through
+// mw_plan_next run on the library's own stream; the first plan launched on another stream afterwards waits for them.
+int order_after_side_plans(mw_ctx *ctx, cudaStream_t st)
+{
+    if (ctx->plans_on_side_stream && st != ctx->plan_stream) {
+        if (cudaStreamWaitEvent(st, ctx->ev_planned, 0) != cudaSuccess) return MW_ERR_CUDA;
+        ctx->plans_on_side_stream = 0;
+    }
+    return MW_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -132,28 +212,34 @@ int mw_create(mw_ctx **out, const mw_config *cfg)
     int hs = 1024;                                    // load factor <= 1/8 keeps probe chains short
     while (hs < 8 * cfg->max_tokens) hs <<= 1;
     c->HS = hs;
-    c->planned_T = -1;
+    c->spin_limit = (cfg->flags & MW_FLAG_SHORT_WAITS) ? (1 << 10) : (1 << 20);       // about a millisecond / a second
+    c->bar_spin_limit = (cfg->flags & MW_FLAG_SHORT_WAITS) ? (1 << 11) : (1 << 21);
+    c->copy_wait_limit = (cfg->flags & MW_FLAG_SHORT_WAITS) ? (1 << 10) : (1 << 20);
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
     cudaDeviceGetAttribute(&c->l2_bytes, cudaDevAttrL2CacheSize, cfg->device);
-    cudaDeviceGetAttribute(&c->coop_ok, cudaDevAttrCooperativeLaunch, cfg->device);
 
     const size_t bytes = carve(c, nullptr);
     if (cudaMalloc(&c->slab, bytes) != cudaSuccess) { cudaGetLastError(); delete c; return MW_ERR_CUDA; }
     carve(c, (uint8_t *)c->slab);
     int rc = MW_OK;
     if (cudaMemset(c->slab, 0, bytes) != cudaSuccess) rc = MW_ERR_CUDA;
-    // empty table: no representative, no leader
+    if (rc == MW_OK) rc = init_scratch(c);
     if (rc == MW_OK) {
-        k_fill_i32<<<64, 256>>>((int32_t *)c->d.slot_key, 2 * (int64_t)c->HS, -1);   // all ones = empty slot
-        k_fill_i32<<<64, 256>>>(c->d.slot_leader, c->HS, 0x7fffffff);
-        if (cudaDeviceSynchronize() != cudaSuccess) rc = MW_ERR_CUDA;
+        // planning stream of mw_plan_next: its few blocks should be placed as soon as an SM has room, ahead of the
+        // copy kernels' backlog, hence the highest priority
+        int lo = 0, hi = 0;
+        if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
+            cudaStreamCreateWithPriority(&c->plan_stream, cudaStreamNonBlocking, hi) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_submitted, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_planned, cudaEventDisableTiming) != cudaSuccess)
+            rc = MW_ERR_CUDA;
     }
     if (rc == MW_OK) rc = mw_plan_smem_setup(c);
     if (rc == MW_OK) rc = mw_copy_smem_setup(c);
     if (rc == MW_OK) rc = mw_small_setup(c);
     if (rc == MW_OK) rc = mw_order_smem_setup(c);
-    if (rc != MW_OK) { cudaFree(c->slab); cudaGetLastError(); delete c; return rc; }
+    if (rc != MW_OK) { release(c); return rc; }
     *out = c;
     return MW_OK;
 }
@@ -162,10 +248,23 @@ int mw_destroy(mw_ctx *ctx)
 {
     if (!ctx) return MW_OK;
     cudaSetDevice(ctx->cfg.device);
-    cudaDeviceSynchronize();
-    const cudaError_t e = cudaFree(ctx->slab);
-    delete ctx;
+    const cudaError_t e = cudaDeviceSynchronize();
+    release(ctx);
     return e == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}
+
+int mw_reset(mw_ctx *ctx)
+{
+    if (!ctx) return MW_ERR_INVALID_ARG;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return MW_ERR_CUDA;
+    return init_scratch(ctx);
+}
+
+int mw_test_skew_waits(mw_ctx *ctx, uint32_t what)
+{
+    if (!ctx || (what & ~(MW_TEST_SKEW_LOOKBACK | MW_TEST_SKEW_BARRIER | MW_TEST_SKEW_BULK_LOAD))) return MW_ERR_INVALID_ARG;
+    ctx->test_skew = what;
+    return MW_OK;
 }
 
 namespace {
@@ -173,15 +272,11 @@ int plan_with_rows(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
                    mw_plan_view *view, void *stream)
 {
     if (!ctx || !expert_to_rank || T < 0 || T > ctx->cfg.max_tokens || (T > 0 && !topk_ids)) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (rows && !aligned16(rows)) return MW_ERR_ALIGNMENT;
-    if (view) {
-        const mw_dev &d = ctx->d;
-        view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
-        view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
-        view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
-        view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
-        view->T = T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
-    }
+    if (view) fill_view(ctx, T, view);
+    const int rc = order_after_side_plans(ctx, as_stream(stream));
+    if (rc != MW_OK) return rc;
     return mw_plan_launch(ctx, topk_ids, expert_to_rank, T, rows, as_stream(stream));
 }
 }  // namespace
@@ -198,16 +293,43 @@ int mw_plan_prefetch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert
     return plan_with_rows(ctx, topk_ids, expert_to_rank, T, x, view, stream);
 }
 
+int mw_plan_next(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *x, void *stream)
+{
+    if (!ctx || !expert_to_rank || T < 0 || T > ctx->cfg.max_tokens || (T > 0 && !topk_ids)) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
+    if (x && !aligned16(x)) return MW_ERR_ALIGNMENT;
+    // everything the caller has submitted so far comes first: the inputs of this plan, and the copy kernels that
+    // still read the slot about to be overwritten (it held the batch before the current one)
+    if (cudaEventRecord(ctx->ev_submitted, as_stream(stream)) != cudaSuccess ||
+        cudaStreamWaitEvent(ctx->plan_stream, ctx->ev_submitted, 0) != cudaSuccess)
+        return MW_ERR_CUDA;
+    swap_slots(ctx);                                   // plan into the slot the data path is not using
+    const int rc = mw_plan_launch(ctx, topk_ids, expert_to_rank, T, x, ctx->plan_stream);
+    swap_slots(ctx);
+    if (rc != MW_OK) return rc;
+    if (cudaEventRecord(ctx->ev_planned, ctx->plan_stream) != cudaSuccess) return MW_ERR_CUDA;
+    ctx->plans_on_side_stream = 1;
+    ctx->next_pending = 1;
+    return MW_OK;
+}
+
+int mw_plan_swap(mw_ctx *ctx, mw_plan_view *view, void *stream)
+{
+    if (!ctx) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
+    if (!ctx->next_pending) return MW_ERR_NO_PLAN;
+    if (cudaStreamWaitEvent(as_stream(stream), ctx->ev_planned, 0) != cudaSuccess) return MW_ERR_CUDA;
+    swap_slots(ctx);
+    ctx->next_pending = 0;
+    if (view) fill_view(ctx, ctx->planned_T, view);
+    return MW_OK;
+}
+
 int mw_get_plan_view(mw_ctx *ctx, mw_plan_view *view)
 {
     if (!ctx || !view) return MW_ERR_INVALID_ARG;
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
-    const mw_dev &d = ctx->d;
-    view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
-    view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
-    view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
-    view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
-    view->T = ctx->planned_T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
+    fill_view(ctx, ctx->planned_T, view);
     return MW_OK;
 }
 
@@ -217,12 +339,17 @@ int mw_get_totals(mw_ctx *ctx, mw_totals *host_out, void *stream)
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (cudaMemcpyAsync(host_out, ctx->d.totals, sizeof(mw_totals), cudaMemcpyDeviceToHost, as_stream(stream)) != cudaSuccess)
         return MW_ERR_CUDA;
-    return cudaStreamSynchronize(as_stream(stream)) == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return MW_ERR_CUDA;
+    // a wait that gave up leaves the shared scratch and the host's running counts out of step: no further
+    // device work on this context until mw_reset
+    if (host_out->status == MW_ERR_TIMEOUT) ctx->poisoned = 1;
+    return MW_OK;
 }
 
 int mw_pack(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t send_capacity_rows, void *stream)
 {
     if (!ctx || !x || !send_buf || send_capacity_rows < 0 || check_layout(layout)) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (!aligned16(x) || !aligned16(send_buf)) return MW_ERR_ALIGNMENT;
     mw_copy_args a = base_args(ctx);
@@ -254,6 +381,7 @@ int mw_deliver(mw_ctx *ctx, int layout, const void *send_buf, void *recv_base, i
 {
     if (!ctx || !send_buf || !recv_base || recv_stride_bytes < 0 || recv_capacity_rows < 0 || check_layout(layout))
         return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (!aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
     if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
@@ -282,6 +410,7 @@ int mw_deliver_ptrs(mw_ctx *ctx, int layout, const void *send_buf, void *const *
                     void *stream)
 {
     if (!ctx || !send_buf || !recv_ptrs || recv_capacity_rows < 0 || check_layout(layout)) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (!aligned16(send_buf) || ((uintptr_t)recv_ptrs & 7u)) return MW_ERR_ALIGNMENT;
     mw_copy_args a = base_args(ctx);
@@ -309,13 +438,14 @@ int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, int64_t 
 {
     if (!ctx || !x || !send_buf || !recv_base) return MW_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(send_buf) || !aligned16(recv_base) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
-    if (ctx->cfg.flags & (MW_FLAG_COPY_BULK | MW_FLAG_COPY_REG_STORE | MW_FLAG_COPY_LDST)) {
+    if (ctx->cfg.flags & MW_FLAG_COPY_BULK) {
         int rc = mw_pack(ctx, x, layout, send_buf, send_capacity_rows, stream);
         if (rc != MW_OK) return rc;
         return mw_deliver(ctx, layout, send_buf, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
     }
     // one pass: every hidden row is read once and written to its send slot(s) and to all its receive slots
     if (recv_stride_bytes < 0 || recv_capacity_rows < 0 || send_capacity_rows < 0 || check_layout(layout)) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
     mw_copy_args a = base_args(ctx);
@@ -351,13 +481,11 @@ int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert
         if (rc != MW_OK) return rc;
         return mw_dispatch(ctx, x, layout, send_buf, send_capacity_rows, recv_base, recv_stride_bytes, recv_capacity_rows, stream);
     }
-    if (view) {
-        const mw_dev &d = ctx->d;
-        view->token_mask = d.token_mask; view->token_ndest = d.token_ndest; view->token_group = d.token_group;
-        view->token_mw_row = d.token_mw_row; view->mw_row_token = d.mw_row_token; view->group_offsets = d.group_offsets;
-        view->group_mask = d.group_mask; view->rank_offsets = d.rank_offsets; view->rank_tokens = d.rank_tokens;
-        view->dest_rank = d.dest_rank; view->dest_pos = d.dest_pos; view->totals = d.totals;
-        view->T = T; view->W = ctx->W; view->Kd = ctx->Kd; view->reserved = 0;
+    MW_REFUSE_IF_POISONED(ctx);
+    if (view) fill_view(ctx, T, view);
+    {
+        const int rc = order_after_side_plans(ctx, as_stream(stream));    // the launch writes the accumulators plans share
+        if (rc != MW_OK) return rc;
     }
     return mw_small_launch(ctx, topk_ids, expert_to_rank, T, x, send_buf, send_capacity_rows, recv_base, recv_stride_bytes,
                            recv_capacity_rows, as_stream(stream));
@@ -393,7 +521,7 @@ int mw_allgather_pack(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int 
     a.dst_count = dst_rank_count;
     a.capacity_rows = INT64_MAX;
     int rc;
-    if (!(ctx->cfg.flags & (MW_FLAG_COPY_BULK | MW_FLAG_COPY_REG_STORE | MW_FLAG_COPY_LDST))) {
+    if (!(ctx->cfg.flags & MW_FLAG_COPY_BULK)) {
         // one pass: every shard is read once and written to its send slot(s) and to its slot in every region of the window
         a.mode = layout == MW_LAYOUT_MULTIWRITE ? MW_CP_AG_FUSED_MW : MW_CP_AG_FUSED_UC;
         a.src = (const uint8_t *)shards; a.dst = (uint8_t *)recv_base; a.dst2 = (uint8_t *)send_buf;
@@ -422,6 +550,17 @@ int64_t mw_pair_balanced_direct_bytes(int64_t shard_bytes, int32_t ranks_per_dom
     if (ranks_per_domain <= 1) return shard_bytes;
     const int64_t c = layout == MW_LAYOUT_MULTIWRITE ? 1 : ranks_per_domain - 1;
     return (shard_bytes * c / (1 + c)) / 16 * 16;
+}
+
+int64_t mw_pair_split_direct_bytes(int64_t shard_bytes, int32_t ranks_per_domain, int layout, double w_direct, double w_pair)
+{
+    if (ranks_per_domain <= 1 || !(w_direct > 0.0) || !(w_pair > 0.0)) return shard_bytes;
+    const double copies = layout == MW_LAYOUT_MULTIWRITE ? 1.0 : (double)(ranks_per_domain - 1);
+    // a direct link carries d bytes, the pair link `copies` times the rest: d / w_direct = copies (s - d) / w_pair
+    const double together = floor((double)shard_bytes * copies * w_direct / (w_pair + copies * w_direct));
+    int64_t d = (int64_t)together / 16 * 16;
+    if (d > shard_bytes) d = shard_bytes / 16 * 16;
+    return d;
 }
 
 int mw_paired_allgather(mw_ctx *ctx, const void *shards, int64_t shard_bytes, int64_t direct_bytes, int layout,

@@ -110,6 +110,7 @@ __global__ void __launch_bounds__(kCombineMaxThreads, kCombineMinBlocks) k_combi
 extern "C" int mw_combine(mw_ctx *ctx, const void *z_base, int64_t z_stride_bytes, const float *weights, void *y, void *stream)
 {
     if (!ctx || !z_base || !y || z_stride_bytes < 0) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (((uintptr_t)z_base & 15u) || ((uintptr_t)y & 15u) || z_stride_bytes % 16 || ((uintptr_t)weights & 3u)) return MW_ERR_ALIGNMENT;
     const int T = ctx->planned_T;

@@ -8,15 +8,11 @@
 //                 a thread loads its vectors once and stores them to every destination of the row.  The deliver
 //                 from a MultiWrite send buffer walks the rows from the last to the first and streams its stores,
 //                 so that the send rows the pack launch just wrote are read from L2.
-// Behind flags, and for the relay's second level: a persistent grid of one block per SM, one pipeline per warp,
-// work item = (row, chunk of at most 7168 bytes), claimed through a ticket counter.
+// Behind MW_FLAG_COPY_BULK: a persistent grid of one block per SM, one pipeline per warp, work item = (row, chunk
+// of at most 7168 bytes), claimed through a ticket counter.
 //   k_copy_bulk   bulk asynchronous copies global -> shared (completion counted on an mbarrier),
 //                 several stages deep, then one shared -> global bulk copy per destination, issued
-//                 by different lanes (MW_FLAG_COPY_BULK).
-//   k_copy_stage  same loads; the staged chunk is read once into registers and written to every
-//                 destination with 16-byte stores (MW_FLAG_COPY_REG_STORE).
-//   k_copy_ldst   no staging: 16-byte loads and stores through registers, static split
-//                 (MW_FLAG_COPY_LDST).
+//                 by different lanes.
 // Measured on B200 (4096 rows of 14336 bytes, 7.7 copies each): deliver 75 us with k_copy_rows after a pack
 // launch (6.8 TB/s), 88 us with k_copy_bulk.
 #include "mw_internal.cuh"
@@ -26,9 +22,6 @@ namespace {
 constexpr int kMaxBulkWarps = 8;       // pipelines per block (one per warp)
 constexpr int kMaxStages = 8;
 constexpr int64_t kMaxChunk = 7168;    // bytes per work item: 4 warps x 8 stages x 7 KB fill the 224 KB a block may use
-constexpr int kRegVec = (int)(kMaxChunk / 512);   // 16-byte vectors per lane for the largest chunk
-constexpr int kLdstThreads = 512;
-constexpr int kWaitLimit = 1 << 20;    // mbarrier polls (about 1 us each) before giving up
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -40,11 +33,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Polls with a suspend-time hint; false after kWaitLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// Polls with a suspend-time hint of 1 us; false after `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int limit)
 {
     const uint32_t addr = smem_u32(bar);
-    for (int i = 0; i < kWaitLimit; ++i) {
+    for (int i = 0; i < limit; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -80,12 +73,6 @@ __device__ __forceinline__ uint64_t policy_evict_normal()
     asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
-__device__ __forceinline__ uint4 lds_v4(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
 __device__ __forceinline__ uint4 ld_stream(const uint8_t *p)
 {
     uint4 v;
@@ -93,17 +80,6 @@ __device__ __forceinline__ uint4 ld_stream(const uint8_t *p)
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-// receive rows are written once and not read again by this path: streaming store
-__device__ __forceinline__ void st_stream(uint8_t *p, const uint4 &v)
-{
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-// send rows are read again by the deliver launch that follows: ordinary store, stays in L2
-__device__ __forceinline__ void st_keep(uint8_t *p, const uint4 &v)
-{
-    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
 __device__ __forceinline__ void flag_error(const mw_copy_args &a, int err) { atomicCAS(&a.totals->status, 0, err); }
 
 // ---- the work list -------------------------------------------------------------------------
@@ -137,7 +113,6 @@ __device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t
 }
 
 // Rows whose source is found through an index array: the index is loaded one item ahead of its use.
-__device__ __forceinline__ const uint8_t *src_row(const mw_copy_args &a, int64_t row) { return src_row(a, row, a.mode); }
 __device__ __forceinline__ bool src_is_indexed(const mw_copy_args &a, int mode)
 {
     return mode == MW_CP_PACK_MW || mode == MW_CP_DISPATCH_MW || mode == MW_CP_DISPATCH_UC || (mode == MW_CP_SCATTER && a.src_index);
@@ -395,122 +370,6 @@ __device__ __forceinline__ ItemGeom geom(const mw_copy_args &a, int64_t item)
     return g;
 }
 
-// ---- bulk-copy loads, register stores ------------------------------------------------------
-// A stage is free as soon as it has been read into registers, so it is refilled right after the
-// stores of its chunk have been issued.
-__global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_stage(const __grid_constant__ mw_copy_args a)
-{
-    extern __shared__ __align__(128) uint8_t stage_mem[];
-    __shared__ __align__(8) uint64_t bars[kMaxBulkWarps * kMaxStages];
-    __shared__ int64_t ring[kMaxBulkWarps * kMaxStages];      // item held by every stage, -1 = none
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nwarps = blockDim.x >> 5;
-    const int nst = a.stages;
-    const uint32_t stage_stride = ((uint32_t)a.chunk_bytes + 127u) & ~127u;
-    uint8_t *stages = stage_mem + (size_t)warp * nst * stage_stride;
-    uint64_t *bar = bars + warp * kMaxStages;
-    int64_t *held = ring + warp * kMaxStages;
-    if (lane == 0)
-        for (int s = 0; s < nst; ++s) mbar_init(bar + s, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    grid_launch_dependents();
-    grid_dependency_wait();        // everything above overlapped the previous kernel's tail
-    if (plan_unusable(a)) return;
-
-    const int64_t items = n_rows(a) * a.chunks_per_row;
-    const bool keep = writes_send_buffer(a);
-    auto issue_load = [&](int64_t item, int index, int s) {
-        const ItemGeom g = geom(a, item);
-        mbar_expect_tx(bar + s, g.bytes);
-        bulk_load(stages + (size_t)s * stage_stride, src_row_with(a, g.row, index) + g.off, g.bytes, bar + s);
-    };
-
-    // first loads: item (lane * warps of the grid + this warp) goes to stage `lane`, issued by that lane, so a
-    // small launch spreads over all warps and a large one starts with every pipeline full
-    const int npro = nst;
-    const int64_t gw = (int64_t)warp * gridDim.x + blockIdx.x;
-    if (lane < nst) {
-        const int64_t it = lane < npro ? (int64_t)lane * gridDim.x * nwarps + gw : -1;
-        const bool has = it >= 0 && it < items;
-        held[lane] = has ? it : -1;
-        if (has) issue_load(it, src_is_indexed(a) ? a.src_index[it / a.chunks_per_row] : 0, lane);
-    }
-    TicketSource src;                 // used by lane 0 only
-    int64_t pend_item = -1;           // next item to load (lane 0), chosen one iteration before its load is issued
-    int pend_index = 0;
-    if (lane == 0) {
-        src.start(a.work_ctr, items, a.batch, (int64_t)gridDim.x * nwarps * npro);
-        pend_item = src.next();
-        if (pend_item >= 0 && src_is_indexed(a)) pend_index = a.src_index[pend_item / a.chunks_per_row];
-    }
-    __syncwarp();
-
-    // descriptors of the first item
-    RawDesc raw_next = {-1, -1, 0};
-    if (held[0] >= 0) raw_next = fetch_raw(a, held[0] / a.chunks_per_row, lane);
-
-    bool ok = true;
-    int n = 0;
-    for (;; ++n) {
-        const int s = n % nst;
-        const int64_t item = held[s];
-        if (item < 0) break;
-        const ItemGeom g = geom(a, item);
-        const int nvec = (int)(g.bytes >> 4);
-        int nd;
-        uint8_t *my_dst = resolve_dst(a, g.row, lane, raw_next, &nd);
-        {   // load the next item's descriptors now; they are looked at one iteration later
-            const int64_t nitem = held[(n + 1) % nst];
-            if (nitem >= 0) raw_next = fetch_raw(a, nitem / a.chunks_per_row, lane);
-        }
-        if (!mbar_wait(bar + s, (uint32_t)(n / nst) & 1u)) { ok = false; break; }
-        const uint32_t stage = smem_u32(stages + (size_t)s * stage_stride);
-        uint4 v[kRegVec];
-#pragma unroll
-        for (int u = 0; u < kRegVec; ++u)
-            if (u * 32 + lane < nvec) v[u] = lds_v4(stage + (uint32_t)(u * 32 + lane) * 16u);
-        for (int qb = 0; qb < nd; qb += 32) {
-            if (qb) my_dst = qb + lane < nd ? dst_row(a, g.row, qb + lane) : nullptr;
-            const int nq = min(32, nd - qb);
-            for (int q = 0; q < nq; ++q) {
-                uint8_t *d = (uint8_t *)__shfl_sync(0xffffffffu, (unsigned long long)my_dst, q);
-                if (!d) continue;
-                d += g.off + (int64_t)lane * 16;
-                if (keep) {
-#pragma unroll
-                    for (int u = 0; u < kRegVec; ++u)
-                        if (u * 32 + lane < nvec) st_keep(d + (int64_t)u * 512, v[u]);
-                } else {
-#pragma unroll
-                    for (int u = 0; u < kRegVec; ++u)
-                        if (u * 32 + lane < nvec) st_stream(d + (int64_t)u * 512, v[u]);
-                }
-            }
-        }
-        __syncwarp();                       // every lane has the chunk in registers: the stage can be reloaded
-        if (lane == 0) {
-            // order this warp's reads of the stage before the asynchronous write that refills it
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            held[s] = pend_item;
-            if (pend_item >= 0) {
-                issue_load(pend_item, pend_index, s);
-                pend_item = src.next();
-                if (pend_item >= 0 && src_is_indexed(a)) pend_index = a.src_index[pend_item / a.chunks_per_row];
-            }
-        }
-        __syncwarp();                       // held[s] is visible to all lanes
-    }
-    if (!ok) {
-        // a load never arrived: report it, then give the loads still in flight a bounded chance to land
-        if (lane == 0) flag_error(a, MW_ERR_TIMEOUT);
-        for (int m = n + 1; m < n + nst; ++m)
-            if (held[m % nst] >= 0) mbar_wait(bar + (m % nst), (uint32_t)(m / nst) & 1u);
-    }
-    tickets_finish(a, lane, (unsigned)(gridDim.x * nwarps), items > (int64_t)gridDim.x * nwarps * npro);
-}
-
 // ---- bulk-copy loads, bulk-copy stores ------------------------------------------------------
 __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_bulk(const __grid_constant__ mw_copy_args a)
 {
@@ -537,7 +396,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_bulk(const __gri
     const uint64_t policy = writes_send_buffer(a) ? policy_evict_normal() : policy_evict_first();
     auto issue_load = [&](int64_t item, int index, int s) {
         const ItemGeom g = geom(a, item);
-        mbar_expect_tx(bar + s, g.bytes);
+        mbar_expect_tx(bar + s, g.bytes + (uint32_t)a.expect_extra);
         bulk_load(stages + (size_t)s * stage_stride, src_row_with(a, g.row, index) + g.off, g.bytes, bar + s);
     };
 
@@ -577,7 +436,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_bulk(const __gri
             const int64_t nitem = held[(n + 1) % nst];
             if (nitem >= 0) raw_next = fetch_raw(a, nitem / a.chunks_per_row, lane);
         }
-        if (!mbar_wait(bar + s, (uint32_t)(n / nst) & 1u)) { ok = false; break; }
+        if (!mbar_wait(bar + s, (uint32_t)(n / nst) & 1u, a.wait_limit)) { ok = false; break; }
         const uint8_t *stage = stages + (size_t)s * stage_stride;
         if (my_dst) bulk_store(my_dst + g.off, stage, g.bytes, policy);
         for (int q = lane + 32; q < nd; q += 32) {
@@ -602,50 +461,10 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32, 1) k_copy_bulk(const __gri
     if (!ok) {
         if (lane == 0) flag_error(a, MW_ERR_TIMEOUT);
         for (int m = n + 1; m < n + nst - 1; ++m)      // stages n+1 .. n+nst-2 hold loads issued ahead
-            if (held[m % nst] >= 0) mbar_wait(bar + (m % nst), (uint32_t)(m / nst) & 1u);
+            if (held[m % nst] >= 0) mbar_wait(bar + (m % nst), (uint32_t)(m / nst) & 1u, a.wait_limit);
     }
     bulk_wait_all();
     tickets_finish(a, lane, (unsigned)(gridDim.x * nwarps), items > (int64_t)gridDim.x * nwarps * npro);
-}
-
-// ---- register copies, no staging ---------------------------------------------------------------
-__global__ void __launch_bounds__(kLdstThreads) k_copy_ldst(const __grid_constant__ mw_copy_args a)
-{
-    grid_launch_dependents();
-    grid_dependency_wait();
-    if (plan_unusable(a)) return;
-    constexpr int U = 4;
-    const int lane = threadIdx.x & 31;
-    const int warps_per_block = kLdstThreads / 32;
-    const int64_t items = n_rows(a) * a.chunks_per_row;
-    const int64_t step = (int64_t)gridDim.x * warps_per_block;
-    for (int64_t item = (int64_t)(threadIdx.x >> 5) * gridDim.x + blockIdx.x; item < items; item += step) {
-        const ItemGeom g = geom(a, item);
-        const int nvec = (int)(g.bytes >> 4);
-        const int nd = n_dst(a, g.row);
-        const uint8_t *src = src_row(a, g.row) + g.off;
-        for (int qb = 0; qb < nd; qb += 32) {
-            uint8_t *my_dst = qb + lane < nd ? dst_row(a, g.row, qb + lane) : nullptr;
-            const int nq = min(32, nd - qb);
-            for (int v0 = 0; v0 < nvec; v0 += 32 * U) {
-                uint4 v[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int vi = v0 + u * 32 + lane;
-                    if (vi < nvec) v[u] = ld_stream(src + (int64_t)vi * 16);
-                }
-                for (int q = 0; q < nq; ++q) {
-                    uint8_t *d = (uint8_t *)__shfl_sync(0xffffffffu, (unsigned long long)my_dst, q);
-                    if (!d) continue;
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        const int vi = v0 + u * 32 + lane;
-                        if (vi < nvec) st_stream(d + g.off + (int64_t)vi * 16, v[u]);
-                    }
-                }
-            }
-        }
-    }
 }
 
 // ---- one block per (row, piece): plain loads and stores, ordinary grid ---------------------------
@@ -770,25 +589,23 @@ CopyShape choose_shape(const mw_ctx *ctx, const mw_copy_args &a, int64_t est_row
 int mw_copy_smem_setup(mw_ctx *ctx)
 {
     const int limit = ctx->max_smem_optin - 2048;
-    if (cudaFuncSetAttribute(k_copy_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, limit) != cudaSuccess ||
-        cudaFuncSetAttribute(k_copy_stage, cudaFuncAttributeMaxDynamicSharedMemorySize, limit) != cudaSuccess)
-        return MW_ERR_CUDA;
+    if (cudaFuncSetAttribute(k_copy_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, limit) != cudaSuccess) return MW_ERR_CUDA;
     return MW_OK;
 }
 
-// Default: one block per (row, piece) on an ordinary grid.  With MW_FLAG_COPY_BULK / _REG_STORE / _LDST (or a grid
-// too large for 32-bit block indices): chooses the work-item size and the pipeline shape and launches a persistent grid.
+// Default: one block per (row, piece) on an ordinary grid.  With MW_FLAG_COPY_BULK (or a launch whose row bound is
+// loose, or a grid too large for 32-bit block indices): chooses the work-item size and the pipeline shape and launches
+// the persistent bulk-copy grid.
 int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
 {
     const bool overlap = !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP);
     const int64_t est_rows = a.host_rows >= 0 ? a.host_rows : 0;
     cudaError_t err;
-    const uint32_t other = MW_FLAG_COPY_LDST | MW_FLAG_COPY_REG_STORE | MW_FLAG_COPY_BULK;
     int64_t pieces = 0;
     int threads = 0;
     // one-to-one copies need more loads in flight per thread; fan-out copies are bound by their stores
     const int V = mode_is_one_to_one(a.mode) ? 2 : 1;
-    if (!(ctx->cfg.flags & other) && a.host_rows >= 0 && !a.loose_bound) {
+    if (!(ctx->cfg.flags & MW_FLAG_COPY_BULK) && a.host_rows >= 0 && !a.loose_bound) {
         // near-equal pieces of at most kRowsMaxVecs vectors; smaller ones while the grid would leave SMs idle
         const int64_t vecs = a.row_bytes / 16;
         pieces = (vecs + kRowsMaxVecs - 1) / kRowsMaxVecs;
@@ -808,8 +625,8 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_PACK_MW: err = rows_launch<2, MW_CP_PACK_MW>(grid, block, st, overlap, a); break;
         case MW_CP_SCATTER:
             // no source index: the rows are a send buffer, packed just before
-            err = a.src_index ? rows_launch<1, MW_CP_SCATTER>(grid, block, st, overlap, a)
-                              : rows_launch<1, MW_CP_SCATTER, true>(grid, block, st, overlap, a);
+            err = (a.src_index || a.src_not_recent) ? rows_launch<1, MW_CP_SCATTER>(grid, block, st, overlap, a)
+                                                    : rows_launch<1, MW_CP_SCATTER, true>(grid, block, st, overlap, a);
             break;
         case MW_CP_DELIVER_UC: err = rows_launch<2, MW_CP_DELIVER_UC>(grid, block, st, overlap, a); break;
         case MW_CP_PAIR_DIRECT: err = rows_launch<1, MW_CP_PAIR_DIRECT>(grid, block, st, overlap, a); break;
@@ -822,13 +639,8 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         case MW_CP_DISPATCH_UC: err = rows_launch<1, MW_CP_DISPATCH_UC>(grid, block, st, overlap, a); break;
         case MW_CP_AG_FUSED_MW: err = rows_launch<1, MW_CP_AG_FUSED_MW>(grid, block, st, overlap, a); break;
         case MW_CP_AG_FUSED_UC: err = rows_launch<1, MW_CP_AG_FUSED_UC>(grid, block, st, overlap, a); break;
-        default: return MW_ERR_INVALID_ARG;     // the two-launch AllGather modes only run with a MW_FLAG_COPY_* bit
+        default: return MW_ERR_INVALID_ARG;     // the two-launch AllGather modes only run with MW_FLAG_COPY_BULK
         }
-    } else if (ctx->cfg.flags & MW_FLAG_COPY_LDST) {
-        const int64_t chunk = choose_chunk(a.row_bytes, est_rows, (int64_t)ctx->sm_count * 2 * (kLdstThreads / 32));
-        a.chunk_bytes = (int32_t)chunk;
-        a.chunks_per_row = (int32_t)((a.row_bytes + chunk - 1) / chunk);
-        err = mw_launch(k_copy_ldst, dim3(ctx->sm_count * 2), dim3(kLdstThreads), 0, st, overlap, a);
     } else {
         const CopyShape s = choose_shape(ctx, a, est_rows);
         if (s.stages < 2 || s.warps < 1 || s.warps > kMaxBulkWarps || s.chunk > kMaxChunk) return MW_ERR_INVALID_ARG;
@@ -838,11 +650,13 @@ int mw_copy_launch(mw_ctx *ctx, mw_copy_args a, cudaStream_t st)
         a.stages = s.stages;
         a.batch = s.batch;
         a.work_ctr = ctx->d.copy_ctr;
+        a.wait_limit = ctx->copy_wait_limit;
+        // test hook: every load is announced 16 bytes larger than it is, so no stage ever completes and the
+        // bounded wait runs out (the loads themselves are untouched and land as usual)
+        a.expect_extra = (ctx->test_skew & MW_TEST_SKEW_BULK_LOAD) ? 16 : 0;
+        ctx->test_skew &= ~(uint32_t)MW_TEST_SKEW_BULK_LOAD;
         const size_t smem = (size_t)(s.warps * s.stages * stage_stride);
-        if (ctx->cfg.flags & MW_FLAG_COPY_REG_STORE)
-            err = mw_launch(k_copy_stage, dim3(ctx->sm_count), dim3(s.warps * 32), smem, st, overlap, a);
-        else
-            err = mw_launch(k_copy_bulk, dim3(ctx->sm_count), dim3(s.warps * 32), smem, st, overlap, a);
+        err = mw_launch(k_copy_bulk, dim3(ctx->sm_count), dim3(s.warps * 32), smem, st, overlap, a);
     }
     ctx->launches += 1;
     if (err != cudaSuccess) { cudaGetLastError(); return MW_ERR_CUDA; }

@@ -51,6 +51,15 @@ struct mw_dev {
     unsigned int *gbar;                            // arrival counter of the fused plan's grid barriers
     unsigned int *copy_ctr;                        // [2] work-ticket and finished-warp counters of the copy kernels
     mw_acc *acc;                                   // [2]
+    unsigned int *gave_up;                         // set by a plan whose wait gave up; later plans refuse to run until mw_reset
+};
+
+// What the data path needs to know about one plan: where its arrays are and what was planned into them.
+struct mw_slot {
+    mw_dev d;               // the slot's arrays (the scratch pointers are the same in both slots)
+    int32_t planned_T;      // T of the plan held by the slot, -1 if none
+    const void *prefetched; // rows that plan's launch brought into L2 (null: none)
+    uint32_t plan_epoch;    // value of mw_ctx::epoch when that plan was issued
 };
 
 struct mw_ctx {
@@ -59,14 +68,28 @@ struct mw_ctx {
     int sm_count;
     int max_smem_optin;
     int l2_bytes;
+    // The current plan slot (the one mw_pack / mw_deliver / ... read), spelled out as members;
+    // `other` is the second slot, which mw_plan_next fills while the current one is in use.
     mw_dev d;
+    int32_t planned_T;      // T of the latest plan, -1 before the first
+    const void *prefetched; // rows the latest plan launch brought into L2 (null: none)
+    uint32_t plan_epoch;    // epoch of the current slot's plan
+    mw_slot other;
+    int next_pending;       // `other` holds a plan issued by mw_plan_next that mw_plan_swap has not taken yet
+    cudaStream_t plan_stream;            // library-owned stream of mw_plan_next (highest priority, non-blocking)
+    cudaEvent_t ev_submitted, ev_planned; // caller's stream -> plan stream; plan stream -> caller's stream
+    int plans_on_side_stream;            // the latest plan launch went to plan_stream and ev_planned marks its end
     void *slab;
+    size_t scratch_bytes;   // the part of the slab mw_reset re-initialises starts at scratch_begin
+    uint8_t *scratch_begin;
     uint32_t epoch;         // plans issued so far (tile records carry it, so they need no clearing)
     uint32_t tickets_used;  // tile tickets handed out by all previous plans
     uint32_t gbar_arrivals; // grid-barrier arrivals made by all previous fused plans
-    int coop_ok;            // device supports cooperative launch
-    int32_t planned_T;      // T of the latest plan, -1 before the first
-    const void *prefetched; // rows the latest plan launch brought into L2 (null: none)
+    int32_t spin_limit;     // polls a look-back waits for a predecessor's record before it gives up
+    int32_t bar_spin_limit; // polls a block waits at a grid barrier
+    int32_t copy_wait_limit;// polls (about 1 us each) the bulk-copy engine waits for a load
+    uint32_t test_skew;     // MW_TEST_SKEW_* bits applied to the next launch (mw_test_skew_waits)
+    int poisoned;           // a wait gave up: host counters and device scratch may be out of step until mw_reset
     uint32_t gm_epoch;      // epoch of the plan the group-major arrays were made from (0: none)
     int64_t launches;
     // host staging (MW_FLAG_HOST_STAGING)
@@ -74,6 +97,9 @@ struct mw_ctx {
     uint8_t *st_x, *st_send, *st_recv;
     int64_t st_recv_rows;
 };
+
+// Calls that use the device refuse a context in which a device-side wait has given up (see mw_reset).
+#define MW_REFUSE_IF_POISONED(ctx) do { if ((ctx)->poisoned) return MW_ERR_TIMEOUT; } while (0)
 
 // Ordinary launch; with `overlap` the kernel's blocks may be scheduled while the previous kernel of
 // the stream drains (programmatic dependent launch).  Such a kernel must execute
@@ -106,6 +132,14 @@ __device__ __forceinline__ uint64_t equal_mask64(int a, int b)
     uint32_t m;
     asm("set.eq.u32.s32 %0, %1, %2;" : "=r"(m) : "r"(a), "r"(b));
     return ((uint64_t)m << 32) | m;
+}
+// Hash step for the table keyed by bitmap (one call per 64-bit word): the golden-ratio combine followed by a
+// 64-bit finaliser, both public-domain constants.
+__device__ __forceinline__ uint64_t mix64(uint64_t h, uint64_t v)
+{
+    h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
+    h ^= h >> 33; h *= 0xff51afd7ed558ccdull; h ^= h >> 29;
+    return h;
 }
 // Word w of a bitmap held in registers.  Indexing the array with the variable of a loop that the compiler does
 // not unroll (a loop over words around a loop over set bits) moves the whole array to local memory, and every
@@ -174,6 +208,9 @@ struct mw_copy_args {
     int keep_in_l2;            // destination rows are read again soon: do not mark them evict-first
     int src_in_l2;             // fused dispatch: the source rows were prefetched into L2 by the plan launch
     int loose_bound;           // host_rows may be far above the row count: take the persistent grid, which pays nothing for absent rows
+    int src_not_recent;        // SCATTER without a source index whose rows were not written by the launch just before
+    int wait_limit;            // bulk-copy engine: polls (about 1 us each) before a wait for a load gives up
+    int expect_extra;          // bulk-copy engine, test hook: bytes added to the announced size of every load
     unsigned int *work_ctr;    // [2] ticket counter, finished-warp counter (both zero between launches)
     int Kd, R, dst_begin, dst_count;
     int pair_n, pair_copies;   // paired AllGather: ranks per domain, copies of the relayed segment on the pair link

@@ -251,12 +251,13 @@ int mw_order_smem_setup(mw_ctx *ctx)
 extern "C" int mw_group_major(mw_ctx *ctx, mw_group_major_view *view, void *stream)
 {
     if (!ctx) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     if (view) {
         view->group_dest_rank = ctx->d.gm_rank; view->group_dest_offset = ctx->d.gm_offset;
         view->dest_pos_gm = ctx->d.dest_pos_gm; view->Kd = ctx->Kd; view->reserved = 0;
     }
-    ctx->gm_epoch = ctx->epoch;
+    ctx->gm_epoch = ctx->plan_epoch;
     const int T = ctx->planned_T;
     if (T == 0) return MW_OK;
     GmArgs a;
@@ -276,7 +277,8 @@ extern "C" int mw_deliver_group_major(mw_ctx *ctx, const void *send_buf, void *r
                                       int64_t recv_capacity_rows, void *stream)
 {
     if (!ctx || !send_buf || !recv_base || recv_stride_bytes < 0 || recv_capacity_rows < 0) return MW_ERR_INVALID_ARG;
-    if (ctx->planned_T < 0 || ctx->gm_epoch != ctx->epoch) return MW_ERR_NO_PLAN;
+    MW_REFUSE_IF_POISONED(ctx);
+    if (ctx->planned_T < 0 || ctx->gm_epoch != ctx->plan_epoch) return MW_ERR_NO_PLAN;
     if (((uintptr_t)send_buf & 15u) || ((uintptr_t)recv_base & 15u) || recv_stride_bytes % 16) return MW_ERR_ALIGNMENT;
     if (recv_stride_bytes && recv_capacity_rows * ctx->cfg.row_bytes > recv_stride_bytes) return MW_ERR_CAPACITY;
     mw_copy_args a;
@@ -304,6 +306,7 @@ extern "C" int mw_expert_index(mw_ctx *ctx, const int32_t *topk_ids, const int32
                                int32_t *expert_token, int32_t *expert_slot, void *stream)
 {
     if (!ctx || !expert_to_rank || !expert_offsets || !expert_token || !expert_slot) return MW_ERR_INVALID_ARG;
+    MW_REFUSE_IF_POISONED(ctx);
     if (ctx->planned_T < 0) return MW_ERR_NO_PLAN;
     const int T = ctx->planned_T;
     if (T > 0 && !topk_ids) return MW_ERR_INVALID_ARG;

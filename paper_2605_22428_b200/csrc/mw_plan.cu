@@ -4,7 +4,7 @@
 // task decomposition in cs_send.  The slot layout rules are stated in mw.h.)
 //
 // Two ways to run the same three phases:
-//   k_plan_fused  one cooperative launch, one block per 256-token tile, all blocks resident, the
+//   k_plan_fused  one launch, one block per 256-token tile, all blocks resident, the
 //                 phases separated by two bounded grid barriers; a token's values stay in the
 //                 registers of "its" thread from phase to phase.  Taken whenever the tiles fit on
 //                 the SMs (T <= 256 x SM count).
@@ -28,13 +28,15 @@ constexpr int kEmpty = -1;
 constexpr unsigned long long kEmptyKey = ~0ull;
 constexpr int kNoLeader = 0x7fffffff;
 constexpr unsigned kFlagAgg = 1u, kFlagPrefix = 2u;
-constexpr int kSpinLimit = 1 << 20;  // look-back polls before a tile gives up (about a second)
 
 struct PlanArgs {
     const int32_t *ids, *e2r;
     int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask, Tm;
     int64_t row_bytes;
     uint32_t epoch, ticket_base, bar_base;
+    uint32_t wait_epoch;      // epoch a look-back expects in its predecessors' records (= epoch, unless a test skews it)
+    int spin_limit;           // look-back polls before a tile gives up (2^20: about a second)
+    int bar_spin_limit;       // polls of the arrival counter before a block gives up at a grid barrier
     const uint8_t *pf_base;   // rows to bring into L2 while the plan runs (fused plan only), or null
     int64_t pf_bytes;
     mw_dev d;
@@ -42,11 +44,21 @@ struct PlanArgs {
 
 __device__ __forceinline__ void set_status(int *status, int err) { atomicCAS(status, 0, err); }
 
-__device__ __forceinline__ uint64_t mix64(uint64_t h, uint64_t v)
+// A wait gave up: the plan under way is invalid, and it will not restore the shared scratch (bitmap table, counters)
+// to the state the next plan expects.  The flag makes every later plan on the context refuse to run until mw_reset
+// has re-initialised the scratch, also when the host has not looked at the status in between.
+__device__ __forceinline__ void give_up(const PlanArgs &a, int *status)
 {
-    h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
-    h ^= h >> 33; h *= 0xff51afd7ed558ccdull; h ^= h >> 29;
-    return h;
+    set_status(status, MW_ERR_TIMEOUT);
+    *(volatile unsigned int *)a.d.gave_up = 1u;
+    __threadfence();                         // both are visible before anything this thread publishes afterwards
+}
+// True (and the slot's accounting says MW_ERR_TIMEOUT) if an earlier plan on this context gave up.
+__device__ __forceinline__ bool refuses_to_plan(const PlanArgs &a)
+{
+    if (*(volatile const unsigned int *)a.d.gave_up == 0u) return false;
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.d.totals->status = MW_ERR_TIMEOUT;
+    return true;
 }
 
 
@@ -89,6 +101,7 @@ __device__ __forceinline__ int table_insert_word(unsigned long long *slot_key, i
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(MW_TILE) k_plan_mask(PlanArgs a)
 {
+    if (refuses_to_plan(a)) return;
     const int t = blockIdx.x * MW_TILE + threadIdx.x;
     mw_acc *acc = a.d.acc + (a.epoch & 1u);
     int valid = 0, self_only = 0, bad = 0;
@@ -175,6 +188,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
     __shared__ int warp_sums[MW_TILE / 32];
     __shared__ int s_tile;
 
+    if (refuses_to_plan(a)) return;
     const int tid = threadIdx.x;
     mw_acc *acc = a.d.acc + (a.epoch & 1u);
     // Tiles are numbered in the order blocks start, so a tile only ever waits for tiles that are already running.
@@ -228,13 +242,13 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
                 volatile unsigned long long *prev = a.d.tile_state + (size_t)j * a.NC + c;
                 unsigned long long s = 0;
                 int spins = 0;
-                for (; spins < kSpinLimit; ++spins) {
+                for (; spins < a.spin_limit; ++spins) {
                     s = *prev;
                     const uint32_t hi = (uint32_t)(s >> 32);
-                    if ((hi >> 2) == (a.epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
+                    if ((hi >> 2) == (a.wait_epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
                     __nanosleep(64);
                 }
-                if (spins == kSpinLimit) { set_status(&acc->status, MW_ERR_TIMEOUT); break; }
+                if (spins == a.spin_limit) { give_up(a, &acc->status); break; }
                 excl += (uint32_t)s;
                 if (((uint32_t)(s >> 32) & 3u) == kFlagPrefix) break;
             }
@@ -381,6 +395,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
     __shared__ RankScratch rank_scratch;
     const int t = blockIdx.x * MW_TILE + threadIdx.x;
     const mw_totals *tot = a.d.totals;
+    if (tot->status == MW_ERR_TIMEOUT) return;      // a look-back gave up (now or in an earlier plan): nothing below can be trusted
     const int Tn = (int)tot->T_nonempty, G = (int)tot->G, SD = (int)tot->total_dest;
     if (t <= a.T && t > G) a.d.group_offsets[t] = -1;
     if (t < a.T) {
@@ -428,7 +443,6 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
 // Fused plan: the three phases in one cooperative launch.
 // ------------------------------------------------------------------------------------------
 constexpr int kLookBack = 8;                  // predecessors a look-back reads per round trip (16 measured slower: more records not ready yet)
-constexpr int kBarrierSpinLimit = 1 << 21;   // polls of the arrival counter before a block gives up (about a second)
 
 __device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p)
 {
@@ -451,7 +465,7 @@ __device__ __forceinline__ void grid_barrier_arrive(unsigned int *counter)
 
 // A block that is still `alive` waits until the counter reaches `target`; returns false for a block
 // that gave up (now or before).  With a single block, block-level ordering is all that is needed.
-__device__ bool grid_barrier_wait(unsigned int *counter, unsigned int target, bool alive, int *status)
+__device__ bool grid_barrier_wait(const PlanArgs &a, unsigned int target, bool alive, int *status)
 {
     __shared__ int s_alive;
     if (gridDim.x == 1) {
@@ -462,8 +476,8 @@ __device__ bool grid_barrier_wait(unsigned int *counter, unsigned int target, bo
         int ok = alive ? 1 : 0;
         if (ok) {
             int spins = 0;
-            while ((int)(ld_volatile_u32(counter) - target) < 0) {
-                if (++spins > kBarrierSpinLimit) { ok = 0; set_status(status, MW_ERR_TIMEOUT); break; }
+            while ((int)(ld_volatile_u32(a.d.gbar) - target) < 0) {
+                if (++spins > a.bar_spin_limit) { ok = 0; give_up(a, status); break; }
                 __nanosleep(32);
             }
         }
@@ -502,6 +516,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
         }
         return;
     }
+    if (refuses_to_plan(a)) return;      // uniform over the grid (the flag only changes between plans): no block waits for another
     const int t = tile * MW_TILE + tid;
     const bool active = t < a.T;
     mw_acc *acc = a.d.acc + (a.epoch & 1u);
@@ -599,8 +614,8 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                         int spins = 0;
                         while (true) {
                             const uint32_t hi = (uint32_t)(s[i] >> 32);
-                            if ((hi >> 2) == (a.epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
-                            if (++spins > kSpinLimit) { set_status(&acc->status, MW_ERR_TIMEOUT); done = true; break; }
+                            if ((hi >> 2) == (a.wait_epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
+                            if (++spins > a.spin_limit) { give_up(a, &acc->status); done = true; break; }
                             __nanosleep(64);
                             s[i] = *(volatile unsigned long long *)(a.d.tile_state + (size_t)(j - i) * a.NC + c);
                         }
@@ -636,7 +651,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     __syncthreads();
     look_back(0, a.R);
     __syncthreads();
-    bool alive = grid_barrier_wait(a.d.gbar, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
+    bool alive = grid_barrier_wait(a, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
 
     // ---- phase B2: leaders and group sizes are final; every tile publishes its two totals ----
     int leader = -1, gcount = 0, lead_excl = 0, gc_excl = 0;
@@ -712,7 +727,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
         }
     }
-    alive = grid_barrier_wait(a.d.gbar, a.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
+    alive = grid_barrier_wait(a, a.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
     if (!alive) {
         if (tid == 0) set_status(&a.d.totals->status, MW_ERR_TIMEOUT);
         return;
@@ -834,11 +849,23 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.row_bytes = ctx->cfg.row_bytes;
     ctx->epoch += 1;
     a.epoch = ctx->epoch & 0x3fffffffu;
+    if (a.epoch == 0) {
+        // the 30-bit epoch of the look-back records starts a new lap: wipe the records of the lap before
+        if (cudaMemsetAsync(ctx->d.tile_state, 0, sizeof(unsigned long long) * (size_t)ctx->max_tiles * (size_t)ctx->NC, st) != cudaSuccess)
+            return MW_ERR_CUDA;
+    }
     a.ticket_base = ctx->tickets_used;
     a.d = ctx->d;
     a.bar_base = ctx->gbar_arrivals;
+    a.wait_epoch = a.epoch;
+    a.spin_limit = ctx->spin_limit;
+    a.bar_spin_limit = ctx->bar_spin_limit;
+    if (ctx->test_skew & MW_TEST_SKEW_LOOKBACK) a.wait_epoch = (a.epoch + 1u) & 0x3fffffffu;   // records nobody writes
+    if (ctx->test_skew & MW_TEST_SKEW_BARRIER) a.bar_base += 1u;                               // a count nobody reaches
+    ctx->test_skew &= ~(uint32_t)(MW_TEST_SKEW_LOOKBACK | MW_TEST_SKEW_BARRIER);
     const int blocks = a.ntiles;
     ctx->planned_T = T;
+    ctx->plan_epoch = ctx->epoch;
     // rows to bring into L2 meanwhile: the first half-L2 of them (the pack step reads them in ascending order)
     a.pf_base = (const uint8_t *)rows;
     ctx->prefetched = nullptr;
@@ -848,24 +875,19 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
         // One launch, at most one block per SM, phases separated by grid barriers.  The blocks wait for
         // one another, so all of them must become resident: an ordinary launch achieves that as soon
         // as earlier kernels of the stream have drained (the grid never exceeds the SM count and needs
-        // a fraction of an SM each); should other work keep SMs occupied for about a second, the
-        // barrier gives up with MW_ERR_TIMEOUT instead of hanging.  MW_FLAG_PLAN_COOPERATIVE asks the
-        // driver for the residency guarantee instead, at the price of a much slower launch call.
+        // a fraction of an SM each); blocks of other streams that occupy an SM are short-lived copy blocks.
+        // Should other work keep SMs occupied for about a second, the barrier gives up with
+        // MW_ERR_TIMEOUT instead of hanging (mw_reset then makes the context usable again;
+        // MW_FLAG_PLAN_MULTIPASS avoids the residency assumption altogether).
         // The plan is not launched as a programmatic dependent of the previous kernel: measured on
         // B200 that costs about 30 us per step, while the pack kernel that follows does overlap its
         // start-up with the plan.
-        cudaError_t e;
         void (*fn)(PlanArgs) = ctx->W <= 1 ? k_plan_fused<1> : ctx->W <= 2 ? k_plan_fused<2>
                              : ctx->W <= 4 ? k_plan_fused<4> : k_plan_fused<16>;
-        if ((ctx->cfg.flags & MW_FLAG_PLAN_COOPERATIVE) && ctx->coop_ok) {
-            void *params[] = {&a};
-            e = cudaLaunchCooperativeKernel((const void *)fn, dim3(blocks), dim3(MW_TILE), params, tile_smem_bytes(ctx), st);
-        } else {
-            // with rows to prefetch, one more block for every SM the tiles leave free
-            const int extra = a.pf_bytes > 0 ? ctx->sm_count - blocks : 0;
-            if (extra > 0 && a.pf_bytes == (int64_t)T * ctx->cfg.row_bytes) ctx->prefetched = rows;     // all of them fit
-            e = mw_launch(fn, dim3(blocks + extra), dim3(MW_TILE), tile_smem_bytes(ctx), st, false, a);
-        }
+        // with rows to prefetch, one more block for every SM the tiles leave free
+        const int extra = a.pf_bytes > 0 ? ctx->sm_count - blocks : 0;
+        if (extra > 0 && a.pf_bytes == (int64_t)T * ctx->cfg.row_bytes) ctx->prefetched = rows;     // all of them fit
+        const cudaError_t e = mw_launch(fn, dim3(blocks + extra), dim3(MW_TILE), tile_smem_bytes(ctx), st, false, a);
         if (e == cudaSuccess) {
             ctx->gbar_arrivals += 2u * (uint32_t)blocks;
             ctx->launches += 1;

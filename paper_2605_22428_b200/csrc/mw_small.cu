@@ -44,13 +44,6 @@ struct SmallArgs {
     mw_totals *totals;
 };
 
-__device__ __forceinline__ uint64_t mix64s(uint64_t h, uint64_t v)
-{
-    h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
-    h ^= h >> 33; h *= 0xff51afd7ed558ccdull; h ^= h >> 29;
-    return h;
-}
-
 // Exclusive prefix sum over the NT threads of the block; `total` is returned to every thread.  V is a packed word:
 // 32 bits hold the three sums of a 256-token batch, the 1024-token batch needs 64.
 template <int NT, class V>
@@ -167,7 +160,7 @@ __global__ void __launch_bounds__(NT) k_dispatch_small(const __grid_constant__ S
     int nd = 0, slot = -1;
     if (active) {
         uint64_t h = 0x2545f4914f6cdd1dull;
-        for (int w = 0; w < a.W; ++w) { const uint64_t m = mask64[t * a.W + w]; nd += __popcll(m); h = mix64s(h, m); }
+        for (int w = 0; w < a.W; ++w) { const uint64_t m = mask64[t * a.W + w]; nd += __popcll(m); h = mix64(h, m); }
         if (a.src_rank >= 0 && nd == 1 && ((mask64[t * a.W + (a.src_rank >> 6)] >> (a.src_rank & 63)) & 1)) atomicAdd(s_acc + 1, 1);
         if (nd > 0) {
             const uint32_t tag = (uint32_t)(h >> 32);
@@ -384,7 +377,7 @@ bool small_fits(const mw_ctx *ctx, int NT)
 bool mw_small_applies(const mw_ctx *ctx, int32_t T, int layout)
 {
     return layout == MW_LAYOUT_MULTIWRITE &&
-           !(ctx->cfg.flags & (MW_FLAG_PLAN_MULTIPASS | MW_FLAG_PLAN_COOPERATIVE | MW_FLAG_COPY_LDST | MW_FLAG_COPY_REG_STORE)) &&
+           !(ctx->cfg.flags & MW_FLAG_PLAN_MULTIPASS) &&
            ((T <= kSmallThreads && small_fits(ctx, kSmallThreads)) || (T <= kMidThreads && small_fits(ctx, kMidThreads)));
 }
 
@@ -432,6 +425,7 @@ int mw_small_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_
     ctx->launches += 1;
     ctx->planned_T = T;
     ctx->epoch += 2;          // a new plan (keeps the parity the tiled plan's double-buffered accumulators rely on)
+    ctx->plan_epoch = ctx->epoch;
     ctx->prefetched = nullptr;
     if (e != cudaSuccess) { cudaGetLastError(); return MW_ERR_CUDA; }
     return MW_OK;

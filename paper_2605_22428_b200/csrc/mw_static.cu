@@ -4,8 +4,7 @@
 // image instead of a workspace obtained from cudaMalloc.  Declared and documented in include/mw.h.
 #include <mutex>
 
-#include "mw.h"
-#include <cuda_runtime.h>
+#include "mw_internal.cuh"
 
 namespace {
 
@@ -27,13 +26,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScr
 
 std::mutex g_setup_mutex;
 StaticScratch *g_scratch_of_device[kMaxDevices];   // device address of the array, per device ordinal
-
-__device__ __forceinline__ uint64_t mix64(uint64_t h, uint64_t v)
-{
-    h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
-    h ^= h >> 33; h *= 0xff51afd7ed558ccdull; h ^= h >> 29;
-    return h;
-}
 
 // The array keeps whatever the previous call left: start every call from an empty table.
 __global__ void k_static_clear(StaticScratch *s, int32_t *status)

@@ -46,18 +46,11 @@ def test_dispatch_parity_large_configurations_reduced_hidden(cfg, seed, separate
     run_dispatch(wl.make_dispatch(cfg, seed, H=264), separate=separate)          # 528-byte rows: ragged against every tile size
 
 
-@pytest.mark.parametrize("cfg", [0, 1])
-def test_register_copy_variant_matches(cfg):
-    inp = wl.make_dispatch(cfg, H=None if cfg == 0 else 520)
-    run_dispatch(inp, flags=mw.MW_FLAG_COPY_LDST)
-
-
-@pytest.mark.parametrize("flags", [mw.MW_FLAG_PLAN_MULTIPASS, mw.MW_FLAG_PLAN_COOPERATIVE, mw.MW_FLAG_NO_OVERLAP,
-                                   mw.MW_FLAG_COPY_REG_STORE, mw.MW_FLAG_COPY_BULK,
-                                   mw.MW_FLAG_PLAN_MULTIPASS | mw.MW_FLAG_COPY_LDST | mw.MW_FLAG_NO_OVERLAP])
+@pytest.mark.parametrize("flags", [mw.MW_FLAG_PLAN_MULTIPASS, mw.MW_FLAG_NO_OVERLAP, mw.MW_FLAG_COPY_BULK, mw.MW_FLAG_SHORT_WAITS,
+                                   mw.MW_FLAG_PLAN_MULTIPASS | mw.MW_FLAG_COPY_BULK | mw.MW_FLAG_NO_OVERLAP])
 def test_launch_and_plan_variants_match(flags):
-    """The multi-pass plan, the grid plan (ordinary and cooperative launch), the non-overlapped launches
-    and the other copy kernels give the same bits as the defaults."""
+    """The multi-pass plan, the non-overlapped launches, the bulk-copy engine and the short wait limits give the
+    same bits as the defaults."""
     run_dispatch(wl.make_random_dispatch(41, T=3000, K=1, E=12, R=6, H=16), flags=flags)       # large groups
     run_dispatch(wl.make_dispatch("large_ep", 100, H=264), flags=flags, repeats=2)
     run_dispatch(wl.make_random_dispatch(31, T=1025, K=2, E=12, R=6, H=24, pad_fraction=0.1), flags=flags)

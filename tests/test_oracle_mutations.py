@@ -39,6 +39,10 @@ MUTATIONS = {
                                                    "return (r / ranks_per_server) * ranks_per_server;"),
     "paired allgather forwards the direct segment": ("relay_buf + ((int64_t)partner * copies + c) * relay_bytes, (size_t)relay_bytes);\n            ++k;",
                                                      "mine, (size_t)relay_bytes);\n            ++k;"),
+    "split ignores the copies on the pair link": ("floor((double)shard_bytes * c * w_direct / (w_pair + c * w_direct));",
+                                                  "floor((double)shard_bytes * w_direct / (w_pair + w_direct));"),
+    "split with the two bandwidths exchanged": ("floor((double)shard_bytes * c * w_direct / (w_pair + c * w_direct));",
+                                                "floor((double)shard_bytes * c * w_pair / (w_direct + c * w_pair));"),
     "bit index taken modulo 32": ("(uint64_t)1 << (r % 64)", "(uint64_t)1 << (r % 32)"),
     "always word 0": ("m[r / 64] |=", "m[0] |="),
     "padding treated as an error": ("if (id == -1) continue;                         /* padding slot            */", ""),
@@ -89,6 +93,7 @@ def run_pins():
     rpins.test_paper_example_four_local_four_remote()
     rpins.test_relay_brute_force(1, 12, 3, 7, 24, 4)
     ppins.test_every_rank_gets_its_domain_in_order(0, 8, 64, 32)
+    ppins.test_split_by_bandwidth_ratio_lets_both_link_classes_finish_together(1, 4096 + 16, 8, 1.0, 7.0)
     opins.test_group_major_brute_force(1, 8, 32, 4, 0.2)
     opins.test_group_major_with_few_large_groups()
     opins.test_expert_index_brute_force(1, 8, 32, 4, 0.2, True)

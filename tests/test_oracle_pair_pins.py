@@ -64,6 +64,50 @@ def test_paper_latencies_full_mesh_tp4():
         assert mwo.paired_allgather(sh, d, 0)[2]["max_link_bytes"] > t_mw * S
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("S,n,w_direct,w_pair", [(1 << 20, 4, 56.0, 56.0), (1 << 20, 4, 56.0, 25.0), (16 << 20, 4, 56.0, 112.0),
+                                                 (4096, 2, 3.0, 1.0), (4096 + 16, 8, 1.0, 7.0), (1 << 24, 4, 450.0, 50.0)])
+def test_split_by_bandwidth_ratio_lets_both_link_classes_finish_together(layout, S, n, w_direct, w_pair):
+    """Section 5.2 step 1.  Enumerate every split that is a multiple of 16 bytes: with exact fractions, the one the
+    oracle returns is the largest for which a direct link is done no later than the pair link."""
+    from fractions import Fraction
+    c = 1 if layout == 0 else n - 1
+    d = mwo.split_direct_bytes(S, n, layout, w_direct, w_pair)
+    assert d % 16 == 0 and 0 <= d <= S
+
+    def t_direct(x):
+        return Fraction(x) / Fraction(w_direct)
+
+    def t_pair(x):
+        return c * Fraction(S - x) / Fraction(w_pair)
+
+    best = max(x for x in range(0, S + 1, 16) if t_direct(x) <= t_pair(x)) if S <= 8192 else None
+    if best is not None:
+        assert d == best
+    assert t_direct(d) <= t_pair(d)
+    assert d + 16 > S or t_direct(d + 16) > t_pair(d + 16)
+    # the oracle's link loads, weighted by the two bandwidths, agree: the slower class decides the transfer time
+    tot = mwo.paired_allgather(np.zeros((2 * n, S), np.uint8), d, layout)[2]
+    assert Fraction(tot["direct_link_bytes"]) / Fraction(w_direct) <= Fraction(tot["pair_link_bytes"]) / Fraction(w_pair)
+    assert tot["forward_link_bytes"] <= tot["pair_link_bytes"]
+
+
+def test_split_with_equal_bandwidths_is_the_papers_split():
+    """Section 3.1: equal links give s/2 direct with MultiWrite (latency s/2w) and 3s/4 with the unicast relay (3s/4w)."""
+    for S in (1 << 20, 16 << 20, 4096, 48):
+        for n in (2, 4, 8):
+            for layout in (0, 1):
+                assert mwo.split_direct_bytes(S, n, layout, 56.0, 56.0) == mwo.balanced_direct_bytes(S, n, layout)
+    assert mwo.split_direct_bytes(1 << 20, 4, 0, 1.0, 1.0) == (1 << 20) // 2
+    assert mwo.split_direct_bytes(1 << 20, 4, 1, 1.0, 1.0) == 3 * (1 << 20) // 4
+    # degenerate inputs: a single-rank domain, or no usable bandwidth figure, sends everything direct
+    assert mwo.split_direct_bytes(4096, 1, 0, 1.0, 1.0) == 4096
+    assert mwo.split_direct_bytes(4096, 4, 0, 0.0, 1.0) == 4096
+    assert mwo.split_direct_bytes(4096, 4, 0, 1.0, -1.0) == 4096
+    # a pair link twice as fast takes two thirds of the shard with MultiWrite
+    assert mwo.split_direct_bytes(3 << 20, 4, 0, 1.0, 2.0) == 1 << 20
+
+
 def test_invalid_arguments():
     sh = np.zeros((8, 64), np.uint8)
     assert mwo.paired_allgather(sh, 80, 0)[3] == mwo.MWO_ERR_INVALID_ARG
