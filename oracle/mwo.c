@@ -350,6 +350,7 @@ typedef struct {
     int64_t inter_multiwrite_bytes; /* source -> other servers, one copy per server that has a destination  */
     int64_t inter_unicast_bytes;    /* source -> other servers, one copy per remote destination (baseline)  */
     int64_t forward_bytes;          /* relays -> destinations in their server (the relay itself excluded)   */
+    int64_t staged_rows;            /* hop rows whose next hop is not itself a destination of the token     */
     int32_t status;
     int32_t reserved;
 } mwo_relay_totals;
@@ -387,6 +388,7 @@ void mwo_relay_expand(const uint8_t *hop_buf, int64_t row_bytes, int32_t T, int3
         for (int32_t q = hop_rank_offsets[h]; q < hop_rank_offsets[h + 1]; ++q) {
             const int32_t t = hop_rank_tokens[q];
             const int remote = h / ranks_per_server != src_rank / ranks_per_server;
+            int is_dest = 0;
             ++totals->hop_rows;
             if (remote) totals->inter_multiwrite_bytes += row_bytes;
             for (int i = 0; i < Kd; ++i) {
@@ -397,6 +399,7 @@ void mwo_relay_expand(const uint8_t *hop_buf, int64_t row_bytes, int32_t T, int3
                                (int64_t)flat_dest_pos[(int64_t)t * Kd + i] * row_bytes,
                            hop_buf + (int64_t)q * row_bytes, (size_t)row_bytes);
                 ++totals->delivered_rows;
+                if (r == h) is_dest = 1;
                 if (remote) {
                     totals->inter_unicast_bytes += row_bytes;
                     if (r != h) totals->forward_bytes += row_bytes;
@@ -404,10 +407,76 @@ void mwo_relay_expand(const uint8_t *hop_buf, int64_t row_bytes, int32_t T, int3
                     totals->direct_bytes += row_bytes;
                 }
             }
+            if (!is_dest) ++totals->staged_rows;
         }
     }
     totals->status = flat_status;
     (void)T;
+}
+
+/*
+ * The same two levels with the receive buffer serving as the relay buffer (Section 6.4, memory usage: the relay's
+ * buffer is the receive buffer that exists anyway, so relaying needs no memory of its own).  A copy whose next hop h
+ * is itself a destination of the token is written by the first level straight into its final slot of region(h); the
+ * relay then forwards it from there.  Only a copy whose next hop is NOT a destination of the token (a pure relay)
+ * needs a place outside the receive regions: it goes to its row of the hop area, laid out as before (region of hop h
+ * at the first-level offset of h), whose other rows are left untouched.
+ *
+ * First level: send row j of the first-level plan (token t) to every next hop h of the token.
+ */
+static int flat_slot_of(const int32_t *flat_dest_rank, const int32_t *flat_dest_pos, int32_t t, int Kd, int32_t r)
+{
+    for (int i = 0; i < Kd; ++i)
+        if (flat_dest_rank[(int64_t)t * Kd + i] == r) return flat_dest_pos[(int64_t)t * Kd + i];
+    return -1;                                           /* r is not a destination of t */
+}
+
+void mwo_relay_first_in_place(const uint8_t *send_mw, int64_t row_bytes, int64_t hop_T_nonempty, int32_t R, int32_t K,
+                              const int32_t *hop_mw_row_token, const int32_t *hop_dest_rank, const int32_t *hop_dest_pos,
+                              const int32_t *hop_rank_offsets,
+                              const int32_t *flat_dest_rank, const int32_t *flat_dest_pos, const int32_t *flat_rank_offsets,
+                              uint8_t *hop_buf, uint8_t *recv_base, int64_t recv_stride_bytes)
+{
+    const int Kd = K < R ? K : R;
+    for (int64_t j = 0; j < hop_T_nonempty; ++j) {
+        const int32_t t = hop_mw_row_token[j];
+        for (int i = 0; i < Kd; ++i) {
+            const int32_t h = hop_dest_rank[(int64_t)t * Kd + i];
+            if (h < 0) break;
+            const int slot = flat_slot_of(flat_dest_rank, flat_dest_pos, t, Kd, h);
+            uint8_t *dst = slot >= 0
+                ? region(recv_base, recv_stride_bytes, flat_rank_offsets, h, row_bytes) + (int64_t)slot * row_bytes
+                : hop_buf + ((int64_t)hop_rank_offsets[h] + hop_dest_pos[(int64_t)t * Kd + i]) * row_bytes;
+            memcpy(dst, send_mw + j * row_bytes, (size_t)row_bytes);
+        }
+    }
+}
+
+/* Second level: every relay forwards the copy it holds (in its own region if it is a destination of the token, else
+ * in the hop area) to the other destinations of the token inside its server (Section 3.2; Section 4.1 step 5). */
+void mwo_relay_forward_in_place(const uint8_t *hop_buf, int64_t row_bytes, int32_t R, int32_t K,
+                                int32_t src_rank, int32_t ranks_per_server,
+                                const int32_t *hop_rank_offsets, const int32_t *hop_rank_tokens,
+                                const int32_t *flat_dest_rank, const int32_t *flat_dest_pos, const int32_t *flat_rank_offsets,
+                                uint8_t *recv_base, int64_t recv_stride_bytes)
+{
+    const int Kd = K < R ? K : R;
+    for (int32_t h = 0; h < R; ++h) {
+        for (int32_t q = hop_rank_offsets[h]; q < hop_rank_offsets[h + 1]; ++q) {
+            const int32_t t = hop_rank_tokens[q];
+            const int slot = flat_slot_of(flat_dest_rank, flat_dest_pos, t, Kd, h);
+            const uint8_t *held = slot >= 0
+                ? region(recv_base, recv_stride_bytes, flat_rank_offsets, h, row_bytes) + (int64_t)slot * row_bytes
+                : hop_buf + (int64_t)q * row_bytes;
+            for (int i = 0; i < Kd; ++i) {
+                const int32_t r = flat_dest_rank[(int64_t)t * Kd + i];
+                if (r < 0 || r == h || mwo_next_hop(r, src_rank, ranks_per_server) != h) continue;
+                memcpy(region(recv_base, recv_stride_bytes, flat_rank_offsets, r, row_bytes) +
+                           (int64_t)flat_dest_pos[(int64_t)t * Kd + i] * row_bytes,
+                       held, (size_t)row_bytes);
+            }
+        }
+    }
 }
 
 /*

@@ -170,7 +170,7 @@ def deliver_definition(p: Plan, x: np.ndarray, topk_ids: np.ndarray, expert_to_r
 class RelayTotals(C.Structure):
     _fields_ = [("hop_rows", C.c_int64), ("delivered_rows", C.c_int64), ("direct_bytes", C.c_int64),
                 ("inter_multiwrite_bytes", C.c_int64), ("inter_unicast_bytes", C.c_int64),
-                ("forward_bytes", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
+                ("forward_bytes", C.c_int64), ("staged_rows", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
@@ -182,9 +182,11 @@ def next_hop(r: int, src_rank: int, ranks_per_server: int) -> int:
 
 
 def relay(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: int, src_rank: int,
-          ranks_per_server: int, x: np.ndarray | None = None, recv_stride_bytes: int = 0, fill: int = 0):
+          ranks_per_server: int, x: np.ndarray | None = None, recv_stride_bytes: int = 0, fill: int = 0,
+          in_place: bool = False):
     """Two-level dispatch.  Returns (hop_plan, flat_plan, send_buf, hop_buf, recv, totals); the buffers are None
-    when no payload is given."""
+    when no payload is given.  in_place: the receive buffer serves as relay buffer (a copy whose next hop is itself a
+    destination goes straight to its final slot; only the other copies use the hop area, whose remaining rows keep `fill`)."""
     e2r = np.ascontiguousarray(expert_to_rank, dtype=np.int32)
     hop_tab = np.zeros_like(e2r)
     lib().mwo_relay_table.restype = None
@@ -200,6 +202,19 @@ def relay(topk_ids: np.ndarray, expert_to_rank: np.ndarray, R: int, row_bytes: i
         hop_buf = deliver_mw(hp, send)                       # first level: one copy per next hop
         recv = np.full(recv_bytes_needed(fp, recv_stride_bytes), fill, np.uint8)
         hop_ptr, recv_ptr = _p(hop_buf), _p(recv)
+    if in_place and x is not None:
+        hop_buf = np.full(hp.totals["total_dest"] * row_bytes, fill, np.uint8)
+        lib().mwo_relay_first_in_place.restype = None
+        lib().mwo_relay_forward_in_place.restype = None
+        lib().mwo_relay_first_in_place(_p(_bytes2d(send)), C.c_int64(row_bytes), C.c_int64(hp.totals["T_nonempty"]), C.c_int32(R),
+                                       C.c_int32(fp.K), _p(hp.mw_row_token), _p(hp.dest_rank), _p(hp.dest_pos), _p(hp.rank_offsets),
+                                       _p(fp.dest_rank), _p(fp.dest_pos), _p(fp.rank_offsets), _p(hop_buf), _p(recv),
+                                       C.c_int64(recv_stride_bytes))
+        lib().mwo_relay_forward_in_place(_p(hop_buf), C.c_int64(row_bytes), C.c_int32(R), C.c_int32(fp.K), C.c_int32(src_rank),
+                                         C.c_int32(ranks_per_server), _p(hp.rank_offsets), _p(hp.rank_tokens),
+                                         _p(fp.dest_rank), _p(fp.dest_pos), _p(fp.rank_offsets), _p(recv),
+                                         C.c_int64(recv_stride_bytes))
+        recv_ptr = C.c_void_p(0)                              # the accounting below is the same; nothing more to write
     tot = RelayTotals()
     lib().mwo_relay_expand(hop_ptr, C.c_int64(row_bytes), C.c_int32(fp.T), C.c_int32(R), C.c_int32(fp.K),
                            C.c_int32(src_rank), C.c_int32(ranks_per_server), _p(hp.rank_offsets), _p(hp.rank_tokens),

@@ -35,6 +35,16 @@ MUTATIONS = {
     "combine truncates instead of rounding": ("double q = nearbyint(ldexp(a, 7 - ex));", "double q = floor(ldexp(a, 7 - ex));"),
     "combine reads the wrong slot": ("(int64_t)dest_pos[(int64_t)t * Kd + i] * row_bytes;\n                const double w",
                                      "(int64_t)(dest_pos[(int64_t)t * Kd + i] > 0 ? dest_pos[(int64_t)t * Kd + i] - 1 : 0) * row_bytes;\n                const double w"),
+    "relay buffer in the receive buffer: the relay forwards a copy to itself again": (
+        "if (r < 0 || r == h || mwo_next_hop(r, src_rank, ranks_per_server) != h) continue;\n                memcpy(region(recv_base, recv_stride_bytes, flat_rank_offsets, r, row_bytes) +\n                           (int64_t)flat_dest_pos[(int64_t)t * Kd + i] * row_bytes,\n                       held,",
+        "if (r < 0 || mwo_next_hop(r, src_rank, ranks_per_server) != h) continue;\n                memcpy(region(recv_base, recv_stride_bytes, flat_rank_offsets, r, row_bytes) +\n                           (int64_t)(flat_dest_pos[(int64_t)t * Kd + i] + (r == h)) * row_bytes,\n                       held,"),
+    "relay buffer in the receive buffer: forwarding always reads the hop area": (
+        "const uint8_t *held = slot >= 0\n                ? region(recv_base, recv_stride_bytes, flat_rank_offsets, h, row_bytes) + (int64_t)slot * row_bytes\n                : hop_buf + (int64_t)q * row_bytes;",
+        "const uint8_t *held = hop_buf + (int64_t)q * row_bytes;"),
+    "relay buffer in the receive buffer: a pure relay's copy lands in the wrong hop row": (
+        ": hop_buf + ((int64_t)hop_rank_offsets[h] + hop_dest_pos[(int64_t)t * Kd + i]) * row_bytes;",
+        ": hop_buf + ((int64_t)hop_rank_offsets[h] + (hop_dest_pos[(int64_t)t * Kd + i] > 0 ? hop_dest_pos[(int64_t)t * Kd + i] - 1 : 0)) * row_bytes;"),
+    "staged rows count every hop row": ("if (!is_dest) ++totals->staged_rows;", "++totals->staged_rows;"),
     "relay sends to rank 0 of the remote server": ("return (r / ranks_per_server) * ranks_per_server + src_rank % ranks_per_server;",
                                                    "return (r / ranks_per_server) * ranks_per_server;"),
     "paired allgather forwards the direct segment": ("relay_buf + ((int64_t)partner * copies + c) * relay_bytes, (size_t)relay_bytes);\n            ++k;",

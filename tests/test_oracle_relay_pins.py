@@ -31,7 +31,9 @@ def brute_relay(ids, e2r, R, P, src, rows):
     forward = sum(1 for d in dest for r in d if server(r) != server(src) and r != relay_of(server(r)))
     recv = [[rows[t] for t in range(T) if r in dest[t]] for r in range(R)]
     hop_recv = [[rows[t] for t in range(T) if h in hops[t]] for h in range(R)]
-    return dict(hop_rows=hop_rows, direct=direct, inter_uc=inter_uc, inter_mw=inter_mw, forward=forward, recv=recv,
+    # with the receive buffer as relay buffer only a pure relay (a next hop that is not a destination) stages its copy
+    staged = [[rows[t] if h not in dest[t] else None for t in range(T) if h in hops[t]] for h in range(R)]
+    return dict(staged=staged, hop_rows=hop_rows, direct=direct, inter_uc=inter_uc, inter_mw=inter_mw, forward=forward, recv=recv,
                 hop_recv=hop_recv, delivered=sum(len(d) for d in dest))
 
 
@@ -56,6 +58,16 @@ def test_relay_brute_force(seed, R, P, src, E, K):
     assert np.array_equal(recv, mwo.deliver_definition(fp, inp.x, inp.topk_ids, inp.expert_to_rank))
     # each row is packed once per group of identical next-hop set
     assert len(send) == hp.totals["T_nonempty"]
+    assert tot["staged_rows"] == sum(1 for rows in bf["staged"] for r in rows if r is not None)
+    # Section 6.4: with the receive buffer as the relay buffer the regions come out the same, the accounting too, and
+    # only the copies held by pure relays appear in the hop area
+    for stride in (0, (int(np.diff(fp.rank_offsets).max()) + 1) * B):
+        _, _, send2, hop2, recv2, tot2 = mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x, stride, 0xEE, in_place=True)
+        _, _, _, _, recv_ref, _ = mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x, stride, 0xEE)
+        assert tot2 == tot and np.array_equal(send2, send)
+        assert np.array_equal(recv2, recv_ref)
+        want_hop = b"".join(b"".join(r if r is not None else b"\xEE" * B for r in rows) for rows in bf["staged"])
+        assert hop2.tobytes() == want_hop
 
 
 def test_paper_example_four_local_four_remote():
@@ -68,6 +80,7 @@ def test_paper_example_four_local_four_remote():
     assert tot["inter_unicast_bytes"] // 16 == c["relay_example_remote_copies_unicast"]
     assert tot["inter_multiwrite_bytes"] // 16 == c["relay_example_remote_copies_multiwrite"]
     assert tot["direct_bytes"] // 16 == 4 and tot["forward_bytes"] // 16 == 4
+    assert tot["staged_rows"] == 1                          # NPU8 relays for 9..12 without being a destination itself
     hops = [int(r) for r in hp.dest_rank[0] if r >= 0]
     assert hops == [1, 2, 3, 4, c["relay_example_relay_rank"]]
     assert mwo.next_hop(12, src, P) == c["relay_example_relay_rank"] and mwo.next_hop(3, src, P) == 3
