@@ -420,11 +420,14 @@ MW_API int mw_dispatch_host(mw_ctx *ctx, const int32_t *topk_ids_host, const int
  * The R ranks form servers of ranks_per_server consecutive ranks; the source is rank cfg.src_rank
  * (it must be a member of the domain).  A destination in the source's own server is its own next
  * hop; every other server's next hop is the rank with the source's index inside that server (Section 3.2),
- * which forwards the row to the destinations inside its server.  First level:
- * an ordinary MultiWrite plan / pack / deliver over next-hop sets into a hop area (one region per
- * next hop).  Second level: every row of the hop area is written to the final destinations whose
- * next hop it is, at the slots of the flat plan, so the final receive regions are byte-identical
- * to those of mw_dispatch.  Byte accounting is per link class.
+ * which forwards the row to the destinations inside its server.  First level: an ordinary MultiWrite plan over
+ * next-hop sets; every hidden row is packed once per group of identical next-hop set and one copy goes to each
+ * next hop.  The receive buffer is the relay buffer (Section 6.4: relaying needs no memory of its own): a copy
+ * whose next hop is itself a destination of the token lands in its final slot of that rank's receive region;
+ * only a copy held by a pure relay (a next hop that is not a destination) is staged in the hop area.  Second
+ * level: every relay forwards the copy it holds to the token's other destinations inside its server, at the
+ * slots of the flat plan, so the final receive regions are byte-identical to those of mw_dispatch.  Byte
+ * accounting is per link class.
  * ------------------------------------------------------------------------------------------------ */
 typedef struct mw_relay mw_relay;   /* opaque: two plans (next hops, final destinations) and the second-level descriptors */
 
@@ -435,6 +438,8 @@ typedef struct {
     int64_t inter_multiwrite_bytes; /* source -> other servers: one copy per server holding a destination    */
     int64_t inter_unicast_bytes;    /* the same traffic with one copy per remote destination (the baseline)  */
     int64_t forward_bytes;          /* relays -> destinations in their server (the relay itself excluded)    */
+    int64_t staged_rows;            /* hop rows whose next hop is not a destination of the token: the only   */
+                                    /* copies that need room outside the receive regions                     */
     int32_t status;                 /* MW_OK or the first device-side MW_ERR_* of either plan or the dispatch */
     int32_t reserved;
 } mw_relay_totals;
@@ -443,18 +448,23 @@ typedef struct {
 MW_API int mw_relay_create(mw_relay **out, const mw_config *cfg, int32_t ranks_per_server);
 MW_API int mw_relay_destroy(mw_relay *relay);
 
-/* Plans both levels (inputs as for mw_plan).  Asynchronous on `stream`. */
+/* After MW_ERR_TIMEOUT in mw_relay_totals.status: mw_reset for both inner contexts.  Synchronous. */
+MW_API int mw_relay_reset(mw_relay *relay);
+
+/* Plans both levels (inputs as for mw_plan; the two plans run concurrently, one of them on a stream the library
+ * owns, and `stream` waits for both).  Asynchronous on `stream`. */
 MW_API int mw_relay_plan(mw_relay *relay, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, void *stream);
 
 /* Waits for `stream`, then copies the per-link accounting of the latest mw_relay_plan / mw_relay_dispatch. */
 MW_API int mw_relay_get_totals(mw_relay *relay, mw_relay_totals *host_out, void *stream);
 
 /*
- * Pack (each row once per group of identical next-hop set), first-level deliver into the hop area,
- * second-level expansion into the final receive regions.
+ * Pack (each row once per group of identical next-hop set) and first-level deliver in one pass, then the relays'
+ * forwarding.
  *   send_buf   device, send_capacity_rows rows
- *   hop_buf    device, compact hop area of hop_capacity_rows rows (region of next hop h starts at the
- *              first-level rank offset of h)
+ *   hop_buf    device, hop area of hop_capacity_rows rows, laid out per next hop (region of next hop h starts at
+ *              the first-level rank offset of h, one row per token that passes through h); only the rows of copies
+ *              held by pure relays are written (mw_relay_totals.staged_rows of them), the others are left untouched
  *   recv_base, recv_stride_bytes, recv_capacity_rows   as for mw_deliver
  */
 MW_API int mw_relay_dispatch(mw_relay *relay, const void *x, void *send_buf, int64_t send_capacity_rows, void *hop_buf,

@@ -33,7 +33,7 @@ MW_TEST_SKEW_LOOKBACK = 0x1
 MW_TEST_SKEW_BARRIER = 0x2
 MW_TEST_SKEW_BULK_LOAD = 0x4
 
-RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
+RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_reset", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")
 INT_EXPORTS = ("mw_create", "mw_destroy", "mw_reset", "mw_plan", "mw_plan_prefetch", "mw_plan_next", "mw_plan_swap",
                "mw_get_plan_view", "mw_get_totals", "mw_pack", "mw_deliver", "mw_deliver_ptrs", "mw_dispatch", "mw_plan_dispatch",
@@ -61,7 +61,7 @@ class mw_totals(C.Structure):
 class mw_relay_totals(C.Structure):
     _fields_ = [("hop_rows", C.c_int64), ("delivered_rows", C.c_int64), ("direct_bytes", C.c_int64),
                 ("inter_multiwrite_bytes", C.c_int64), ("inter_unicast_bytes", C.c_int64),
-                ("forward_bytes", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
+                ("forward_bytes", C.c_int64), ("staged_rows", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
@@ -143,6 +143,7 @@ def lib():
         L.mw_kernel_launches.restype = C.c_int64
         L.mw_relay_create.argtypes = [C.POINTER(vp), C.POINTER(mw_config), i32]
         L.mw_relay_destroy.argtypes = [vp]
+        L.mw_relay_reset.argtypes = [vp]
         L.mw_relay_plan.argtypes = [vp, vp, vp, i32, vp]
         L.mw_relay_get_totals.argtypes = [vp, C.POINTER(mw_relay_totals), vp]
         L.mw_relay_dispatch.argtypes = [vp, vp, vp, i64, vp, i64, vp, i64, i64, vp]
@@ -246,6 +247,8 @@ class Context:
         return self
 
     def close(self):
+        if C is None:                      # interpreter shutdown: the module globals are already gone
+            return
         if self._h and getattr(self, "_owned", True):
             lib().mw_destroy(self._h)
         self._h = C.c_void_p()
@@ -466,6 +469,8 @@ class Relay:
         self.R, self.Kd, self.row_bytes = R, min(K, R), row_bytes
 
     def close(self):
+        if C is None:
+            return
         if self._h:
             lib().mw_relay_destroy(self._h)
             self._h = C.c_void_p()
@@ -486,6 +491,12 @@ class Relay:
         for ctx in (self.hop, self.flat) if rc == MW_OK else ():
             if ctx.view is None:
                 ctx.view = _view_of(ctx)
+        return rc
+
+    def mw_relay_reset(self) -> int:
+        rc = lib().mw_relay_reset(self._h)
+        if rc != MW_OK:
+            raise MwError(rc, "mw_relay_reset")
         return rc
 
     def mw_relay_get_totals(self, stream=None) -> dict:

@@ -185,6 +185,18 @@ int order_after_side_plans(mw_ctx *ctx, cudaStream_t st)
 
 }  // namespace
 
+int mw_plan_on_side_stream(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t user)
+{
+    if (cudaEventRecord(ctx->ev_submitted, user) != cudaSuccess ||
+        cudaStreamWaitEvent(ctx->plan_stream, ctx->ev_submitted, 0) != cudaSuccess)
+        return MW_ERR_CUDA;
+    const int rc = mw_plan_launch(ctx, topk_ids, expert_to_rank, T, nullptr, ctx->plan_stream);
+    if (rc != MW_OK) return rc;
+    if (cudaEventRecord(ctx->ev_planned, ctx->plan_stream) != cudaSuccess) return MW_ERR_CUDA;
+    ctx->plans_on_side_stream = 1;
+    return MW_OK;
+}
+
 extern "C" {
 
 int mw_create(mw_ctx **out, const mw_config *cfg)

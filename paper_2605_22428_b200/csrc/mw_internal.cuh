@@ -91,12 +91,20 @@ struct mw_ctx {
     uint32_t test_skew;     // MW_TEST_SKEW_* bits applied to the next launch (mw_test_skew_waits)
     int poisoned;           // a wait gave up: host counters and device scratch may be out of step until mw_reset
     uint32_t gm_epoch;      // epoch of the plan the group-major arrays were made from (0: none)
+    int32_t relay_src, relay_P;   // relay_P > 0: plans map every rank to its next hop as seen from rank relay_src (servers of relay_P ranks)
     int64_t launches;
     // host staging (MW_FLAG_HOST_STAGING)
     int32_t *st_ids, *st_e2r;
     uint8_t *st_x, *st_send, *st_recv;
     int64_t st_recv_rows;
 };
+
+// Next hop of a write from rank `src` to rank r when ranks form servers of P consecutive ranks: a destination in
+// the source's own server is reached directly, any other through the rank with the source's index in its server.
+__host__ __device__ inline int mw_next_hop(int r, int src, int P)
+{
+    return (r / P == src / P) ? r : (r / P) * P + src % P;
+}
 
 // Calls that use the device refuse a context in which a device-side wait has given up (see mw_reset).
 #define MW_REFUSE_IF_POISONED(ctx) do { if ((ctx)->poisoned) return MW_ERR_TIMEOUT; } while (0)
@@ -158,6 +166,9 @@ __device__ __forceinline__ uint64_t bitmap_word(const uint64_t (&m)[WT], int w)
 // `rows` (may be null): the hidden rows [T, row_bytes] the pack step will read; they are brought into L2 while the plan runs
 int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, const void *rows, cudaStream_t st);
 int mw_plan_smem_setup(mw_ctx *ctx);
+// Plans into the current slot on the context's own planning stream, ordered after everything submitted to `user`
+// so far; the caller makes its stream wait for ctx->ev_planned before it uses the plan (mw_api.cu).
+int mw_plan_on_side_stream(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T, cudaStream_t user);
 
 // ---- single-launch small-batch path (mw_small.cu) ----
 bool mw_small_applies(const mw_ctx *ctx, int32_t T, int layout);

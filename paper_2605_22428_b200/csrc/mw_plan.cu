@@ -32,6 +32,7 @@ constexpr unsigned kFlagAgg = 1u, kFlagPrefix = 2u;
 struct PlanArgs {
     const int32_t *ids, *e2r;
     int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask, Tm;
+    int relay_src, relay_P;   // relay_P > 0: a rank stands for its next hop as seen from relay_src (first level of a relayed dispatch)
     int64_t row_bytes;
     uint32_t epoch, ticket_base, bar_base;
     uint32_t wait_epoch;      // epoch a look-back expects in its predecessors' records (= epoch, unless a test skews it)
@@ -116,8 +117,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_mask(PlanArgs a)
                 const int id = my[k];
                 if (id == -1) continue;                               // padding slot
                 if (id < 0 || id >= a.E) { bad |= (w == 0); continue; }
-                const int r = a.e2r[id];
+                int r = a.e2r[id];
                 if (r < 0 || r >= a.R) { bad |= (w == 0); continue; }
+                if (a.relay_P > 0) r = mw_next_hop(r, a.relay_src, a.relay_P);    // one copy per distinct next hop (Section 4.1)
                 valid += (w == 0);
                 if ((r >> 6) == w) word |= 1ull << (r & 63);          // OR = per-rank dedup
             }
@@ -546,6 +548,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                     const bool ok = r[j] >= 0 && r[j] < a.R;
                     bad |= (id[j] >= 0 && id[j] < a.E && !ok);
                     valid += ok;
+                    if (a.relay_P > 0 && ok) r[j] = mw_next_hop(r[j], a.relay_src, a.relay_P);   // one copy per distinct next hop (Section 4.1)
                     const uint64_t rank_bit = ok ? 1ull << (r[j] & 63) : 0ull;
 #pragma unroll
                     for (int w = 0; w < WT; ++w) m[w] |= rank_bit & equal_mask64(r[j] >> 6, w);   // OR = per-rank dedup
@@ -844,6 +847,7 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.ids = topk_ids; a.e2r = expert_to_rank;
     a.T = T; a.K = ctx->cfg.K; a.E = ctx->cfg.E; a.R = ctx->cfg.R; a.W = ctx->W; a.Kd = ctx->Kd;
     a.src_rank = ctx->cfg.src_rank;
+    a.relay_src = ctx->relay_src; a.relay_P = ctx->relay_P;
     a.ntiles = T > 0 ? (T + MW_TILE - 1) / MW_TILE : 1;
     a.NC = ctx->NC; a.hs_mask = ctx->HS - 1; a.Tm = ctx->cfg.max_tokens;
     a.row_bytes = ctx->cfg.row_bytes;

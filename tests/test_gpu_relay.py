@@ -16,11 +16,14 @@ def run_relay(inp, P, src, strided=False, flags=0, max_tokens=None):
     torch = torch_mod()
     s = inp.shape
     T, B, R = inp.T, s.row_bytes, s.R
-    hp, fp, want_send, want_hop, _, want_tot = mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x)
+    # the receive buffer is the relay buffer: only copies held by pure relays are staged in the hop area
+    hp, fp, want_send, want_hop, _, want_tot = mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x, 0, SENTINEL, in_place=True)
     counts = np.diff(fp.rank_offsets)
     cap = int(counts.max()) + 1 if strided else fp.totals["total_dest"]
     stride = cap * B if strided else 0
-    _, _, _, _, want_recv, _ = mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x, stride, SENTINEL)
+    _, _, _, _, want_recv, _ = mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x, stride, SENTINEL, in_place=True)
+    # the relayed route must end in the regions of the flat dispatch (the definitional two-buffer form agrees)
+    assert np.array_equal(want_recv, mwo.relay(inp.topk_ids, inp.expert_to_rank, R, B, src, P, inp.x, stride, SENTINEL)[4])
     ids_d = torch.from_numpy(inp.topk_ids).cuda()
     e2r_d = torch.from_numpy(inp.expert_to_rank).cuda()
     x_d = torch.from_numpy(inp.x.view(np.int16)).cuda()
@@ -46,7 +49,8 @@ def run_relay(inp, P, src, strided=False, flags=0, max_tokens=None):
 
 
 @pytest.mark.parametrize("R,P,src,E,K,T", [(16, 8, 0, 64, 8, 1500), (8, 4, 5, 16, 3, 700), (12, 3, 7, 24, 4, 300),
-                                           (6, 6, 2, 12, 3, 257), (5, 1, 3, 10, 2, 64), (128, 8, 77, 256, 8, 2000)])
+                                           (6, 6, 2, 12, 3, 257), (5, 1, 3, 10, 2, 64), (128, 8, 77, 256, 8, 2000),
+                                           (64, 8, 13, 128, 12, 900), (64, 4, 62, 128, 20, 515)])   # 12 and 20 destinations per token
 def test_relay_parity_random(R, P, src, E, K, T):
     inp = wl.make_random_dispatch(R + T, T=T, K=K, E=E, R=R, H=40, pad_fraction=0.1, contiguous_map=(E % R == 0))
     run_relay(inp, P, src)
@@ -89,7 +93,7 @@ def test_relay_errors():
         mw.Relay(16, 32, 4, 64, 32, 0, 5)                  # ranks per server must divide R
     buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
     ids = torch.zeros((16, 4), dtype=torch.int32, device="cuda")
-    e2r = torch.zeros(32, dtype=torch.int32, device="cuda")
+    e2r = torch.full((32,), 9, dtype=torch.int32, device="cuda")   # every token goes to rank 9: rank 8 relays without being a destination
     with mw.Relay(16, 32, 4, 64, 32, 0, 8) as relay:
         assert relay.mw_relay_dispatch(buf, buf, 64, buf, 64, buf, 0, 64, check=False) == mw.MW_ERR_NO_PLAN
         assert relay.mw_relay_plan(ids, e2r, 65, check=False) == mw.MW_ERR_INVALID_ARG
@@ -98,5 +102,6 @@ def test_relay_errors():
         # hop area one row short: reported, nothing written past it
         hop = Guarded(15 * 32)
         relay.mw_relay_dispatch(buf, buf, 64, hop.ptr(), 15, buf, 0, 64)
-        assert relay.mw_relay_get_totals()["status"] == mw.MW_ERR_CAPACITY
+        tot = relay.mw_relay_get_totals()
+        assert tot["status"] == mw.MW_ERR_CAPACITY and tot["staged_rows"] == 16
         assert hop.guards_intact()
