@@ -354,7 +354,7 @@ MW_API int mw_deliver_group_major(mw_ctx *ctx, const void *send_buf, void *recv_
  *     expert_token    device int32 [T * K]  per expert in id order, its tokens ascending; -1 beyond the total
  *     expert_slot     device int32 [T * K]  slot of that token in the region of the expert's rank (token-major
  *                                           order, i.e. the order mw_deliver and mw_dispatch produce)
- * MW_ERR_CAPACITY when E is too large for the kernel's shared-memory bit matrix (32 bytes per expert) or for
+ * MW_ERR_CAPACITY when E is too large for the kernel's shared memory (36 bytes per expert) or for
  * the per-tile count table (max_tokens / 256 x E entries, at most 256 MB).
  */
 MW_API int mw_expert_index(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t *expert_offsets,

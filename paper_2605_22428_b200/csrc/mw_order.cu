@@ -10,8 +10,10 @@
 // of its tokens and of their slots in the region of the expert's rank.  A per-expert exclusive prefix sum over
 // tokens, done as a bit matrix (expert x token of the tile) plus per-tile counts.
 //
-// Both are small integer passes over the plan (kilobytes to a few megabytes); they run as a few short kernels
-// of one block per 256 groups / tokens and are bound by launch and memory latency, not by bandwidth.
+// Both are small integer passes over the plan (kilobytes to a few megabytes), bound by launch and memory latency,
+// not by bandwidth, so each runs as two short kernels of one block per 256 groups / tokens: per-tile counts, then
+// everything else, every block summing the counts of the tiles before it by itself (up to 32 tiles; beyond that a
+// scan kernel sits between the two).
 #include <string.h>
 
 #include "mw_internal.cuh"
@@ -45,11 +47,12 @@ __global__ void __launch_bounds__(kTile) k_gm_sum(GmArgs a)
     for (int i = threadIdx.x; i < n * a.W; i += kTile) mask[i] = a.d.group_mask[(size_t)g0 * a.W + i];
     if (threadIdx.x < n) size[threadIdx.x] = a.d.group_offsets[g0 + threadIdx.x + 1] - a.d.group_offsets[g0 + threadIdx.x];
     __syncthreads();
-    // one warp per rank; lane l covers groups [8 l, 8 l + 8) of the tile
+    // one warp per rank; lane l covers groups l, l + 32, ... of the tile (neighbouring lanes read neighbouring bitmaps:
+    // with eight consecutive groups per lane the shared-memory reads of a warp fell into two banks)
     const int lane = threadIdx.x & 31;
     for (int r = threadIdx.x >> 5; r < a.R; r += kTile / 32) {
         int sum = 0;
-        for (int j = lane * 8; j < min(lane * 8 + 8, n); ++j)
+        for (int j = lane; j < n; j += 32)
             if (bit_of(mask + (size_t)j * a.W, r)) sum += size[j];
         sum = __reduce_add_sync(0xffffffffu, sum);
         if (lane == 0) a.d.gm_tile_sum[(size_t)blockIdx.x * a.R + r] = sum;
@@ -69,64 +72,102 @@ __global__ void __launch_bounds__(kTile) k_gm_scan(GmArgs a)
     }
 }
 
-// Per tile: the warp of rank r walks the tile's groups in order and hands every group that contains r its block.
+constexpr int kFuseTiles = 32;     // up to this many tiles every block adds up the earlier tiles' counts itself
+
+// Per tile of 256 groups: the warp of rank r walks the tile's groups in order and hands every group that contains r
+// its block of the region; then the block's threads take the send rows of those groups (they are consecutive) and
+// give every member token its slots, per token and per send row (plane layout, for the deliver kernel).
+// SCANNED: gm_tile_sum already holds the exclusive prefix over tiles (k_gm_scan ran); else the raw per-tile sums.
+// The block with index b also marks the tokens [256 b, 256 b + 256) that have no destination.
+template <bool SCANNED>
 __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
 {
     extern __shared__ uint64_t sm64[];
     uint64_t *mask = sm64;
     int *size = (int *)(mask + (size_t)kTile * a.W);
+    int *before_s = size + kTile;                         // [R]
+    __shared__ int gstart[kTile + 1];
     if (a.d.totals->status == MW_ERR_TIMEOUT) return;
+    {   // tokens without destinations belong to no group: their slots are -1
+        const int t = blockIdx.x * kTile + threadIdx.x;
+        if (t < a.T && a.d.token_group[t] < 0)
+            for (int i = 0; i < a.Kd; ++i) a.d.dest_pos_gm[(size_t)t * a.Kd + i] = -1;
+    }
     const int G = (int)a.d.totals->G;
     const int g0 = blockIdx.x * kTile;
     const int n = min(kTile, G - g0);
     if (n <= 0) return;
     for (int i = threadIdx.x; i < n * a.W; i += kTile) mask[i] = a.d.group_mask[(size_t)g0 * a.W + i];
+    if (threadIdx.x < n) gstart[threadIdx.x] = a.d.group_offsets[g0 + threadIdx.x];
+    if (threadIdx.x == 0) gstart[n] = a.d.group_offsets[g0 + n];
+    __syncthreads();
     if (threadIdx.x < n) {
-        size[threadIdx.x] = a.d.group_offsets[g0 + threadIdx.x + 1] - a.d.group_offsets[g0 + threadIdx.x];
+        size[threadIdx.x] = gstart[threadIdx.x + 1] - gstart[threadIdx.x];
         for (int i = 0; i < a.Kd; ++i) {
             a.d.gm_rank[(size_t)(g0 + threadIdx.x) * a.Kd + i] = -1;
             a.d.gm_offset[(size_t)(g0 + threadIdx.x) * a.Kd + i] = -1;
         }
     }
+    // rows the earlier tiles put into every region: all ranks at once (independent, coalesced loads), not rank by rank
+    for (int r = threadIdx.x; r < a.R; r += kTile) {
+        int before = 0;
+        if (SCANNED) before = a.d.gm_tile_sum[(size_t)blockIdx.x * a.R + r];
+        else
+            for (int t = 0; t < (int)blockIdx.x; ++t) before += a.d.gm_tile_sum[(size_t)t * a.R + r];
+        before_s[r] = before;
+    }
     __syncthreads();
-    // one warp per rank; lane l covers groups [8 l, 8 l + 8): an exclusive scan over the lanes gives each its start
+    // one warp per rank, 32 groups of the tile per round (lane l takes group 32 k + l, so neighbouring lanes read
+    // neighbouring bitmaps): an exclusive scan over the lanes gives each group that contains r the start of its block
     const int lane = threadIdx.x & 31;
     for (int r = threadIdx.x >> 5; r < a.R; r += kTile / 32) {
-        int sum = 0;
-        for (int j = lane * 8; j < min(lane * 8 + 8, n); ++j)
-            if (bit_of(mask + (size_t)j * a.W, r)) sum += size[j];
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-        int run = a.d.gm_tile_sum[(size_t)blockIdx.x * a.R + r] + incl - sum;
-        for (int j = lane * 8; j < min(lane * 8 + 8, n); ++j) {
+        int run = before_s[r];
+        for (int j0 = 0; j0 < n; j0 += 32) {
+            const int j = j0 + lane;
             const uint64_t *m = mask + (size_t)j * a.W;
-            if (!bit_of(m, r)) continue;
-            int i = __popcll(m[r >> 6] & ((1ull << (r & 63)) - 1));      // index of r among the group's destinations
-            for (int w = 0; w < (r >> 6); ++w) i += __popcll(m[w]);
-            a.d.gm_rank[(size_t)(g0 + j) * a.Kd + i] = r;
-            a.d.gm_offset[(size_t)(g0 + j) * a.Kd + i] = run;
-            run += size[j];
+            const bool has = j < n && bit_of(m, r);
+            const int mine = has ? size[j] : 0;
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+            if (has) {
+                int i = __popcll(m[r >> 6] & ((1ull << (r & 63)) - 1));  // index of r among the group's destinations
+                for (int w = 0; w < (r >> 6); ++w) i += __popcll(m[w]);
+                a.d.gm_rank[(size_t)(g0 + j) * a.Kd + i] = r;
+                a.d.gm_offset[(size_t)(g0 + j) * a.Kd + i] = run + incl - mine;
+            }
+            run += __shfl_sync(0xffffffffu, incl, 31);
         }
     }
-}
-
-// Per token: its slots in group-major order, and the same per send row in plane layout for the deliver kernel.
-__global__ void __launch_bounds__(kTile) k_gm_tokens(GmArgs a)
-{
-    if (a.d.totals->status == MW_ERR_TIMEOUT) return;
-    const int t = blockIdx.x * kTile + threadIdx.x;
-    if (t >= a.T) return;
-    const int g = a.d.token_group[t];
-    const int row = a.d.token_mw_row[t];
-    const int within = g >= 0 ? row - a.d.group_offsets[g] : 0;
-    for (int i = 0; i < a.Kd; ++i) {
-        const int r = g >= 0 ? a.d.gm_rank[(size_t)g * a.Kd + i] : -1;
-        const int pos = r >= 0 ? a.d.gm_offset[(size_t)g * a.Kd + i] + within : -1;
-        a.d.dest_pos_gm[(size_t)t * a.Kd + i] = pos;
-        if (g >= 0) {
-            a.d.row_dest_pos_gm[(size_t)i * a.Tm + row] = pos;
-            a.d.row_dest_flat_gm[(size_t)i * a.Tm + row] = r >= 0 ? a.d.rank_offsets[r] + pos : -1;
+    __syncthreads();                                      // the tile's gm_rank / gm_offset rows are complete (and visible to the block)
+    // member tokens: send rows [gstart[0], gstart[n]) belong to the tile's groups, in group order
+    for (int row = gstart[0] + threadIdx.x; row < gstart[n]; row += kTile) {
+        int lo = 0, hi = n;                               // group of the row: the last j with gstart[j] <= row
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (gstart[mid] <= row) lo = mid; else hi = mid;
+        }
+        const int g = g0 + lo, within = row - gstart[lo];
+        const int t = a.d.mw_row_token[row];
+        // eight destinations at a time: all loads first, then the stores (a store in between would hold the next loads back,
+        // since the compiler must assume that the arrays overlap)
+        for (int i0 = 0; i0 < a.Kd; i0 += 8) {
+            int r[8], pos[8], region[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                r[u] = i0 + u < a.Kd ? a.d.gm_rank[(size_t)g * a.Kd + i0 + u] : -1;
+                pos[u] = i0 + u < a.Kd ? a.d.gm_offset[(size_t)g * a.Kd + i0 + u] : -1;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) region[u] = r[u] >= 0 ? a.d.rank_offsets[r[u]] : 0;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (i0 + u >= a.Kd) break;
+                const int p = r[u] >= 0 ? pos[u] + within : -1;
+                a.d.dest_pos_gm[(size_t)t * a.Kd + i0 + u] = p;
+                a.d.row_dest_pos_gm[(size_t)(i0 + u) * a.Tm + row] = p;
+                a.d.row_dest_flat_gm[(size_t)(i0 + u) * a.Tm + row] = r[u] >= 0 ? region[u] + p : -1;
+            }
         }
     }
 }
@@ -145,12 +186,15 @@ __device__ __forceinline__ void expert_bits(const ExArgs &a, uint32_t *bits, int
     for (int i = threadIdx.x; i < a.E * 8; i += kTile) bits[i] = 0;
     __syncthreads();
     if (t < a.T) {
-        for (int k = 0; k < a.K; ++k) {
-            const int e = a.ids[(size_t)t * a.K + k];
-            if (e < 0 || e >= a.E) continue;
-            const int r = a.e2r[e];
-            if (r < 0 || r >= a.R) continue;
-            atomicOr(bits + (size_t)e * 8 + (threadIdx.x >> 5), 1u << (threadIdx.x & 31));
+        for (int k0 = 0; k0 < a.K; k0 += 8) {                  // eight independent loads at a time, twice
+            int e[8], r[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) e[u] = k0 + u < a.K ? a.ids[(size_t)t * a.K + k0 + u] : -1;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) r[u] = (e[u] >= 0 && e[u] < a.E) ? a.e2r[e[u]] : -1;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (r[u] >= 0 && r[u] < a.R) atomicOr(bits + (size_t)e[u] * 8 + (threadIdx.x >> 5), 1u << (threadIdx.x & 31));
         }
     }
     __syncthreads();
@@ -201,39 +245,100 @@ __global__ void __launch_bounds__(1024) k_ex_scan(ExArgs a)
     if (threadIdx.x == 0) a.offsets[a.E] = carry_s;
 }
 
+// FUSED: ex_tile_cnt holds the raw per-tile counts; every block adds up the tiles before it and scans the experts
+// itself (block 0 also writes expert_offsets).  Otherwise k_ex_scan has already done both.
+template <bool FUSED>
 __global__ void __launch_bounds__(kTile) k_ex_fill(ExArgs a)
 {
     extern __shared__ uint32_t sm32[];
+    __shared__ int warp_tot[kTile / 32];
+    __shared__ int carry_s;
+    int *start = (int *)(sm32 + (size_t)a.E * 8);          // [E] (FUSED) first list position of this tile's tokens per expert
     const int t = blockIdx.x * kTile + threadIdx.x;
     expert_bits(a, sm32, t);
-    const int P = a.offsets[a.E];
+    int P;
+    if (FUSED) {
+        if (threadIdx.x == 0) carry_s = 0;
+        __syncthreads();
+        for (int e0 = 0; e0 < a.E; e0 += kTile) {
+            const int e = e0 + threadIdx.x;
+            int total = 0, before = 0;
+            if (e < a.E)
+                for (int b = 0; b < a.tiles; ++b) {
+                    const int v = a.d.ex_tile_cnt[(size_t)b * a.E + e];
+                    if (b < (int)blockIdx.x) before += v;
+                    total += v;
+                }
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            int incl = total;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += n; }
+            if (lane == 31) warp_tot[warp] = incl;
+            __syncthreads();
+            int excl = carry_s + incl - total, all = 0;
+            for (int w = 0; w < kTile / 32; ++w) { if (w < warp) excl += warp_tot[w]; all += warp_tot[w]; }
+            if (e < a.E) {
+                start[e] = excl + before;
+                if (blockIdx.x == 0) a.offsets[e] = excl;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) carry_s += all;
+            __syncthreads();
+        }
+        P = carry_s;
+        if (blockIdx.x == 0 && threadIdx.x == 0) a.offsets[a.E] = P;
+    } else {
+        P = a.offsets[a.E];
+    }
     // tails: every index of the two lists at or beyond P is covered by some thread of the grid
     for (int64_t i = (int64_t)blockIdx.x * kTile + threadIdx.x; i < (int64_t)a.T * a.K; i += (int64_t)gridDim.x * kTile)
         if (i >= P) { a.token[i] = -1; a.slot[i] = -1; }
     if (t >= a.T) return;
     const int warp = threadIdx.x >> 5;
     const uint32_t below = (1u << (threadIdx.x & 31)) - 1;
-    for (int k = 0; k < a.K; ++k) {
-        const int e = a.ids[(size_t)t * a.K + k];
-        if (e < 0 || e >= a.E) continue;
-        const int r = a.e2r[e];
-        if (r < 0 || r >= a.R) continue;
-        bool first = true;                                     // an expert named twice by a token counts once
-        for (int j = 0; j < k; ++j) first &= (a.ids[(size_t)t * a.K + j] != e);
-        if (!first) continue;
-        int pos = a.offsets[e] + a.d.ex_tile_cnt[(size_t)blockIdx.x * a.E + e];
-        for (int w = 0; w < warp; ++w) pos += __popc(sm32[(size_t)e * 8 + w]);
-        pos += __popc(sm32[(size_t)e * 8 + warp] & below);
-        int slot = -1;
-        for (int i = 0; i < a.Kd; ++i)
-            if (a.d.dest_rank[(size_t)t * a.Kd + i] == r) slot = a.d.dest_pos[(size_t)t * a.Kd + i];
-        a.token[pos] = t;
-        a.slot[pos] = slot;
+    // eight expert slots at a time: all loads first, then the stores (see k_gm_fill)
+    for (int k0 = 0; k0 < a.K; k0 += 8) {
+        int e[8], r[8], slot[8];
+        bool use[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) e[u] = k0 + u < a.K ? a.ids[(size_t)t * a.K + k0 + u] : -1;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const bool ok = e[u] >= 0 && e[u] < a.E;
+            r[u] = ok ? a.e2r[e[u]] : -1;
+            use[u] = ok;
+            slot[u] = -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) use[u] = use[u] && r[u] >= 0 && r[u] < a.R;
+        for (int j = 0; j < k0 + 7 && j < a.K; ++j) {          // an expert named twice by a token counts once (the first time)
+            const int ej = a.ids[(size_t)t * a.K + j];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) use[u] = use[u] && !(j < k0 + u && ej == e[u]);
+        }
+#pragma unroll 4
+        for (int i = 0; i < a.Kd; ++i) {
+            const int dr = a.d.dest_rank[(size_t)t * a.Kd + i], dp = a.d.dest_pos[(size_t)t * a.Kd + i];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) slot[u] = (use[u] && dr == r[u]) ? dp : slot[u];
+        }
+        int pos[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            pos[u] = 0;
+            if (!use[u]) continue;
+            pos[u] = FUSED ? start[e[u]] : a.offsets[e[u]] + a.d.ex_tile_cnt[(size_t)blockIdx.x * a.E + e[u]];
+            for (int w = 0; w < warp; ++w) pos[u] += __popc(sm32[(size_t)e[u] * 8 + w]);
+            pos[u] += __popc(sm32[(size_t)e[u] * 8 + warp] & below);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (use[u]) { a.token[pos[u]] = t; a.slot[pos[u]] = slot[u]; }
     }
 }
 
-size_t gm_smem(const mw_ctx *ctx) { return (size_t)kTile * ctx->W * 8 + (size_t)kTile * 4; }
-size_t ex_smem(const mw_ctx *ctx) { return (size_t)ctx->cfg.E * 32; }
+size_t gm_smem(const mw_ctx *ctx) { return (size_t)kTile * ctx->W * 8 + (size_t)kTile * 4 + (size_t)ctx->cfg.R * 4; }
+size_t ex_smem(const mw_ctx *ctx) { return (size_t)ctx->cfg.E * 36; }     // bit matrix (32 bytes per expert) + one list position
 
 }  // namespace
 
@@ -242,7 +347,8 @@ int mw_order_smem_setup(mw_ctx *ctx)
     const size_t ex = ex_smem(ctx);
     if (ex > 48 * 1024 && ex + 1024 <= (size_t)ctx->max_smem_optin) {
         if (cudaFuncSetAttribute(k_ex_count, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ex) != cudaSuccess ||
-            cudaFuncSetAttribute(k_ex_fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ex) != cudaSuccess)
+            cudaFuncSetAttribute(k_ex_fill<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ex) != cudaSuccess ||
+            cudaFuncSetAttribute(k_ex_fill<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ex) != cudaSuccess)
             return MW_ERR_CUDA;
     }
     return MW_OK;
@@ -266,10 +372,14 @@ extern "C" int mw_group_major(mw_ctx *ctx, mw_group_major_view *view, void *stre
     cudaStream_t st = (cudaStream_t)stream;
     const size_t smem = gm_smem(ctx);
     k_gm_sum<<<a.tiles, kTile, smem, st>>>(a);
-    k_gm_scan<<<(a.R + kTile - 1) / kTile, kTile, 0, st>>>(a);
-    k_gm_fill<<<a.tiles, kTile, smem, st>>>(a);
-    k_gm_tokens<<<a.tiles, kTile, 0, st>>>(a);
-    ctx->launches += 4;
+    if (a.tiles <= kFuseTiles) {
+        k_gm_fill<false><<<a.tiles, kTile, smem, st>>>(a);
+        ctx->launches += 2;
+    } else {
+        k_gm_scan<<<(a.R + kTile - 1) / kTile, kTile, 0, st>>>(a);
+        k_gm_fill<true><<<a.tiles, kTile, smem, st>>>(a);
+        ctx->launches += 3;
+    }
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
 }
 
@@ -317,9 +427,15 @@ extern "C" int mw_expert_index(mw_ctx *ctx, const int32_t *topk_ids, const int32
     a.T = T; a.K = ctx->cfg.K; a.E = ctx->cfg.E; a.R = ctx->cfg.R; a.Kd = ctx->Kd;
     a.tiles = (T + kTile - 1) / kTile;
     cudaStream_t st = (cudaStream_t)stream;
-    if (T > 0) k_ex_count<<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
-    k_ex_scan<<<1, 1024, 0, st>>>(a);
-    if (T > 0) k_ex_fill<<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
-    ctx->launches += T > 0 ? 3 : 1;
+    if (T > 0 && a.tiles <= kFuseTiles) {
+        k_ex_count<<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
+        k_ex_fill<true><<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
+        ctx->launches += 2;
+    } else {
+        if (T > 0) k_ex_count<<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
+        k_ex_scan<<<1, 1024, 0, st>>>(a);
+        if (T > 0) k_ex_fill<false><<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
+        ctx->launches += T > 0 ? 3 : 1;
+    }
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
 }
