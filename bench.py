@@ -1,17 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the MultiWrite dispatch hot path (plan -> pack -> deliver) on B200.
 
-One step = one whole pass over one batch: mw_plan, then mw_pack and mw_deliver in the MultiWrite
+One step = one whole pass over one batch: mw_plan_prefetch, then mw_pack and mw_deliver in the MultiWrite
 layout, all through the C ABI, inputs resident in device memory.  The workload is the
 DeepSeek-V3-shaped prefill dispatch (64 ranks, 256 experts, top-8, 4096 tokens, 7168 bf16 per row).
 The step cycles over several buffer sets so that every step's inputs and outputs come from HBM,
-not L2.  Prints one JSON line (see README / DESIGN for the fields).
+not L2.  Prints one JSON line: the headline keys first, then the blocks for the other shapes and paths; the
+last keys are tiny, unicast, large_ep, pipelined, bytes_saved_pct and decode.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
 
-With N > 1 (launched by torch.distributed.run) every rank runs the same workload on its own GPU
-with its own seed: independent replicas, no collective on the data path; the time is the maximum
-over ranks.  `--impl reference` times the CPU oracle on the host cores instead.
+With N > 1 every rank runs the same workload on its own GPU with its own seed: independent replicas, no
+collective on the data path; the time is the maximum over ranks.  Started without a launcher (no WORLD_SIZE in
+the environment) the script starts the N ranks itself through torch.distributed.run.
+`--impl reference` times the CPU oracle on the host cores instead.
 """
 from __future__ import annotations
 
@@ -51,10 +53,10 @@ def algorithmic_bytes(tot: dict, B: int) -> dict:
     return {"pack": 2 * Tn * B, "deliver": (Tn + SD) * B, "step": (3 * Tn + SD) * B}
 
 
-def recorded_traffic():
-    """DRAM bytes per deliver launch from the committed ncu summary, or None when the kernel source
+def recorded_traffic(workload: str = WORKLOAD):
+    """DRAM bytes per deliver launch from the committed ncu summary of that workload, or None when the kernel source
     has changed since the counters were taken."""
-    path = os.path.join(ROOT, "profiles", "deliver_dsv3_prefill_ncu.md")
+    path = os.path.join(ROOT, "profiles", f"deliver_{workload}_ncu.md")
     try:
         text = open(path).read()
         m_t = re.search(r"traffic_bytes_per_launch\s*=\s*(\d+)", text)
@@ -72,6 +74,39 @@ def kernel_source_hash() -> str:
         with open(os.path.join(ROOT, "paper_2605_22428_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
+
+
+def roofline_block(kernel: str, alg_bytes: int, times_ms: list, traffic, peak: float, peak_src: str) -> dict:
+    """The roofline object of one kernel from its per-launch CUDA-event durations: `achieved` counts the algorithmic
+    bytes, `dram_gbs` the DRAM bytes ncu recorded for one launch (reads served by L2 are not in it)."""
+    mean_ms = statistics.mean(times_ms)
+    achieved = alg_bytes / (mean_ms * 1e-3) / 1e9
+    out = {"bound": "hbm", "kernel": kernel, "launches_timed": len(times_ms), "achieved": round(achieved, 1), "peak": peak,
+           "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_source": peak_src,
+           "mean_us": round(mean_ms * 1e3, 2), "p50_us": round(statistics.median(times_ms) * 1e3, 2),
+           "algorithmic_bytes_per_launch": alg_bytes, "traffic": traffic}
+    if traffic:
+        out["dram_gbs"] = round(traffic / (mean_ms * 1e-3) / 1e9, 1)
+        out["dram_frac"] = round(out["dram_gbs"] / peak, 4)
+        out["dram_frac_of_nominal_8TBs"] = round(out["dram_gbs"] / NOMINAL_HBM_GBS, 4)
+    return out
+
+
+def time_deliver_launches(ctx, mw, torch, ids, e2r, T, sets, Tn, SD, launches: int = 200, warmup: int = 20) -> list:
+    """CUDA-event duration (ms) of `launches` deliver launches, each right after the plan and pack launches of its
+    step (so the send rows are where the step leaves them), cycling over the buffer sets."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+    for i in range(warmup + launches):
+        x, send, recv = sets[i % len(sets)]
+        ctx.mw_plan_prefetch(ids, e2r, T, x)
+        ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+        if i >= warmup:
+            evs[i - warmup][0].record()
+        ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
+        if i >= warmup:
+            evs[i - warmup][1].record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
 
 
 # ---- clocks ------------------------------------------------------------------------------------------
@@ -164,15 +199,71 @@ def sample_inputs(inp, T: int):
                              np.ascontiguousarray(inp.x[:T]))
 
 
-def cpu_baseline(inp, R: int, B: int, budget_s: float = 12.0) -> dict:
-    secs, tot = oracle_pass(inp, R, B)          # first pass also warms the page cache
+def oracle_stages(inp, R: int, B: int, threads: int = 1, keep: bool = False):
+    """One pass of the oracle, stage by stage: (plan s, pack s, deliver s, totals).  With threads > 1 the send rows are
+    cut into contiguous slices and the oracle's own pack / deliver functions run on one slice per thread (the C calls
+    release the interpreter lock; slices write disjoint rows); the plan is a sequential walk and stays on one core."""
+    import ctypes as C
+    from oracle import mwo
+    t0 = time.perf_counter()
+    p = mwo.plan(inp.topk_ids, inp.expert_to_rank, R, B)
+    t1 = time.perf_counter()
+    Tn, SD = p.totals["T_nonempty"], p.totals["total_dest"]
+    if threads <= 1:
+        send = mwo.pack_mw(p, inp.x)
+        t2 = time.perf_counter()
+        recv = mwo.deliver_mw(p, send)
+        t3 = time.perf_counter()
+        return (t1 - t0, t2 - t1, t3 - t2, p.totals) + ((send, recv) if keep else ())
+    from concurrent.futures import ThreadPoolExecutor
+    lib = mwo.lib()
+    xb = np.ascontiguousarray(inp.x).view(np.uint8).reshape(inp.T, B)
+    send = np.empty((max(Tn, 1), B), np.uint8)
+    recv = np.empty(max(SD, 1) * B, np.uint8)
+    cuts = [Tn * k // threads for k in range(threads + 1)]
+    vp = C.c_void_p
+
+    def pack(k):
+        j0, n = cuts[k], cuts[k + 1] - cuts[k]
+        lib.mwo_pack_mw(vp(xb.ctypes.data), C.c_int64(B), vp(p.mw_row_token.ctypes.data + 4 * j0), C.c_int64(n),
+                        vp(send.ctypes.data + j0 * B))
+
+    def deliver(k):
+        j0, n = cuts[k], cuts[k + 1] - cuts[k]
+        lib.mwo_deliver_mw(vp(send.ctypes.data + j0 * B), C.c_int64(B), C.c_int64(n), C.c_int32(R), C.c_int32(p.K),
+                           vp(p.mw_row_token.ctypes.data + 4 * j0), vp(p.token_group.ctypes.data), vp(p.group_mask.ctypes.data),
+                           vp(p.dest_pos.ctypes.data), vp(p.rank_offsets.ctypes.data), vp(recv.ctypes.data), C.c_int64(0))
+
+    with ThreadPoolExecutor(threads) as pool:
+        list(pool.map(pack, range(threads)))
+        t2 = time.perf_counter()
+        list(pool.map(deliver, range(threads)))
+        t3 = time.perf_counter()
+    return (t1 - t0, t2 - t1, t3 - t2, p.totals) + ((send[:Tn], recv[:SD * B]) if keep else ())
+
+
+def cpu_baseline(inp, R: int, B: int, budget_s: float = 10.0) -> dict:
+    """The oracle on the host cores: single thread (the headline figure of this block) and all cores, per stage."""
+    first = oracle_stages(inp, R, B)                # also warms the page cache
+    secs = sum(first[:3])
     reps = max(1, min(8, int(budget_s / max(secs, 1e-3))))
-    times = [oracle_pass(inp, R, B)[0] for _ in range(reps)]
-    best = min(times)
-    return {"value": algorithmic_bytes(tot, B)["step"] / best / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+    runs = [oracle_stages(inp, R, B) for _ in range(reps)]
+    best = min(runs, key=lambda r: sum(r[:3]))
+    tot = best[3]
+    step_bytes = algorithmic_bytes(tot, B)["step"]
+    cores = os.cpu_count() or 1
+    par_runs = [oracle_stages(inp, R, B, threads=cores) for _ in range(max(1, min(4, reps)))]
+    par = min(par_runs, key=lambda r: sum(r[:3]))
+    ms = lambda v: round(v * 1e3, 2)
+    return {"value": step_bytes / sum(best[:3]) / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
             "sample": f"full {WORKLOAD} batch ({inp.T} tokens), best of {reps} passes after one warm-up pass, "
-                      f"plan+pack+deliver in plain single-threaded C; median {statistics.median(times) * 1e3:.1f} ms",
-            "ms_per_step": best * 1e3}
+                      f"plan+pack+deliver in plain single-threaded C",
+            "ms_per_step": ms(sum(best[:3])), "plan_ms": ms(best[0]), "pack_ms": ms(best[1]), "deliver_ms": ms(best[2]),
+            "median_ms": ms(statistics.median(sum(r[:3]) for r in runs)),
+            "all_cores": {"value": step_bytes / sum(par[:3]) / 1e9, "unit": "GB/s", "cores": cores,
+                          "ms_per_step": ms(sum(par[:3])), "plan_ms": ms(par[0]), "pack_ms": ms(par[1]), "deliver_ms": ms(par[2]),
+                          "how": "send rows cut into one slice per core, the oracle's pack and deliver run per slice on a "
+                                 "thread each; the plan stays sequential"}}
 
 
 def run_reference(args):
@@ -330,7 +421,7 @@ def allgather_sweep(mw, wl, torch) -> list:
     return out
 
 
-def relay_measure(mw, wl, torch) -> dict:
+def relay_measure(mw, wl, torch, n: int = 50) -> dict:
     """Two-level dispatch (Section 3.2) on the dsv3_prefill routing: 8 servers of 8 ranks, source = rank 0."""
     inp = wl.make_dispatch(WORKLOAD)
     s = inp.shape
@@ -354,22 +445,33 @@ def relay_measure(mw, wl, torch) -> dict:
             step(i)
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n = 50
         a.record()
         for i in range(n):
             step(i)
         b.record()
         torch.cuda.synchronize()
         us = a.elapsed_time(b) * 1e3 / n
+        a.record()
+        for i in range(n):
+            relay.mw_relay_plan(ids, e2r, T)
+        b.record()
+        torch.cuda.synchronize()
+        plan_us = a.elapsed_time(b) * 1e3 / n
         assert relay.mw_relay_get_totals()["status"] == 0
-    moved = ((2 * rows_send + H) + (H + SD)) * B                       # first level in one pass (x read once), second level
-    return {"servers": s.R // P, "ranks_per_server": P, "src_rank": src, "hop_rows": H, "delivered_rows": SD,
+    fwd = tot["forward_bytes"] // B                                     # copies the relays forward
+    held = tot["inter_multiwrite_bytes"] // B                           # copies held by relays (read back unless there is nothing to forward)
+    alg = (2 * rows_send + H + held + fwd) * B                          # x read, send + hop copies written, copies read back, forwards written
+    dram = (2 * rows_send + H + fwd) * B                                # the read-backs come out of L2
+    return {"servers": s.R // P, "ranks_per_server": P, "src_rank": src, "hop_rows": H, "staged_rows": tot["staged_rows"],
+            "delivered_rows": SD,
             "inter_server_unicast_mb": round(tot["inter_unicast_bytes"] / 1e6, 1),
             "inter_server_multiwrite_mb": round(tot["inter_multiwrite_bytes"] / 1e6, 1),
             "inter_server_bytes_saved_pct": round(100 * (1 - tot["inter_multiwrite_bytes"] / tot["inter_unicast_bytes"]), 2),
             "direct_mb": round(tot["direct_bytes"] / 1e6, 1), "relay_forward_mb": round(tot["forward_bytes"] / 1e6, 1),
-            "step_us": round(us, 1), "gbs": round(moved / us / 1e3, 1),
-            "note": "step = both plans + descriptors + first level (pack and deliver in one pass) + second-level expansion"}
+            "step_us": round(us, 1), "plan_us": round(plan_us, 1), "gbs": round(alg / us / 1e3, 1),
+            "dram_side_gbs": round(dram / us / 1e3, 1), "frac_of_measured_peak": round(alg / us / 1e3 / measured_peak()[0], 4),
+            "note": "step = both plans (concurrent) + descriptors + one launch for both levels; gbs counts x read, send and hop "
+                    "copies written, relay copies read back (upper bound) and forwards written; dram_side_gbs leaves the read-backs out"}
 
 
 def paper_setup_measure(mw, wl, torch) -> list:
@@ -505,9 +607,15 @@ def large_ep_measure(mw, wl, torch) -> dict:
             b.record()
             torch.cuda.synchronize()
             out[name] = round(a.elapsed_time(b) * 1e3 / n, 1)
+        peak, peak_src = measured_peak()
+        deliver_roofline = roofline_block("k_copy_rows<1, SCATTER, after pack> (deliver, MultiWrite layout, large_ep)", (Tn + SD) * B,
+                                          time_deliver_launches(ctx, mw, torch, ids, e2r, T, sets, Tn, SD),
+                                          recorded_traffic("large_ep"), peak, peak_src)
         assert ctx.mw_get_totals()["status"] == 0
     nbytes = (3 * Tn + SD) * B
+    out["roofline"] = deliver_roofline
     out.update({"rows_packed": Tn, "rows_delivered": SD, "groups": tot["G"], "algorithmic_bytes_per_step": nbytes,
+                "step_frac_of_measured_peak": round(nbytes / out["step_us"] / 1e3 / measured_peak()[0], 4),
                 "step_gbs": round(nbytes / out["step_us"] / 1e3, 1),
                 "pack_plus_deliver_gbs": round(nbytes / out["pack_plus_deliver_us"] / 1e3, 1),
                 "pack_plus_deliver_fraction_of_nominal_8TBs": round(nbytes / out["pack_plus_deliver_us"] / 1e3 / 8000.0, 4),
@@ -578,54 +686,159 @@ def mid_batch_measure(mw, wl, torch) -> list:
     return out
 
 
-def two_stream_measure(mw, wl, torch) -> dict:
-    """The headline step with consecutive batches alternating between two contexts on two streams, so that the plan of
-    one batch (a latency chain on a few SMs) runs under the deliver of the previous one.  An orchestration the caller
-    chooses; the headline figure is the single-stream step."""
-    inp = wl.make_dispatch(WORKLOAD)
+def pipelined_measure(mw, wl, torch, name: str, steps: int = 400) -> dict:
+    """The headline step with the plan of batch i+1 made while batch i is packed and delivered, through ONE context
+    (mw_plan_swap / mw_plan_next): time per step (p50 over `steps` steps, CUDA events between the steps) and the latency
+    of one batch from the moment its plan may start to the end of its deliver."""
+    inp = wl.make_dispatch(name)
     s = inp.shape
     B, T = s.row_bytes, s.T
     ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
     xh = torch.from_numpy(inp.x.view(np.int16))
-    ctxs = [mw.Context(s.R, s.E, s.K, T, B) for _ in range(2)]
-    try:
-        ctxs[0].mw_plan(ids, e2r, T)
-        tot = ctxs[0].mw_get_totals()
+    nsets = 3 if name == WORKLOAD else 2
+    with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+        ctx.mw_plan(ids, e2r, T)
+        tot = ctx.mw_get_totals()
         Tn, SD = tot["T_nonempty"], tot["total_dest"]
         sets = [(xh.cuda(), torch.empty(Tn * B, dtype=torch.uint8, device="cuda"),
-                 torch.empty(SD * B, dtype=torch.uint8, device="cuda")) for _ in range(4)]
-        streams = [torch.cuda.Stream() for _ in range(2)]
-        main = torch.cuda.current_stream()
+                 torch.empty(SD * B, dtype=torch.uint8, device="cuda")) for _ in range(nsets)]
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 2)]
 
-        def step(i):
-            c, st = ctxs[i % 2], streams[i % 2]
-            x, send, recv = sets[i % 4]
-            c.mw_plan_prefetch(ids, e2r, T, x, stream=st)
-            c.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn, stream=st)
-            c.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD, stream=st)
+        def step(i, mark=None):
+            x, send, recv = sets[i % nsets]
+            ctx.mw_plan_swap()                                   # the plan of this batch, issued one step ago
+            if mark is not None:
+                mark.record()                                    # from here the next batch's plan may run
+            ctx.mw_plan_next(ids, e2r, T)                        # no prefetch: DRAM is busy with this batch's copies
+            ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+            ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
 
-        for i in range(8):
+        ctx.mw_plan_next(ids, e2r, T)
+        for i in range(20):
             step(i)
         torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n = 400
-        a.record()
-        for st in streams:
-            st.wait_stream(main)
-        for i in range(n):
-            step(i)
-        for st in streams:
-            main.wait_stream(st)
-        b.record()
+        for i in range(steps + 1):
+            step(i, marks[i])
+        marks[steps + 1].record()
         torch.cuda.synchronize()
-        us = a.elapsed_time(b) * 1e3 / n
-        assert all(c.mw_get_totals()["status"] == 0 for c in ctxs)
-    finally:
-        for c in ctxs:
-            c.close()
+        ctx.mw_plan_swap()
+        assert ctx.mw_get_totals()["status"] == 0
+    per_step = [marks[i].elapsed_time(marks[i + 1]) * 1e3 for i in range(steps)]
+    # batch i+1: its plan may start at mark i, its deliver ends where step i+2 begins (mark i+2)
+    latency = [marks[i].elapsed_time(marks[i + 2]) * 1e3 for i in range(steps)]
     nbytes = (3 * Tn + SD) * B
-    return {"step_us": round(us, 1), "step_gbs": round(nbytes / us / 1e3, 1), "tokens_per_s": round(T / us * 1e6, 1),
-            "note": "two contexts, two streams, batches alternate; time per step over 400 steps"}
+    us = statistics.median(per_step)
+    return {"steps": steps, "step_p50_us": round(us, 2), "step_mean_us": round(marks[0].elapsed_time(marks[steps]) * 1e3 / steps, 2),
+            "step_p99_us": round(percentile(per_step, 0.99), 2), "batch_latency_p50_us": round(statistics.median(latency), 2),
+            "step_gbs": round(nbytes / us / 1e3, 1), "frac_of_measured_peak": round(nbytes / us / 1e3 / measured_peak()[0], 4),
+            "tokens_per_s": round(T / us * 1e6, 1),
+            "note": "one context, one caller stream; mw_plan_swap + mw_plan_next + mw_pack + mw_deliver per step; the plan runs on "
+                    "the library's planning stream under the previous batch's copies; latency = plan may start -> deliver done"}
+
+
+def unicast_measure(mw, wl, torch, name: str, n: int = 100) -> dict:
+    """The unicast layout (one copy per destination in the send buffer: Sections 2.2, 6.3) against the MultiWrite layout on
+    the same batch: pack, deliver and whole step of each, same context, same plan."""
+    inp = wl.make_dispatch(name)
+    s = inp.shape
+    B, T = s.row_bytes, s.T
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    xh = torch.from_numpy(inp.x.view(np.int16))
+    out = {}
+    with mw.Context(s.R, s.E, s.K, T, B) as ctx:
+        ctx.mw_plan(ids, e2r, T)
+        tot = ctx.mw_get_totals()
+        Tn, SD = tot["T_nonempty"], tot["total_dest"]
+        xs = [xh.cuda() for _ in range(2)]
+        recvs = [torch.empty(SD * B, dtype=torch.uint8, device="cuda") for _ in range(2)]
+        for layout, lname, rows in ((mw.MW_LAYOUT_UNICAST, "unicast", SD), (mw.MW_LAYOUT_MULTIWRITE, "multiwrite", Tn)):
+            sends = [torch.empty(rows * B, dtype=torch.uint8, device="cuda") for _ in range(2)]
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n)]
+            for i in range(10 + n):
+                x, send, recv = xs[i % 2], sends[i % 2], recvs[i % 2]
+                e = evs[i - 10] if i >= 10 else None
+                if e:
+                    e[0].record()
+                ctx.mw_plan_prefetch(ids, e2r, T, x)
+                if e:
+                    e[1].record()
+                ctx.mw_pack(x, layout, send, rows)
+                if e:
+                    e[2].record()
+                ctx.mw_deliver(layout, send, recv, 0, SD)
+                if e:
+                    e[3].record()
+            torch.cuda.synchronize()
+            med = lambda a, b: statistics.median(e[a].elapsed_time(e[b]) for e in evs) * 1e3
+            pack_b = (Tn + rows) * B                              # hidden rows read once, send rows written
+            deliver_b = (rows + SD) * B
+            out[lname] = {"pack_us": round(med(1, 2), 1), "deliver_us": round(med(2, 3), 1), "step_us": round(med(0, 3), 1),
+                          "send_rows": rows, "pack_gbs": round(pack_b / med(1, 2) / 1e3, 1),
+                          "deliver_gbs": round(deliver_b / med(2, 3) / 1e3, 1),
+                          "bytes_moved_per_step": pack_b + deliver_b}
+            del sends
+        assert ctx.mw_get_totals()["status"] == 0
+    u, m = out["unicast"], out["multiwrite"]
+    out["time_saved_pct"] = round(100 * (1 - m["step_us"] / u["step_us"]), 2)
+    out["transmitted_bytes_saved_pct"] = round(100.0 * (1 - tot["mw_bytes"] / tot["unicast_bytes"]), 3)
+    out["note"] = "p50 of CUDA events around each call over %d steps; one GPU emulates every link, so time follows bytes moved in HBM" % n
+    return out
+
+
+def tiny_measure(mw, wl, torch, launches: int = 500) -> dict:
+    """The smallest configuration (8 ranks, 256 tokens of 2 KB): latency in microseconds (its working set lives in L2)."""
+    inp = wl.make_dispatch("tiny")
+    s = inp.shape
+    B = s.row_bytes
+    ids, e2r = torch.from_numpy(inp.topk_ids).cuda(), torch.from_numpy(inp.expert_to_rank).cuda()
+    x = torch.from_numpy(inp.x.view(np.int16)).cuda()
+    out = {}
+    with mw.Context(s.R, s.E, s.K, s.T, B) as ctx:
+        ctx.mw_plan(ids, e2r, s.T)
+        tot = ctx.mw_get_totals()
+        Tn, SD = tot["T_nonempty"], tot["total_dest"]
+        send = torch.empty(Tn * B, dtype=torch.uint8, device="cuda")
+        recv = torch.empty(SD * B, dtype=torch.uint8, device="cuda")
+
+        def three():
+            ctx.mw_plan(ids, e2r, s.T)
+            ctx.mw_pack(x, mw.MW_LAYOUT_MULTIWRITE, send, Tn)
+            ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send, recv, 0, SD)
+
+        def one_call():
+            ctx.mw_plan_dispatch(ids, e2r, s.T, x, mw.MW_LAYOUT_MULTIWRITE, send, Tn, recv, 0, SD)
+
+        for name, fn in (("three_calls", three), ("one_call", one_call)):
+            for _ in range(30):
+                fn()
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+            torch.cuda.synchronize()
+            for a, b in evs:
+                a.record()
+                fn()
+                b.record()
+            torch.cuda.synchronize()
+            us = [a.elapsed_time(b) * 1e3 for a, b in evs]
+            out[name] = {"p50_us": round(percentile(us, 0.5), 2), "p99_us": round(percentile(us, 0.99), 2)}
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_call()
+        for _ in range(10):
+            graph.replay()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+        torch.cuda.synchronize()
+        for a, b in evs:
+            a.record()
+            graph.replay()
+            b.record()
+        torch.cuda.synchronize()
+        us = [a.elapsed_time(b) * 1e3 for a, b in evs]
+        out["one_call_graph"] = {"p50_us": round(percentile(us, 0.5), 2), "p99_us": round(percentile(us, 0.99), 2)}
+        assert ctx.mw_get_totals()["status"] == 0
+    out["rows_delivered"], out["groups"] = SD, tot["G"]
+    out["note"] = "L2-resident (0.5 MB in, 1.8 MB out): microseconds, not an HBM fraction; host launch cost included except one_call_graph"
+    return out
 
 
 def order_measure(mw, wl, torch) -> dict:
@@ -662,7 +875,7 @@ def order_measure(mw, wl, torch) -> dict:
         assert ctx.mw_get_totals()["status"] == 0
     out["deliver_group_major_gbs"] = round((Tn + SD) * B / out["deliver_group_major_us"] / 1e3, 1)
     out["groups"] = tot["G"]
-    out["note"] = "4 + 3 short kernels over the plan (latency-bound); the deliver is the same row-copy kernel with other slots"
+    out["note"] = "2 + 2 short kernels over the plan (latency-bound); the deliver is the same row-copy kernel with other slots"
     return out
 
 
@@ -772,7 +985,12 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    inp = wl.make_dispatch(WORKLOAD, seed=1 + 1000 * rank if rank else None)
+    workload = WORKLOAD
+    if args.profile_workload:
+        if not args.kernels_only:
+            raise SystemExit("--profile-workload goes with --kernels-only (the benchmark line is always quoted on " + WORKLOAD + ")")
+        workload = args.profile_workload
+    inp = wl.make_dispatch(workload, seed=1 + 1000 * rank if rank else None)
     s = inp.shape
     B, T = s.row_bytes, s.T
     ids = torch.from_numpy(inp.topk_ids).cuda()
@@ -837,10 +1055,14 @@ def run_cuda(args):
     plan_ms = [e[0].elapsed_time(e[1]) for e in evs.values()]
     pack_ms = [e[1].elapsed_time(e[2]) for e in evs.values()]
     deliver_ms = [e[2].elapsed_time(e[3]) for e in evs.values()]
+    # the roofline kernel's duration does not depend on --steps: 20 warm-up + 200 timed launches of their own, each after
+    # the plan and pack launches of its step
+    roof_ms = time_deliver_launches(ctx, mw, torch, ids, e2r, T, sets, Tn, SD, launches=50 if args.kernels_only else 200)
 
     if args.kernels_only:
         sampler.stop()
         print(json.dumps({"kernels_only": True, "ms_per_step": total_ms / args.steps, "steps": args.steps,
+                          "deliver_launch_mean_us": statistics.mean(roof_ms) * 1e3,
                           "combine": combine_measure(mw, wl, torch),
                           "stages_us": {"plan": statistics.mean(plan_ms) * 1e3, "pack": statistics.mean(pack_ms) * 1e3,
                                         "deliver": statistics.mean(deliver_ms) * 1e3}}))
@@ -874,8 +1096,20 @@ def run_cuda(args):
     ms_per_step = total_ms / args.steps
     value = step_bytes_all / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
-    d_ms = statistics.mean(deliver_ms)
-    achieved = alg["deliver"] / (d_ms * 1e-3) / 1e9
+    d_ms, p_ms = statistics.mean(deliver_ms), statistics.mean(pack_ms)
+    roof = roofline_block("k_copy_rows<1, SCATTER, after pack> (deliver, MultiWrite layout)", alg["deliver"], roof_ms,
+                          recorded_traffic(WORKLOAD), peak, peak_src)
+    roof["timed_region_mean_us"] = round(d_ms * 1e3, 2)
+    roof["timed_region_samples"] = len(evs)
+    stages = {"plan": round(statistics.mean(plan_ms) * 1e3, 2), "pack": round(p_ms * 1e3, 2), "deliver": round(d_ms * 1e3, 2),
+              "pack_gbs": round(alg["pack"] / p_ms / 1e6, 1),
+              "pack_plus_deliver_gbs": round((alg["pack"] + alg["deliver"]) / (p_ms + d_ms) / 1e6, 1),
+              "sampled_steps": len(evs), "note": "CUDA events on every 8th step of the timed region"}
+    if roof["traffic"]:
+        # the same two launches counted in DRAM bytes: pack reads and writes every row once, deliver as ncu recorded it
+        dram = (alg["pack"] + roof["traffic"]) / (p_ms + d_ms) / 1e6
+        stages["pack_plus_deliver_dram_gbs"] = round(dram, 1)
+        stages["pack_plus_deliver_dram_frac_of_nominal_8TBs"] = round(dram / NOMINAL_HBM_GBS, 4)
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
@@ -887,14 +1121,10 @@ def run_cuda(args):
                    "rows_packed": Tn, "rows_delivered": SD, "groups": tot["G"],
                    "algorithmic_bytes_per_step": alg["step"]},
         "tokens_per_s": round(T * world / (ms_per_step * 1e-3), 1),
+        "fraction_of_measured_peak": round(value / world / peak, 4),
         "fraction_of_nominal_8TBs": round(value / world / NOMINAL_HBM_GBS, 4),
-        "stages_us": {"plan": round(statistics.mean(plan_ms) * 1e3, 2), "pack": round(statistics.mean(pack_ms) * 1e3, 2),
-                      "deliver": round(d_ms * 1e3, 2), "pack_gbs": round(alg["pack"] / statistics.mean(pack_ms) / 1e6, 1),
-                      "pack_plus_deliver_gbs": round((alg["pack"] + alg["deliver"]) / (statistics.mean(pack_ms) + d_ms) / 1e6, 1),
-                      "sampled_steps": len(evs), "note": "CUDA events on every 8th step of the timed region"},
-        "roofline": {"bound": "hbm", "kernel": "k_copy_rows<1, SCATTER> (deliver, MultiWrite layout)", "launches_timed": len(evs), "achieved": round(achieved, 1),
-                     "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": alg["deliver"], "traffic": recorded_traffic()},
+        "stages_us": stages,
+        "roofline": roof,
         "e2e": {"value": round(step_bytes_all / (e2e_ms * 1e-3) / 1e9, 3), "unit": "GB/s", "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": int(ids_h.numel() * 4 + e2r_h.numel() * 4 + T * B),
                 "d2h_bytes_per_step": int(SD * B + (s.R + 1) * 4 + 64), "steps": e2e_steps,
@@ -907,9 +1137,9 @@ def run_cuda(args):
     if rank == 0 and world == 1:
         del sets
         torch.cuda.empty_cache()
+        line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
+        line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
         if not args.no_extras:
-            line["decode"] = decode_latency(mw, wl, torch)
-            line["bytes_saved_pct"] = bytes_saved(wl)
             line["allgather_r64"] = allgather_sweep(mw, wl, torch)
             line["relay_two_level"] = relay_measure(mw, wl, torch)
             line["paper_setup_2x8"] = paper_setup_measure(mw, wl, torch)
@@ -917,16 +1147,49 @@ def run_cuda(args):
             line["combine_dsv3_prefill"] = combine_measure(mw, wl, torch)
             line["dispatch_fused"] = fused_dispatch_measure(mw, wl, torch)
             line["receiver_order"] = order_measure(mw, wl, torch)
-            line["large_ep"] = large_ep_measure(mw, wl, torch)
-            line["two_streams"] = two_stream_measure(mw, wl, torch)
             line["mid_batches"] = mid_batch_measure(mw, wl, torch)
-        line["cpu_baseline"] = cpu_baseline(inp, s.R, B)
-        line["paper_context"] = "paper reports up to 33% lower operator latency on Ascend 910B (other hardware; not a target)"
+            # the keys the metric names come last
+            line["tiny"] = tiny_measure(mw, wl, torch)
+            line["unicast"] = {name: unicast_measure(mw, wl, torch, name) for name in (WORKLOAD, "large_ep")}
+            line["large_ep"] = large_ep_measure(mw, wl, torch)
+            line["pipelined"] = {name: pipelined_measure(mw, wl, torch, name) for name in (WORKLOAD, "large_ep")}
+            line["bytes_saved_pct"] = bytes_saved(wl)
+            line["decode"] = decode_latency(mw, wl, torch)
     if rank == 0:
         print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
     return 0
+
+
+def selftest_aggregate(args):
+    """Launcher and aggregation check without a GPU (gloo on the CPU): every rank contributes made-up figures, rank 0
+    prints what the real run would print from them."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    total, e2e, units = aggregate_over_ranks(dist if world > 1 else None, 10.0 + rank, 100.0 - rank, 1000.0 * (rank + 1),
+                                             torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"selftest": "aggregate", "n_gpus": world, "total_ms": total, "e2e_ms": e2e, "units": units}))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def launch_ranks(n: int) -> int:
+    """Starts n ranks of this script on this node through torch.distributed.run (one per GPU; 127.0.0.1 rendezvous) and
+    returns its exit code.  Used when the script is started plainly with --gpus n > 1."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -941,6 +1204,11 @@ def main():
                     help="only the device-timed steps (for profiler runs): no end-to-end leg, extras or CPU baseline")
     ap.add_argument("--no-prefetch", action="store_true",
                     help="plan with mw_plan instead of mw_plan_prefetch (hidden rows not brought into L2 while planning)")
+    ap.add_argument("--profile-workload", default="", help="with --kernels-only: run that dispatch shape instead (profiler captures)")
+    ap.add_argument("--relay-only", type=int, default=0, metavar="STEPS",
+                    help="only the two-level relayed dispatch measurement with this many timed steps (for profiler runs)")
+    ap.add_argument("--selftest-aggregate", action="store_true",
+                    help="no GPU work: check the rank launcher and the max/sum aggregation over ranks on the CPU (gloo)")
     ap.add_argument("--decode-only", type=int, default=0, metavar="LAUNCHES",
                     help="only the decode-shape latency measurement with this many launches per figure (for profiler runs)")
     args = ap.parse_args()
@@ -951,9 +1219,22 @@ def main():
         torch.cuda.set_device(0)
         print(json.dumps({"decode_only": True, "decode": decode_latency(mw, wl, torch, args.decode_only)}))
         return 0
+    if args.relay_only and args.impl == "cuda":
+        import torch
+        from paper_2605_22428_b200 import binding as mw
+        from paper_2605_22428_b200 import workloads as wl
+        torch.cuda.set_device(0)
+        print(json.dumps({"relay_only": True, "relay_two_level": relay_measure(mw, wl, torch, n=args.relay_only)}))
+        return 0
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")
-    return run_reference(args) if args.impl == "reference" else run_cuda(args)
+    if args.impl == "reference":
+        return run_reference(args)                  # rank 0 alone works; started plainly it is the only process
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return launch_ranks(args.gpus)              # one replica per GPU
+    if args.selftest_aggregate:
+        return selftest_aggregate(args)
+    return run_cuda(args)
 
 
 if __name__ == "__main__":

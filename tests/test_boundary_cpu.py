@@ -102,6 +102,31 @@ def test_replica_aggregation_two_ranks_gloo():
         assert total == 11.0 and e2e == 100.0 and units == 3000.0     # max time, max time, summed work
 
 
+def test_plain_start_with_gpus_2_launches_two_ranks():
+    """`bench.py --gpus 2` started without a launcher starts the ranks itself; here on the CPU (gloo), figures made up."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-aggregate"],
+                         capture_output=True, text=True, timeout=300, check=True, env=env).stdout.strip()
+    line = json.loads(out.splitlines()[-1])
+    assert line == {"selftest": "aggregate", "n_gpus": 2, "total_ms": 11.0, "e2e_ms": 100.0, "units": 3000.0}
+
+
+def test_all_core_leg_of_the_cpu_baseline_moves_the_same_bytes():
+    """The benchmark's all-core leg runs the oracle's own pack / deliver on slices of the send rows from several threads:
+    the buffers must equal those of the plain single call."""
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2605_22428_b200 import workloads as wl
+    inp = wl.make_dispatch("dsv3_prefill", T=777, H=40)
+    one = bench.oracle_stages(inp, inp.shape.R, inp.shape.row_bytes, keep=True)
+    many = bench.oracle_stages(inp, inp.shape.R, inp.shape.row_bytes, threads=5, keep=True)
+    assert one[3] == many[3]
+    assert np.array_equal(one[4], many[4]) and np.array_equal(one[5].reshape(-1), many[5].reshape(-1))
+
+
 def test_reference_arm_prints_one_json_line():
     import json
     import subprocess
