@@ -28,6 +28,7 @@ struct GmArgs {
     mw_dev d;
     int R, W, Kd, Tm, T;
     int tiles;                 // tiles launched (covers every possible G)
+    int stash;                 // k_gm_fill keeps the tile's (rank, block start) rows in shared memory as well (Kd <= 16)
 };
 
 // Per tile of 256 groups and per rank: rows the tile's groups add to the rank's region.
@@ -36,8 +37,10 @@ __global__ void __launch_bounds__(kTile) k_gm_sum(GmArgs a)
     extern __shared__ uint64_t sm64[];
     uint64_t *mask = sm64;                          // [kTile, W]
     int *size = (int *)(mask + (size_t)kTile * a.W);  // [kTile]
-    if (a.d.totals->status == MW_ERR_TIMEOUT) return;
-    const int G = (int)a.d.totals->G;
+    grid_dependency_wait();        // launched as a programmatic dependent: only its start-up overlaps the kernel before it
+    grid_launch_dependents();      // k_gm_fill may start: all it does before its grid_dependency_wait() depends on the plan only
+    const int status = a.d.totals->status, G = (int)a.d.totals->G;      // both before the first branch: one round trip
+    if (status == MW_ERR_TIMEOUT) return;
     const int g0 = blockIdx.x * kTile;
     const int n = min(kTile, G - g0);
     if (n <= 0) {
@@ -62,6 +65,7 @@ __global__ void __launch_bounds__(kTile) k_gm_sum(GmArgs a)
 // Exclusive prefix over the tiles, per rank, in place (one thread per rank; tiles are few).
 __global__ void __launch_bounds__(kTile) k_gm_scan(GmArgs a)
 {
+    grid_launch_dependents();
     const int r = blockIdx.x * kTile + threadIdx.x;
     if (r >= a.R) return;
     int run = 0;
@@ -86,6 +90,9 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
     uint64_t *mask = sm64;
     int *size = (int *)(mask + (size_t)kTile * a.W);
     int *before_s = size + kTile;                         // [R]
+    int *region_s = before_s + a.R;                       // [R + 1] region starts of the plan
+    int *rank_s = region_s + a.R + 1;                     // [kTile, Kd] (stash) destination ranks of the tile's groups
+    int *start_s = rank_s + (a.stash ? kTile * a.Kd : 0); // [kTile, Kd] (stash) start of each group's block in that region
     __shared__ int gstart[kTile + 1];
     if (a.d.totals->status == MW_ERR_TIMEOUT) return;
     {   // tokens without destinations belong to no group: their slots are -1
@@ -101,19 +108,33 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
     if (threadIdx.x < n) gstart[threadIdx.x] = a.d.group_offsets[g0 + threadIdx.x];
     if (threadIdx.x == 0) gstart[n] = a.d.group_offsets[g0 + n];
     __syncthreads();
+    for (int r = threadIdx.x; r <= a.R; r += kTile) region_s[r] = a.d.rank_offsets[r];
+    // the token of this thread's first send row (the member-token part below starts with it)
+    const int first_row = gstart[0] + threadIdx.x;
+    const int first_token = first_row < gstart[n] ? a.d.mw_row_token[first_row] : -1;
     if (threadIdx.x < n) {
         size[threadIdx.x] = gstart[threadIdx.x + 1] - gstart[threadIdx.x];
         for (int i = 0; i < a.Kd; ++i) {
             a.d.gm_rank[(size_t)(g0 + threadIdx.x) * a.Kd + i] = -1;
             a.d.gm_offset[(size_t)(g0 + threadIdx.x) * a.Kd + i] = -1;
+            if (a.stash) rank_s[threadIdx.x * a.Kd + i] = -1;
         }
     }
+    // Everything above needs the plan only and has run while the kernel before this one (the per-tile sums, or their
+    // scan) was still at work; its results are needed from here on.
+    grid_dependency_wait();
     // rows the earlier tiles put into every region: all ranks at once (independent, coalesced loads), not rank by rank
     for (int r = threadIdx.x; r < a.R; r += kTile) {
         int before = 0;
         if (SCANNED) before = a.d.gm_tile_sum[(size_t)blockIdx.x * a.R + r];
         else
-            for (int t = 0; t < (int)blockIdx.x; ++t) before += a.d.gm_tile_sum[(size_t)t * a.R + r];
+            for (int t0 = 0; t0 < (int)blockIdx.x; t0 += 8) {             // eight independent loads per round trip
+                int v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = t0 + u < (int)blockIdx.x ? a.d.gm_tile_sum[(size_t)(t0 + u) * a.R + r] : 0;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) before += v[u];
+            }
         before_s[r] = before;
     }
     __syncthreads();
@@ -135,6 +156,7 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
                 for (int w = 0; w < (r >> 6); ++w) i += __popcll(m[w]);
                 a.d.gm_rank[(size_t)(g0 + j) * a.Kd + i] = r;
                 a.d.gm_offset[(size_t)(g0 + j) * a.Kd + i] = run + incl - mine;
+                if (a.stash) { rank_s[j * a.Kd + i] = r; start_s[j * a.Kd + i] = run + incl - mine; }
             }
             run += __shfl_sync(0xffffffffu, incl, 31);
         }
@@ -148,18 +170,19 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
             if (gstart[mid] <= row) lo = mid; else hi = mid;
         }
         const int g = g0 + lo, within = row - gstart[lo];
-        const int t = a.d.mw_row_token[row];
+        const int t = row == first_row ? first_token : a.d.mw_row_token[row];
         // eight destinations at a time: all loads first, then the stores (a store in between would hold the next loads back,
         // since the compiler must assume that the arrays overlap)
         for (int i0 = 0; i0 < a.Kd; i0 += 8) {
             int r[8], pos[8], region[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                r[u] = i0 + u < a.Kd ? a.d.gm_rank[(size_t)g * a.Kd + i0 + u] : -1;
-                pos[u] = i0 + u < a.Kd ? a.d.gm_offset[(size_t)g * a.Kd + i0 + u] : -1;
+                const bool in = i0 + u < a.Kd;
+                r[u] = !in ? -1 : a.stash ? rank_s[lo * a.Kd + i0 + u] : a.d.gm_rank[(size_t)g * a.Kd + i0 + u];
+                pos[u] = (!in || r[u] < 0) ? -1 : a.stash ? start_s[lo * a.Kd + i0 + u] : a.d.gm_offset[(size_t)g * a.Kd + i0 + u];
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) region[u] = r[u] >= 0 ? a.d.rank_offsets[r[u]] : 0;
+            for (int u = 0; u < 8; ++u) region[u] = r[u] >= 0 ? region_s[r[u]] : 0;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 if (i0 + u >= a.Kd) break;
@@ -203,6 +226,7 @@ __device__ __forceinline__ void expert_bits(const ExArgs &a, uint32_t *bits, int
 __global__ void __launch_bounds__(kTile) k_ex_count(ExArgs a)
 {
     extern __shared__ uint32_t sm32[];
+    grid_launch_dependents();      // k_ex_fill may build its bit matrix meanwhile
     expert_bits(a, sm32, blockIdx.x * kTile + threadIdx.x);
     for (int e = threadIdx.x; e < a.E; e += kTile) {
         int c = 0;
@@ -217,6 +241,7 @@ __global__ void __launch_bounds__(1024) k_ex_scan(ExArgs a)
 {
     __shared__ int warp_tot[32];
     __shared__ int carry_s;
+    grid_launch_dependents();
     if (threadIdx.x == 0) carry_s = 0;
     __syncthreads();
     for (int e0 = 0; e0 < a.E; e0 += 1024) {
@@ -256,6 +281,7 @@ __global__ void __launch_bounds__(kTile) k_ex_fill(ExArgs a)
     int *start = (int *)(sm32 + (size_t)a.E * 8);          // [E] (FUSED) first list position of this tile's tokens per expert
     const int t = blockIdx.x * kTile + threadIdx.x;
     expert_bits(a, sm32, t);
+    grid_dependency_wait();        // the counts of the kernel before this one are needed from here on
     int P;
     if (FUSED) {
         if (threadIdx.x == 0) carry_s = 0;
@@ -337,13 +363,26 @@ __global__ void __launch_bounds__(kTile) k_ex_fill(ExArgs a)
     }
 }
 
-size_t gm_smem(const mw_ctx *ctx) { return (size_t)kTile * ctx->W * 8 + (size_t)kTile * 4 + (size_t)ctx->cfg.R * 4; }
+bool gm_stash(const mw_ctx *ctx) { return ctx->Kd <= 16; }
+size_t gm_smem(const mw_ctx *ctx)
+{
+    return (size_t)kTile * ctx->W * 8 + (size_t)kTile * 4 + ((size_t)2 * ctx->cfg.R + 1) * 4 +
+           (gm_stash(ctx) ? (size_t)2 * kTile * ctx->Kd * 4 : 0);
+}
 size_t ex_smem(const mw_ctx *ctx) { return (size_t)ctx->cfg.E * 36; }     // bit matrix (32 bytes per expert) + one list position
 
 }  // namespace
 
 int mw_order_smem_setup(mw_ctx *ctx)
 {
+    const size_t gm = gm_smem(ctx);
+    if (gm > 48 * 1024) {
+        if (gm > (size_t)ctx->max_smem_optin) return MW_ERR_INVALID_ARG;
+        if (cudaFuncSetAttribute(k_gm_sum, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gm) != cudaSuccess ||
+            cudaFuncSetAttribute(k_gm_fill<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gm) != cudaSuccess ||
+            cudaFuncSetAttribute(k_gm_fill<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gm) != cudaSuccess)
+            return MW_ERR_CUDA;
+    }
     const size_t ex = ex_smem(ctx);
     if (ex > 48 * 1024 && ex + 1024 <= (size_t)ctx->max_smem_optin) {
         if (cudaFuncSetAttribute(k_ex_count, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ex) != cudaSuccess ||
@@ -369,15 +408,16 @@ extern "C" int mw_group_major(mw_ctx *ctx, mw_group_major_view *view, void *stre
     GmArgs a;
     a.d = ctx->d; a.R = ctx->cfg.R; a.W = ctx->W; a.Kd = ctx->Kd; a.Tm = ctx->cfg.max_tokens; a.T = T;
     a.tiles = (T + kTile - 1) / kTile;
+    a.stash = gm_stash(ctx) ? 1 : 0;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t smem = gm_smem(ctx);
-    k_gm_sum<<<a.tiles, kTile, smem, st>>>(a);
+    mw_launch(k_gm_sum, dim3(a.tiles), dim3(kTile), smem, st, true, a);
     if (a.tiles <= kFuseTiles) {
-        k_gm_fill<false><<<a.tiles, kTile, smem, st>>>(a);
+        mw_launch(k_gm_fill<false>, dim3(a.tiles), dim3(kTile), smem, st, true, a);
         ctx->launches += 2;
     } else {
         k_gm_scan<<<(a.R + kTile - 1) / kTile, kTile, 0, st>>>(a);
-        k_gm_fill<true><<<a.tiles, kTile, smem, st>>>(a);
+        mw_launch(k_gm_fill<true>, dim3(a.tiles), dim3(kTile), smem, st, true, a);
         ctx->launches += 3;
     }
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
@@ -429,12 +469,12 @@ extern "C" int mw_expert_index(mw_ctx *ctx, const int32_t *topk_ids, const int32
     cudaStream_t st = (cudaStream_t)stream;
     if (T > 0 && a.tiles <= kFuseTiles) {
         k_ex_count<<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
-        k_ex_fill<true><<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
+        mw_launch(k_ex_fill<true>, dim3(a.tiles), dim3(kTile), ex_smem(ctx), st, true, a);
         ctx->launches += 2;
     } else {
         if (T > 0) k_ex_count<<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
         k_ex_scan<<<1, 1024, 0, st>>>(a);
-        if (T > 0) k_ex_fill<false><<<a.tiles, kTile, ex_smem(ctx), st>>>(a);
+        if (T > 0) mw_launch(k_ex_fill<false>, dim3(a.tiles), dim3(kTile), ex_smem(ctx), st, true, a);
         ctx->launches += T > 0 ? 3 : 1;
     }
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
