@@ -235,7 +235,7 @@ struct RowsArgs {
     mw_totals *totals;           // first-level accounting: row count, status
 };
 
-constexpr int kRelayMaxThreads = 512;
+constexpr int kRelayMaxThreads = 256;
 constexpr int kRelayBatch = 4;   // relay copies a thread reads back before it starts storing
 
 __device__ __forceinline__ uint4 ld_row(const uint8_t *p)
@@ -321,9 +321,13 @@ __global__ void __launch_bounds__(kRelayMaxThreads) k_relay_rows(const __grid_co
     __syncthreads();
     if (!mine) return;
     // first level: the send slot and one copy per next hop
-    if (row < a.send_capacity_rows) *(uint4 *)(a.send + (int64_t)row * a.row_bytes + off) = v;
-    for (int i = 0; i < nh; ++i)
-        if (held_s[i]) *(uint4 *)(held_s[i] + off) = v;
+    // (a copy that is read back below is stored normally and stays in L2; everything else is written once and streams)
+    if (row < a.send_capacity_rows) __stcs((uint4 *)(a.send + (int64_t)row * a.row_bytes + off), v);
+    for (int i = 0; i < nh; ++i) {
+        if (!held_s[i]) continue;
+        if (cnt_s[i] > 0) *(uint4 *)(held_s[i] + off) = v;
+        else __stcs((uint4 *)(held_s[i] + off), v);
+    }
     if (n2 == 0) return;
     // second level: every relay's copy is read back from where it is held and forwarded
     int k0 = 0;                                         // first forwarded copy of the hops of this batch

@@ -156,3 +156,27 @@ def test_plan_ahead_large_ep_shape_two_words():
             assert np.array_equal(rb.host(), c.want_recv)
             assert sb.guards_intact() and rb.guards_intact()
         assert_plan_equal(ctx.plan_arrays(batches[1].T), batches[1].p, ctx.mw_get_totals())
+
+
+@pytest.mark.parametrize("flags", [mw.MW_FLAG_PLAN_MULTIPASS, mw.MW_FLAG_COPY_BULK | mw.MW_FLAG_NO_OVERLAP])
+def test_plan_ahead_with_the_multi_kernel_plan_and_the_bulk_copy_engine(flags):
+    torch = torch_mod()
+    s, e2r, batches = make_batches(72)
+    B = s.row_bytes
+    with mw.Context(s.R, s.E, s.K, s.T, B, flags=flags) as ctx:
+        ctx.mw_plan_next(batches[0].ids, e2r, batches[0].T)
+        outs = []
+        for i in range(5):
+            cur, nxt = batches[i % 2], batches[(i + 1) % 2]
+            ctx.mw_plan_swap()
+            ctx.mw_plan_next(nxt.ids, e2r, nxt.T)
+            send, recv = Guarded(cur.Tn * B), Guarded(cur.SD * B)
+            ctx.mw_pack(cur.x, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), cur.Tn)
+            ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send.ptr(), recv.ptr(), 0, cur.SD)
+            outs.append((cur, send, recv))
+        torch.cuda.synchronize()
+        for c, sb, rb in outs:
+            assert np.array_equal(sb.host().reshape(-1, B), c.want_send)
+            assert np.array_equal(rb.host(), c.want_recv)
+            assert sb.guards_intact() and rb.guards_intact()
+        assert_plan_equal(ctx.plan_arrays(batches[0].T), batches[0].p, ctx.mw_get_totals())
