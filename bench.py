@@ -1110,6 +1110,8 @@ def run_cuda(args):
         dram = (alg["pack"] + roof["traffic"]) / (p_ms + d_ms) / 1e6
         stages["pack_plus_deliver_dram_gbs"] = round(dram, 1)
         stages["pack_plus_deliver_dram_frac_of_nominal_8TBs"] = round(dram / NOMINAL_HBM_GBS, 4)
+        # the whole step in DRAM bytes (plan traffic is under 1 MB): what `value` is in the other byte counting
+        stages["step_dram_gbs"] = round((alg["pack"] + roof["traffic"]) / (ms_per_step * 1e-3) / 1e9, 1)
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
