@@ -82,6 +82,7 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.copy_ctr = k.take<unsigned int>(2);
     d.acc = k.take<mw_acc>(2);
     d.gave_up = k.take<unsigned int>(1);
+    d.gm_tile_rec = k.take<unsigned long long>((size_t)32 * R);
     c->scratch_bytes = k.used - scratch_from;
     {   // the second slot shares everything that is not a plan array
         mw_dev &o = c->other.d;
@@ -90,7 +91,7 @@ size_t carve(mw_ctx *c, uint8_t *base)
         o.gm_tile_sum = d.gm_tile_sum; o.ex_tile_cnt = d.ex_tile_cnt;
         o.slot_key = d.slot_key; o.slot_leader = d.slot_leader; o.slot_count = d.slot_count;
         o.tile_state = d.tile_state; o.tile_agg = d.tile_agg; o.ticket = d.ticket; o.gbar = d.gbar;
-        o.copy_ctr = d.copy_ctr; o.acc = d.acc; o.gave_up = d.gave_up;
+        o.copy_ctr = d.copy_ctr; o.acc = d.acc; o.gave_up = d.gave_up; o.gm_tile_rec = d.gm_tile_rec;
     }
     if (c->cfg.flags & MW_FLAG_HOST_STAGING) {
         const size_t B = (size_t)c->cfg.row_bytes;
@@ -157,7 +158,7 @@ int init_scratch(mw_ctx *c)
     c->epoch = 0; c->tickets_used = 0; c->gbar_arrivals = 0;
     c->planned_T = -1; c->prefetched = nullptr; c->plan_epoch = 0;
     c->other.planned_T = -1; c->other.prefetched = nullptr; c->other.plan_epoch = 0;
-    c->next_pending = 0; c->plans_on_side_stream = 0; c->gm_epoch = 0;
+    c->next_pending = 0; c->plans_on_side_stream = 0; c->gm_epoch = 0; c->gm_calls = 0;
     c->test_skew = 0; c->poisoned = 0;
     return MW_OK;
 }

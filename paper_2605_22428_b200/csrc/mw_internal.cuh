@@ -41,6 +41,7 @@ struct mw_dev {
     int32_t *row_dest_pos_gm;       // [Kd, Tm] the same per send row, plane layout
     int32_t *row_dest_flat_gm;      // [Kd, Tm] row of the compact receive area per send row and destination
     int32_t *gm_tile_sum;           // [max_tiles, R] rows each tile of 256 groups adds to each region
+    unsigned long long *gm_tile_rec;   // [32, R] the same as (call number, value) records, for the one-kernel route
     int32_t *ex_tile_cnt;           // [max_tiles, E] tokens of each tile that selected each expert (nullptr: too large)
     // scratch
     unsigned long long *slot_key;                  // [HS] open-addressed table keyed by bitmap: (hash tag, first token)
@@ -91,6 +92,7 @@ struct mw_ctx {
     uint32_t test_skew;     // MW_TEST_SKEW_* bits applied to the next launch (mw_test_skew_waits)
     int poisoned;           // a wait gave up: host counters and device scratch may be out of step until mw_reset
     uint32_t gm_epoch;      // epoch of the plan the group-major arrays were made from (0: none)
+    uint32_t gm_calls;      // mw_group_major calls so far (tags the per-tile records of the one-kernel route)
     int32_t relay_src, relay_P;   // relay_P > 0: plans map every rank to its next hop as seen from rank relay_src (servers of relay_P ranks)
     int64_t launches;
     // host staging (MW_FLAG_HOST_STAGING)

@@ -11,9 +11,9 @@
 // tokens, done as a bit matrix (expert x token of the tile) plus per-tile counts.
 //
 // Both are small integer passes over the plan (kilobytes to a few megabytes), bound by launch and memory latency,
-// not by bandwidth, so each runs as two short kernels of one block per 256 groups / tokens: per-tile counts, then
-// everything else, every block summing the counts of the tiles before it by itself (up to 32 tiles; beyond that a
-// scan kernel sits between the two).
+// not by bandwidth.  Up to 32 tiles of 256 groups / tokens the group-major arrays take one kernel (every tile publishes
+// its per-rank sums and adds up those of the tiles before it) and the expert index two (per-tile counts, then everything
+// else, every block summing the earlier tiles' counts by itself); beyond that, a scan kernel sits in between.
 #include <string.h>
 
 #include "mw_internal.cuh"
@@ -29,6 +29,8 @@ struct GmArgs {
     int R, W, Kd, Tm, T;
     int tiles;                 // tiles launched (covers every possible G)
     int stash;                 // k_gm_fill keeps the tile's (rank, block start) rows in shared memory as well (Kd <= 16)
+    uint32_t call;             // number of this mw_group_major call on the context (tags the per-tile records, never 0)
+    int spin_limit;            // polls before a tile gives up waiting for an earlier tile's record
 };
 
 // Per tile of 256 groups and per rank: rows the tile's groups add to the rank's region.
@@ -37,8 +39,6 @@ __global__ void __launch_bounds__(kTile) k_gm_sum(GmArgs a)
     extern __shared__ uint64_t sm64[];
     uint64_t *mask = sm64;                          // [kTile, W]
     int *size = (int *)(mask + (size_t)kTile * a.W);  // [kTile]
-    grid_dependency_wait();        // launched as a programmatic dependent: only its start-up overlaps the kernel before it
-    grid_launch_dependents();      // k_gm_fill may start: all it does before its grid_dependency_wait() depends on the plan only
     const int status = a.d.totals->status, G = (int)a.d.totals->G;      // both before the first branch: one round trip
     if (status == MW_ERR_TIMEOUT) return;
     const int g0 = blockIdx.x * kTile;
@@ -76,15 +76,19 @@ __global__ void __launch_bounds__(kTile) k_gm_scan(GmArgs a)
     }
 }
 
+constexpr int kFillThreads = 1024;  // k_gm_fill: 32 warps share the ranks of the tile (the per-rank walk is a chain of warp scans)
 constexpr int kFuseTiles = 32;     // up to this many tiles every block adds up the earlier tiles' counts itself
 
 // Per tile of 256 groups: the warp of rank r walks the tile's groups in order and hands every group that contains r
 // its block of the region; then the block's threads take the send rows of those groups (they are consecutive) and
 // give every member token its slots, per token and per send row (plane layout, for the deliver kernel).
-// SCANNED: gm_tile_sum already holds the exclusive prefix over tiles (k_gm_scan ran); else the raw per-tile sums.
+// SCANNED: gm_tile_sum already holds the exclusive prefix over tiles (k_gm_sum and k_gm_scan ran before).  Otherwise
+// this is the only kernel: every tile first publishes its own per-rank sums as one 64-bit record each (call number,
+// value), then adds up the records of the tiles before it, waiting (with a limit) for those not yet there; a tile
+// only waits for tiles with a smaller block index, and at most kFuseTiles blocks exist, all resident.
 // The block with index b also marks the tokens [256 b, 256 b + 256) that have no destination.
 template <bool SCANNED>
-__global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
+__global__ void __launch_bounds__(kFillThreads) k_gm_fill(GmArgs a)
 {
     extern __shared__ uint64_t sm64[];
     uint64_t *mask = sm64;
@@ -94,21 +98,22 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
     int *rank_s = region_s + a.R + 1;                     // [kTile, Kd] (stash) destination ranks of the tile's groups
     int *start_s = rank_s + (a.stash ? kTile * a.Kd : 0); // [kTile, Kd] (stash) start of each group's block in that region
     __shared__ int gstart[kTile + 1];
+    if (!SCANNED) grid_dependency_wait();    // launched as a programmatic dependent: only its start-up overlaps the kernel before it
     if (a.d.totals->status == MW_ERR_TIMEOUT) return;
     {   // tokens without destinations belong to no group: their slots are -1
         const int t = blockIdx.x * kTile + threadIdx.x;
-        if (t < a.T && a.d.token_group[t] < 0)
+        if (threadIdx.x < kTile && t < a.T && a.d.token_group[t] < 0)
             for (int i = 0; i < a.Kd; ++i) a.d.dest_pos_gm[(size_t)t * a.Kd + i] = -1;
     }
     const int G = (int)a.d.totals->G;
     const int g0 = blockIdx.x * kTile;
     const int n = min(kTile, G - g0);
     if (n <= 0) return;
-    for (int i = threadIdx.x; i < n * a.W; i += kTile) mask[i] = a.d.group_mask[(size_t)g0 * a.W + i];
+    for (int i = threadIdx.x; i < n * a.W; i += kFillThreads) mask[i] = a.d.group_mask[(size_t)g0 * a.W + i];
     if (threadIdx.x < n) gstart[threadIdx.x] = a.d.group_offsets[g0 + threadIdx.x];
     if (threadIdx.x == 0) gstart[n] = a.d.group_offsets[g0 + n];
     __syncthreads();
-    for (int r = threadIdx.x; r <= a.R; r += kTile) region_s[r] = a.d.rank_offsets[r];
+    for (int r = threadIdx.x; r <= a.R; r += kFillThreads) region_s[r] = a.d.rank_offsets[r];
     // the token of this thread's first send row (the member-token part below starts with it)
     const int first_row = gstart[0] + threadIdx.x;
     const int first_token = first_row < gstart[n] ? a.d.mw_row_token[first_row] : -1;
@@ -120,28 +125,52 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
             if (a.stash) rank_s[threadIdx.x * a.Kd + i] = -1;
         }
     }
-    // Everything above needs the plan only and has run while the kernel before this one (the per-tile sums, or their
-    // scan) was still at work; its results are needed from here on.
-    grid_dependency_wait();
-    // rows the earlier tiles put into every region: all ranks at once (independent, coalesced loads), not rank by rank
-    for (int r = threadIdx.x; r < a.R; r += kTile) {
-        int before = 0;
-        if (SCANNED) before = a.d.gm_tile_sum[(size_t)blockIdx.x * a.R + r];
-        else
-            for (int t0 = 0; t0 < (int)blockIdx.x; t0 += 8) {             // eight independent loads per round trip
-                int v[8];
+    const int lane = threadIdx.x & 31;
+    if (SCANNED) {
+        // Everything above needs the plan only and has run while the scan of the per-tile sums was still at work.
+        grid_dependency_wait();
+        for (int r = threadIdx.x; r < a.R; r += kFillThreads) before_s[r] = a.d.gm_tile_sum[(size_t)blockIdx.x * a.R + r];
+    } else {
+        __syncthreads();                                  // bitmaps and sizes are in shared memory
+        // this tile's rows per region: one warp per rank, lanes stride the groups; published at once
+        for (int r = threadIdx.x >> 5; r < a.R; r += kFillThreads / 32) {
+            int sum = 0;
+            for (int j = lane; j < n; j += 32)
+                if (bit_of(mask + (size_t)j * a.W, r)) sum += size[j];
+            sum = __reduce_add_sync(0xffffffffu, sum);
+            if (lane == 0)
+                *(volatile unsigned long long *)(a.d.gm_tile_rec + (size_t)blockIdx.x * a.R + r) =
+                    ((unsigned long long)a.call << 32) | (uint32_t)sum;
+        }
+        // rows the earlier tiles put into every region: all ranks at once, eight records per round trip
+        for (int r = threadIdx.x; r < a.R; r += kFillThreads) {
+            int before = 0;
+            bool gave_up = false;
+            for (int t0 = 0; t0 < (int)blockIdx.x && !gave_up; t0 += 8) {
+                unsigned long long v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = t0 + u < (int)blockIdx.x ? a.d.gm_tile_sum[(size_t)(t0 + u) * a.R + r] : 0;
+                for (int u = 0; u < 8; ++u)
+                    v[u] = t0 + u < (int)blockIdx.x ? *(volatile unsigned long long *)(a.d.gm_tile_rec + (size_t)(t0 + u) * a.R + r)
+                                                    : ((unsigned long long)a.call << 32);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) before += v[u];
+                for (int u = 0; u < 8; ++u) {
+                    int spins = 0;
+                    while ((uint32_t)(v[u] >> 32) != a.call) {                // not this call's record yet
+                        if (++spins > a.spin_limit) { gave_up = true; break; }
+                        __nanosleep(64);
+                        v[u] = *(volatile unsigned long long *)(a.d.gm_tile_rec + (size_t)(t0 + u) * a.R + r);
+                    }
+                    before += (int)(uint32_t)v[u];
+                }
             }
-        before_s[r] = before;
+            if (gave_up) atomicCAS(&a.d.totals->status, 0, MW_ERR_TIMEOUT);
+            before_s[r] = before;
+        }
     }
     __syncthreads();
     // one warp per rank, 32 groups of the tile per round (lane l takes group 32 k + l, so neighbouring lanes read
     // neighbouring bitmaps): an exclusive scan over the lanes gives each group that contains r the start of its block
-    const int lane = threadIdx.x & 31;
-    for (int r = threadIdx.x >> 5; r < a.R; r += kTile / 32) {
+    for (int r = threadIdx.x >> 5; r < a.R; r += kFillThreads / 32) {
         int run = before_s[r];
         for (int j0 = 0; j0 < n; j0 += 32) {
             const int j = j0 + lane;
@@ -163,7 +192,7 @@ __global__ void __launch_bounds__(kTile) k_gm_fill(GmArgs a)
     }
     __syncthreads();                                      // the tile's gm_rank / gm_offset rows are complete (and visible to the block)
     // member tokens: send rows [gstart[0], gstart[n]) belong to the tile's groups, in group order
-    for (int row = gstart[0] + threadIdx.x; row < gstart[n]; row += kTile) {
+    for (int row = gstart[0] + threadIdx.x; row < gstart[n]; row += kFillThreads) {
         int lo = 0, hi = n;                               // group of the row: the last j with gstart[j] <= row
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -411,13 +440,19 @@ extern "C" int mw_group_major(mw_ctx *ctx, mw_group_major_view *view, void *stre
     a.stash = gm_stash(ctx) ? 1 : 0;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t smem = gm_smem(ctx);
-    mw_launch(k_gm_sum, dim3(a.tiles), dim3(kTile), smem, st, true, a);
+    if (++ctx->gm_calls == 0) {                         // the records' 32-bit call number starts a new lap: wipe the old lap
+        ctx->gm_calls = 1;
+        if (cudaMemsetAsync(ctx->d.gm_tile_rec, 0, sizeof(unsigned long long) * (size_t)kFuseTiles * a.R, st) != cudaSuccess) return MW_ERR_CUDA;
+    }
+    a.call = ctx->gm_calls;
+    a.spin_limit = ctx->spin_limit;
     if (a.tiles <= kFuseTiles) {
-        mw_launch(k_gm_fill<false>, dim3(a.tiles), dim3(kTile), smem, st, true, a);
-        ctx->launches += 2;
+        mw_launch(k_gm_fill<false>, dim3(a.tiles), dim3(kFillThreads), smem, st, true, a);
+        ctx->launches += 1;
     } else {
+        k_gm_sum<<<a.tiles, kTile, smem, st>>>(a);
         k_gm_scan<<<(a.R + kTile - 1) / kTile, kTile, 0, st>>>(a);
-        mw_launch(k_gm_fill<true>, dim3(a.tiles), dim3(kTile), smem, st, true, a);
+        mw_launch(k_gm_fill<true>, dim3(a.tiles), dim3(kFillThreads), smem, st, true, a);
         ctx->launches += 3;
     }
     return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
