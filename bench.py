@@ -875,7 +875,7 @@ def order_measure(mw, wl, torch) -> dict:
         assert ctx.mw_get_totals()["status"] == 0
     out["deliver_group_major_gbs"] = round((Tn + SD) * B / out["deliver_group_major_us"] / 1e3, 1)
     out["groups"] = tot["G"]
-    out["note"] = "2 + 2 short kernels over the plan (latency-bound); the deliver is the same row-copy kernel with other slots"
+    out["note"] = "1 + 2 short kernels over the plan (latency-bound); the deliver is the same row-copy kernel with other slots"
     return out
 
 
