@@ -180,3 +180,32 @@ def test_plan_ahead_with_the_multi_kernel_plan_and_the_bulk_copy_engine(flags):
             assert np.array_equal(rb.host(), c.want_recv)
             assert sb.guards_intact() and rb.guards_intact()
         assert_plan_equal(ctx.plan_arrays(batches[0].T), batches[0].p, ctx.mw_get_totals())
+
+
+def test_plan_ahead_with_an_empty_batch_and_a_reset_in_between():
+    torch = torch_mod()
+    s, e2r, (a, b) = make_batches(24)
+    B = s.row_bytes
+    none = torch.zeros((0, s.K), dtype=torch.int32, device="cuda")
+    buf = torch.zeros(1 << 12, dtype=torch.uint8, device="cuda")
+    with mw.Context(s.R, s.E, s.K, s.T, B) as ctx:
+        ctx.mw_plan_next(a.ids, e2r, a.T)
+        ctx.mw_plan_swap()
+        ctx.mw_plan_next(none, e2r, 0)                                    # an empty batch is a plan like any other
+        send, recv = Guarded(a.Tn * B), Guarded(a.SD * B)
+        ctx.mw_pack(a.x, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), a.Tn)
+        ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send.ptr(), recv.ptr(), 0, a.SD)
+        assert np.array_equal(recv.host(), a.want_recv) and recv.guards_intact()
+        ctx.mw_plan_swap()
+        tot = ctx.mw_get_totals()
+        assert tot["T_nonempty"] == 0 and tot["total_dest"] == 0 and tot["G"] == 0 and tot["status"] == 0
+        ctx.mw_pack(buf, mw.MW_LAYOUT_MULTIWRITE, buf, 0)                   # nothing to move
+        ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, buf, buf, 0, 0)
+        assert not buf.any()
+        # a reset drops an outstanding plan as well
+        ctx.mw_plan_next(b.ids, e2r, b.T)
+        ctx.mw_reset()
+        assert ctx.mw_plan_swap(check=False) == mw.MW_ERR_NO_PLAN
+        ctx.mw_plan_next(b.ids, e2r, b.T)
+        ctx.mw_plan_swap()
+        assert_plan_equal(ctx.plan_arrays(b.T), b.p, ctx.mw_get_totals())
