@@ -148,8 +148,8 @@ MW_API int mw_destroy(mw_ctx *ctx);
 
 /*
  * Makes a context usable again after MW_ERR_TIMEOUT.  The device-side waits of this library (a plan tile waiting
- * for the counts of the tiles before it, a plan block waiting at a grid barrier, a copy pipeline waiting for a
- * bulk load) are bounded; when one gives up, mw_totals.status says MW_ERR_TIMEOUT, the kernels that follow skip
+ * for the counts of the tiles before it, a plan block waiting at a grid barrier, a tile of mw_group_major waiting
+ * for the sums of the tiles before it, a copy pipeline waiting for a bulk load) are bounded; when one gives up, mw_totals.status says MW_ERR_TIMEOUT, the kernels that follow skip
  * their work, and from the mw_get_totals that reported it every call on the context except mw_get_totals,
  * mw_reset and mw_destroy returns MW_ERR_TIMEOUT.  (A plan can run into this when other work keeps the GPU's SMs
  * occupied for about a second, so that its blocks cannot all become resident.)  mw_reset waits for the device,
