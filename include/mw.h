@@ -528,12 +528,14 @@ MW_API int mw_read_device(mw_ctx *ctx, void *host_dst, const void *device_src, i
  *   MW_TEST_SKEW_BARRIER    the next fused plan's grid barriers wait for one arrival more than there are blocks
  *   MW_TEST_SKEW_BULK_LOAD  the next launch of the bulk-copy engine announces every load 16 bytes too large, so
  *                           no pipeline stage ever completes
+ *   MW_TEST_SKEW_GROUP_MAJOR the next mw_group_major's tiles look for records of another call
  * Use with MW_FLAG_SHORT_WAITS, or each wait takes about a second to give up.  The outcome is MW_ERR_TIMEOUT in
  * mw_totals.status; recover with mw_reset.
  */
 #define MW_TEST_SKEW_LOOKBACK  0x1u
 #define MW_TEST_SKEW_BARRIER   0x2u
 #define MW_TEST_SKEW_BULK_LOAD 0x4u
+#define MW_TEST_SKEW_GROUP_MAJOR 0x8u
 MW_API int mw_test_skew_waits(mw_ctx *ctx, uint32_t what);
 
 /* Number of kernels this context has launched since mw_create (for launch accounting). */

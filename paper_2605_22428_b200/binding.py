@@ -32,6 +32,7 @@ MW_FLAG_SHORT_WAITS = 0x80
 MW_TEST_SKEW_LOOKBACK = 0x1
 MW_TEST_SKEW_BARRIER = 0x2
 MW_TEST_SKEW_BULK_LOAD = 0x4
+MW_TEST_SKEW_GROUP_MAJOR = 0x8
 
 RELAY_EXPORTS = ("mw_relay_create", "mw_relay_destroy", "mw_relay_reset", "mw_relay_plan", "mw_relay_get_totals", "mw_relay_dispatch",
                  "mw_relay_contexts")

@@ -275,7 +275,7 @@ int mw_reset(mw_ctx *ctx)
 
 int mw_test_skew_waits(mw_ctx *ctx, uint32_t what)
 {
-    if (!ctx || (what & ~(MW_TEST_SKEW_LOOKBACK | MW_TEST_SKEW_BARRIER | MW_TEST_SKEW_BULK_LOAD))) return MW_ERR_INVALID_ARG;
+    if (!ctx || (what & ~(MW_TEST_SKEW_LOOKBACK | MW_TEST_SKEW_BARRIER | MW_TEST_SKEW_BULK_LOAD | MW_TEST_SKEW_GROUP_MAJOR))) return MW_ERR_INVALID_ARG;
     ctx->test_skew = what;
     return MW_OK;
 }

@@ -30,6 +30,7 @@ struct GmArgs {
     int tiles;                 // tiles launched (covers every possible G)
     int stash;                 // k_gm_fill keeps the tile's (rank, block start) rows in shared memory as well (Kd <= 16)
     uint32_t call;             // number of this mw_group_major call on the context (tags the per-tile records, never 0)
+    uint32_t wait_call;        // tag a tile expects in the records of the tiles before it (= call, unless a test skews it)
     int spin_limit;            // polls before a tile gives up waiting for an earlier tile's record
 };
 
@@ -151,11 +152,11 @@ __global__ void __launch_bounds__(kFillThreads) k_gm_fill(GmArgs a)
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
                     v[u] = t0 + u < (int)blockIdx.x ? *(volatile unsigned long long *)(a.d.gm_tile_rec + (size_t)(t0 + u) * a.R + r)
-                                                    : ((unsigned long long)a.call << 32);
+                                                    : ((unsigned long long)a.wait_call << 32);
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     int spins = 0;
-                    while ((uint32_t)(v[u] >> 32) != a.call) {                // not this call's record yet
+                    while ((uint32_t)(v[u] >> 32) != a.wait_call) {           // not this call's record yet
                         if (++spins > a.spin_limit) { gave_up = true; break; }
                         __nanosleep(64);
                         v[u] = *(volatile unsigned long long *)(a.d.gm_tile_rec + (size_t)(t0 + u) * a.R + r);
@@ -445,6 +446,8 @@ extern "C" int mw_group_major(mw_ctx *ctx, mw_group_major_view *view, void *stre
         if (cudaMemsetAsync(ctx->d.gm_tile_rec, 0, sizeof(unsigned long long) * (size_t)kFuseTiles * a.R, st) != cudaSuccess) return MW_ERR_CUDA;
     }
     a.call = ctx->gm_calls;
+    a.wait_call = (ctx->test_skew & MW_TEST_SKEW_GROUP_MAJOR) ? a.call + 0x40000000u : a.call;    // records nobody writes
+    ctx->test_skew &= ~(uint32_t)MW_TEST_SKEW_GROUP_MAJOR;
     a.spin_limit = ctx->spin_limit;
     if (a.tiles <= kFuseTiles) {
         mw_launch(k_gm_fill<false>, dim3(a.tiles), dim3(kFillThreads), smem, st, true, a);

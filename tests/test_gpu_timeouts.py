@@ -128,6 +128,32 @@ def test_bulk_copy_wait_runs_out_then_reset_recovers():
         dispatch_and_check(ctx, inp, p, ids, e2r, x)
 
 
+def test_group_major_wait_runs_out_then_reset_recovers():
+    inp, p, ids, e2r, x = setup()
+    B = inp.shape.row_bytes
+    Tn, SD = p.totals["T_nonempty"], p.totals["total_dest"]
+    gdr, gdo, gm = mwo.group_major(p)
+    with mw.Context(64, 256, 8, 2000, B, flags=mw.MW_FLAG_SHORT_WAITS) as ctx:
+        ctx.mw_plan(ids, e2r, inp.T)
+        _, view = ctx.mw_group_major()
+        got = ctx.group_major_arrays(inp.T, p.totals["G"], view)
+        assert np.array_equal(got["group_dest_offset"], gdo) and np.array_equal(got["dest_pos_gm"], gm)
+        ctx.mw_test_skew_waits(mw.MW_TEST_SKEW_GROUP_MAJOR)
+        ctx.mw_group_major()                                                # tiles after the first wait for records nobody writes
+        send, recv = Guarded(Tn * B), Guarded(SD * B)
+        ctx.mw_deliver_group_major(send.ptr(), recv.ptr(), 0, SD)           # must skip
+        assert ctx.mw_get_totals()["status"] == mw.MW_ERR_TIMEOUT
+        assert untouched(recv)
+        assert ctx.mw_group_major(check=False)[0] == mw.MW_ERR_TIMEOUT
+        ctx.mw_reset()
+        ctx.mw_plan(ids, e2r, inp.T)
+        _, view = ctx.mw_group_major()
+        got = ctx.group_major_arrays(inp.T, p.totals["G"], view)
+        assert np.array_equal(got["group_dest_rank"], gdr) and np.array_equal(got["group_dest_offset"], gdo)
+        assert np.array_equal(got["dest_pos_gm"], gm)
+        assert ctx.mw_get_totals()["status"] == 0
+
+
 def test_reset_on_a_healthy_context_and_argument_checks():
     inp, p, ids, e2r, x = setup(T=300)
     with mw.Context(64, 256, 8, 512, inp.shape.row_bytes) as ctx:
