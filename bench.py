@@ -6,7 +6,7 @@ layout, all through the C ABI, inputs resident in device memory.  The workload i
 DeepSeek-V3-shaped prefill dispatch (64 ranks, 256 experts, top-8, 4096 tokens, 7168 bf16 per row).
 The step cycles over several buffer sets so that every step's inputs and outputs come from HBM,
 not L2.  Prints one JSON line: the headline keys first, then the blocks for the other shapes and paths; the
-last keys are tiny, unicast, large_ep, pipelined, bytes_saved_pct and decode.
+last keys are tiny, unicast, large_ep, pipelined, bytes_saved_pct, decode and a compact metric_summary.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
 
@@ -377,10 +377,8 @@ def decode_latency(mw, wl, torch, launches: int = 1000) -> dict:
         out["one_call_graph_chained"] = {"p50_us": round(percentile(us, 0.5), 2), "calls_per_graph": n_chain}
         assert ctx.mw_get_totals()["status"] == 0
     out["launches"] = launches
-    out["note"] = ("L2-resident working set (0.9 MB in, 7.3 MB out): a latency figure, not an HBM fraction; chain = "
-                   "mw_plan + mw_dispatch (2 launches: mw_dispatch packs and delivers in one pass), one_call = mw_plan_dispatch (1 launch); each figure includes "
-                   "the host's launch cost through the Python binding, except one_call_graph (the same call replayed from a "
-                   "CUDA graph, one call per graph) and one_call_graph_chained (20 calls per graph, time per call)")
+    out["note"] = ("L2-resident (0.9 MB in, 7.3 MB out): latency, not an HBM fraction; chain = mw_plan + mw_dispatch, one_call = "
+                   "mw_plan_dispatch (1 launch); host launch cost included except in the graph replays (chained: 20 calls per graph)")
     return out
 
 
@@ -732,8 +730,7 @@ def pipelined_measure(mw, wl, torch, name: str, steps: int = 400) -> dict:
             "step_p99_us": round(percentile(per_step, 0.99), 2), "batch_latency_p50_us": round(statistics.median(latency), 2),
             "step_gbs": round(nbytes / us / 1e3, 1), "frac_of_measured_peak": round(nbytes / us / 1e3 / measured_peak()[0], 4),
             "tokens_per_s": round(T / us * 1e6, 1),
-            "note": "one context, one caller stream; mw_plan_swap + mw_plan_next + mw_pack + mw_deliver per step; the plan runs on "
-                    "the library's planning stream under the previous batch's copies; latency = plan may start -> deliver done"}
+            "note": "one context, one caller stream: mw_plan_swap + mw_plan_next + mw_pack + mw_deliver per step; latency = plan may start -> deliver done"}
 
 
 def unicast_measure(mw, wl, torch, name: str, n: int = 100) -> dict:
@@ -781,7 +778,7 @@ def unicast_measure(mw, wl, torch, name: str, n: int = 100) -> dict:
     u, m = out["unicast"], out["multiwrite"]
     out["time_saved_pct"] = round(100 * (1 - m["step_us"] / u["step_us"]), 2)
     out["transmitted_bytes_saved_pct"] = round(100.0 * (1 - tot["mw_bytes"] / tot["unicast_bytes"]), 3)
-    out["note"] = "p50 of CUDA events around each call over %d steps; one GPU emulates every link, so time follows bytes moved in HBM" % n
+    out["note"] = "p50 of CUDA events around each call, %d steps; one GPU emulates every link: time follows bytes moved in HBM" % n
     return out
 
 
@@ -1157,6 +1154,27 @@ def run_cuda(args):
             line["pipelined"] = {name: pipelined_measure(mw, wl, torch, name) for name in (WORKLOAD, "large_ep")}
             line["bytes_saved_pct"] = bytes_saved(wl)
             line["decode"] = decode_latency(mw, wl, torch)
+            # the three parts of the metric once more, compactly, as the very end of the line
+            dec, pipe, uni, lep = line["decode"], line["pipelined"], line["unicast"], line["large_ep"]
+            line["metric_summary"] = {
+                "pack_plus_deliver_gbs": {WORKLOAD: stages["pack_plus_deliver_gbs"], "large_ep": lep["pack_plus_deliver_gbs"]},
+                "pack_plus_deliver_pct_of_measured_peak": {WORKLOAD: round(100 * stages["pack_plus_deliver_gbs"] / peak, 1),
+                                                           "large_ep": round(100 * lep["pack_plus_deliver_gbs"] / peak, 1)},
+                "pack_plus_deliver_pct_of_nominal_8TBs": {WORKLOAD: round(100 * stages["pack_plus_deliver_gbs"] / NOMINAL_HBM_GBS, 1),
+                                                          "large_ep": round(100 * lep["pack_plus_deliver_gbs"] / NOMINAL_HBM_GBS, 1)},
+                "pack_plus_deliver_dram_pct_of_nominal_8TBs": round(100 * stages.get("pack_plus_deliver_dram_frac_of_nominal_8TBs", 0), 1) or None,
+                "deliver_roofline_frac": {WORKLOAD: roof["frac"], "large_ep": lep["roofline"]["frac"]},
+                "deliver_dram_frac": {WORKLOAD: roof.get("dram_frac"), "large_ep": lep["roofline"].get("dram_frac")},
+                "step_us": {WORKLOAD: round(ms_per_step * 1e3, 2), "large_ep": lep["step_us"]},
+                "pipelined_step_p50_us": {k: v["step_p50_us"] for k, v in pipe.items()},
+                "unicast_vs_multiwrite_step_us": {k: [v["unicast"]["step_us"], v["multiwrite"]["step_us"]] for k, v in uni.items()},
+                "tokens_per_s": line["tokens_per_s"],
+                "decode_us": {"one_call_p50": dec["one_call"]["p50_us"], "one_call_p99": dec["one_call"]["p99_us"],
+                              "graph_p50": dec["one_call_graph"]["p50_us"], "graph_p99": dec["one_call_graph"]["p99_us"],
+                              "graph_chained_per_call": dec["one_call_graph_chained"]["p50_us"],
+                              "plan_p50": dec["plan"]["p50_us"], "three_launch_chain_p50": dec["chain"]["p50_us"]},
+                "tiny_one_call_p50_us": line["tiny"]["one_call"]["p50_us"],
+                "bytes_saved_pct": line["bytes_saved_pct"]}
     if rank == 0:
         print(json.dumps(line))
     if dist:
