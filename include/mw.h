@@ -153,7 +153,7 @@ MW_API int mw_destroy(mw_ctx *ctx);
  * their work, and from the mw_get_totals that reported it every call on the context except mw_get_totals,
  * mw_reset and mw_destroy returns MW_ERR_TIMEOUT.  (A plan can run into this when other work keeps the GPU's SMs
  * occupied for about a second, so that its blocks cannot all become resident.)  mw_reset waits for the device,
- * empties the scratch the plans share and rewinds the host-side counters; no plan exists afterwards (the next
+ * empties the scratch the plans share (their running counts included); no plan exists afterwards (the next
  * call must be a plan).  Nothing is reallocated.  Synchronous.
  */
 MW_API int mw_reset(mw_ctx *ctx);
@@ -275,8 +275,10 @@ MW_API int mw_dispatch(mw_ctx *ctx, const void *x, int layout, void *send_buf, i
  * batches, the unicast layout and contexts created with MW_FLAG_PLAN_MULTIPASS take the
  * ordinary three-kernel route (planning through mw_plan_prefetch).
  * The single launch keeps no state on the host, so a call captured into a CUDA graph may be replayed
- * (new ids and rows in the same buffers).  mw_plan and mw_plan_prefetch may not: the look-back epoch
- * and the barrier targets of their kernel are launch arguments that advance with every call.
+ * (new ids and rows in the same buffers).  So may mw_plan / mw_plan_prefetch followed by mw_pack, mw_deliver or
+ * mw_dispatch: the running counts of the tiled plan (epoch of its look-back records, barrier arrivals, tile tickets)
+ * live on the device and are advanced by the plan kernels themselves.  (mw_plan_next / mw_plan_swap use a second
+ * stream and events; capturing them is not covered here.)
  */
 MW_API int mw_plan_dispatch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_to_rank, int32_t T,
                             const void *x, int layout, void *send_buf, int64_t send_capacity_rows, void *recv_base,

@@ -83,6 +83,7 @@ size_t carve(mw_ctx *c, uint8_t *base)
     d.acc = k.take<mw_acc>(2);
     d.gave_up = k.take<unsigned int>(1);
     d.gm_tile_rec = k.take<unsigned long long>((size_t)32 * R);
+    d.plan_state = k.take<mw_plan_state>(1);
     c->scratch_bytes = k.used - scratch_from;
     {   // the second slot shares everything that is not a plan array
         mw_dev &o = c->other.d;
@@ -91,7 +92,7 @@ size_t carve(mw_ctx *c, uint8_t *base)
         o.gm_tile_sum = d.gm_tile_sum; o.ex_tile_cnt = d.ex_tile_cnt;
         o.slot_key = d.slot_key; o.slot_leader = d.slot_leader; o.slot_count = d.slot_count;
         o.tile_state = d.tile_state; o.tile_agg = d.tile_agg; o.ticket = d.ticket; o.gbar = d.gbar;
-        o.copy_ctr = d.copy_ctr; o.acc = d.acc; o.gave_up = d.gave_up; o.gm_tile_rec = d.gm_tile_rec;
+        o.copy_ctr = d.copy_ctr; o.acc = d.acc; o.gave_up = d.gave_up; o.gm_tile_rec = d.gm_tile_rec; o.plan_state = d.plan_state;
     }
     if (c->cfg.flags & MW_FLAG_HOST_STAGING) {
         const size_t B = (size_t)c->cfg.row_bytes;
@@ -147,15 +148,15 @@ void swap_slots(mw_ctx *ctx)
     ctx->other = cur;
 }
 
-// Brings the scratch that all plans share (bitmap table, look-back records, counters, accumulators) and the
-// host-side running counts back to their initial state.  The device must be idle as far as this context goes.
+// Brings the scratch that all plans share (bitmap table, look-back records, counters and running counts, accumulators)
+// and the host-side bookkeeping back to their initial state.  The device must be idle as far as this context goes.
 int init_scratch(mw_ctx *c)
 {
     if (cudaMemset(c->scratch_begin, 0, c->scratch_bytes) != cudaSuccess) return MW_ERR_CUDA;
     k_fill_i32<<<64, 256>>>((int32_t *)c->d.slot_key, 2 * (int64_t)c->HS, -1);   // all ones = empty slot
     k_fill_i32<<<64, 256>>>(c->d.slot_leader, c->HS, 0x7fffffff);                 // no leader
     if (cudaDeviceSynchronize() != cudaSuccess) return MW_ERR_CUDA;
-    c->epoch = 0; c->tickets_used = 0; c->gbar_arrivals = 0;
+    c->epoch = 0;
     c->planned_T = -1; c->prefetched = nullptr; c->plan_epoch = 0;
     c->other.planned_T = -1; c->other.prefetched = nullptr; c->other.plan_epoch = 0;
     c->next_pending = 0; c->plans_on_side_stream = 0; c->gm_epoch = 0; c->gm_calls = 0;

@@ -17,6 +17,13 @@ struct mw_acc {
     int status;                      // first data-dependent error seen while planning
 };
 
+// Running counts of the plans made on a context, kept on the device and advanced by the plan kernels themselves.
+struct mw_plan_state {
+    uint32_t plans;      // plans completed (the next plan's epoch is this + 1)
+    uint32_t tickets;    // tile tickets handed out by all multi-kernel plans so far
+    uint32_t bars;       // grid-barrier arrivals made by all fused plans so far
+};
+
 // Device workspace (all pointers into one slab owned by the context).
 struct mw_dev {
     // public plan arrays (exposed through mw_plan_view)
@@ -53,6 +60,7 @@ struct mw_dev {
     unsigned int *copy_ctr;                        // [2] work-ticket and finished-warp counters of the copy kernels
     mw_acc *acc;                                   // [2]
     unsigned int *gave_up;                         // set by a plan whose wait gave up; later plans refuse to run until mw_reset
+    mw_plan_state *plan_state;                     // running counts of the plans (epoch, tickets, barrier arrivals)
 };
 
 // What the data path needs to know about one plan: where its arrays are and what was planned into them.
@@ -83,9 +91,7 @@ struct mw_ctx {
     void *slab;
     size_t scratch_bytes;   // the part of the slab mw_reset re-initialises starts at scratch_begin
     uint8_t *scratch_begin;
-    uint32_t epoch;         // plans issued so far (tile records carry it, so they need no clearing)
-    uint32_t tickets_used;  // tile tickets handed out by all previous plans
-    uint32_t gbar_arrivals; // grid-barrier arrivals made by all previous fused plans
+    uint32_t epoch;         // plans issued so far: tells on the host which plan a slot holds (the kernels keep their own counts)
     int32_t spin_limit;     // polls a look-back waits for a predecessor's record before it gives up
     int32_t bar_spin_limit; // polls a block waits at a grid barrier
     int32_t copy_wait_limit;// polls (about 1 us each) the bulk-copy engine waits for a load

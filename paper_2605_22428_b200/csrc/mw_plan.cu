@@ -34,8 +34,8 @@ struct PlanArgs {
     int T, K, E, R, W, Kd, src_rank, ntiles, NC, hs_mask, Tm;
     int relay_src, relay_P;   // relay_P > 0: a rank stands for its next hop as seen from relay_src (first level of a relayed dispatch)
     int64_t row_bytes;
-    uint32_t epoch, ticket_base, bar_base;
-    uint32_t wait_epoch;      // epoch a look-back expects in its predecessors' records (= epoch, unless a test skews it)
+    uint32_t skew_epoch;      // test hook: added to the epoch a look-back expects in its predecessors' records (0 normally)
+    uint32_t skew_bar;        // test hook: added to the arrival count the grid barriers wait for (0 normally)
     int spin_limit;           // look-back polls before a tile gives up (2^20: about a second)
     int bar_spin_limit;       // polls of the arrival counter before a block gives up at a grid barrier
     const uint8_t *pf_base;   // rows to bring into L2 while the plan runs (fused plan only), or null
@@ -44,6 +44,46 @@ struct PlanArgs {
 };
 
 __device__ __forceinline__ void set_status(int *status, int err) { atomicCAS(status, 0, err); }
+
+// The running counts of a context's plans live in device memory (mw_dev::plan_state), so that a plan launch carries no
+// host-side state and a captured launch can be replayed: every block reads them when it starts; the plan's last tile
+// advances them when everything that depends on them is done.  Plans of a context never overlap.
+struct PlanCounters {
+    uint32_t epoch;        // number of this plan, 30 bits (look-back records carry it, so they need no clearing)
+    uint32_t wait_epoch;   // epoch expected in predecessors' records
+    uint32_t ticket_base;  // tile tickets handed out by all previous multi-kernel plans
+    uint32_t bar_base;     // grid-barrier arrivals made by all previous fused plans (plus the test skew)
+};
+
+__device__ __forceinline__ PlanCounters load_counters(const PlanArgs &a)
+{
+    const volatile mw_plan_state *st = a.d.plan_state;
+    const uint32_t plans = st->plans, tickets = st->tickets, bars = st->bars;
+    PlanCounters pc;
+    pc.epoch = (plans + 1u) & 0x3fffffffu;
+    pc.wait_epoch = (pc.epoch + a.skew_epoch) & 0x3fffffffu;
+    pc.ticket_base = tickets;
+    pc.bar_base = bars + a.skew_bar;
+    return pc;
+}
+
+// Called by one thread of the plan's last tile, after every block has read the counters.
+__device__ __forceinline__ void advance_counters(const PlanArgs &a, uint32_t tickets_taken, uint32_t barrier_arrivals)
+{
+    mw_plan_state *st = a.d.plan_state;
+    st->plans += 1u;
+    st->tickets += tickets_taken;
+    st->bars += barrier_arrivals;
+}
+
+// The 30-bit epoch is about to start a new lap: the last tile of the lap's last plan wipes the look-back records, once
+// every look-back of the plan is done (all threads of the block call this).
+__device__ __forceinline__ void wipe_records_at_lap_end(const PlanArgs &a, uint32_t epoch)
+{
+    if (epoch != 0x3fffffffu) return;
+    const size_t n = (size_t)((a.Tm + MW_TILE - 1) / MW_TILE) * (size_t)a.NC;
+    for (size_t i = threadIdx.x; i < n; i += blockDim.x) a.d.tile_state[i] = 0ull;
+}
 
 // A wait gave up: the plan under way is invalid, and it will not restore the shared scratch (bitmap table, counters)
 // to the state the next plan expects.  The flag makes every later plan on the context refuse to run until mw_reset
@@ -103,8 +143,9 @@ __device__ __forceinline__ int table_insert_word(unsigned long long *slot_key, i
 __global__ void __launch_bounds__(MW_TILE) k_plan_mask(PlanArgs a)
 {
     if (refuses_to_plan(a)) return;
+    const PlanCounters pc = load_counters(a);
     const int t = blockIdx.x * MW_TILE + threadIdx.x;
-    mw_acc *acc = a.d.acc + (a.epoch & 1u);
+    mw_acc *acc = a.d.acc + (pc.epoch & 1u);
     int valid = 0, self_only = 0, bad = 0;
     if (t < a.T) {
         const int32_t *my = a.ids + (int64_t)t * a.K;
@@ -191,10 +232,11 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
     __shared__ int s_tile;
 
     if (refuses_to_plan(a)) return;
+    const PlanCounters pc = load_counters(a);      // read before the ticket is taken: the tile with the last ticket advances them
     const int tid = threadIdx.x;
-    mw_acc *acc = a.d.acc + (a.epoch & 1u);
+    mw_acc *acc = a.d.acc + (pc.epoch & 1u);
     // Tiles are numbered in the order blocks start, so a tile only ever waits for tiles that are already running.
-    if (tid == 0) s_tile = (int)(atomicAdd(a.d.ticket, 1u) - a.ticket_base);
+    if (tid == 0) s_tile = (int)(atomicAdd(a.d.ticket, 1u) - pc.ticket_base);
     for (int i = tid; i < a.R * 8; i += MW_TILE) bits[i] = 0;
     __syncthreads();
     const int tile = s_tile;
@@ -237,9 +279,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
         volatile unsigned long long *rec = a.d.tile_state + (size_t)tile * a.NC + c;
         uint32_t excl = 0;
         if (tile == 0) {
-            *rec = pack_state(a.epoch, kFlagPrefix, mine);
+            *rec = pack_state(pc.epoch, kFlagPrefix, mine);
         } else {
-            *rec = pack_state(a.epoch, kFlagAgg, mine);
+            *rec = pack_state(pc.epoch, kFlagAgg, mine);
             for (int j = tile - 1; j >= 0; --j) {
                 volatile unsigned long long *prev = a.d.tile_state + (size_t)j * a.NC + c;
                 unsigned long long s = 0;
@@ -247,14 +289,14 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
                 for (; spins < a.spin_limit; ++spins) {
                     s = *prev;
                     const uint32_t hi = (uint32_t)(s >> 32);
-                    if ((hi >> 2) == (a.wait_epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
+                    if ((hi >> 2) == pc.wait_epoch && (hi & 3u) != 0) break;
                     __nanosleep(64);
                 }
                 if (spins == a.spin_limit) { give_up(a, &acc->status); break; }
                 excl += (uint32_t)s;
                 if (((uint32_t)(s >> 32) & 3u) == kFlagPrefix) break;
             }
-            *rec = pack_state(a.epoch, kFlagPrefix, excl + mine);
+            *rec = pack_state(pc.epoch, kFlagPrefix, excl + mine);
         }
         base[c] = (int)excl;
     }
@@ -304,9 +346,11 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_tile(PlanArgs a)
             tt.status = acc->status;
             tt.reserved = 0;
             *a.d.totals = tt;
-            mw_acc *next = a.d.acc + ((a.epoch + 1u) & 1u);
+            mw_acc *next = a.d.acc + ((pc.epoch + 1u) & 1u);
             next->valid_slots = 0; next->self_only = 0; next->status = 0;
+            advance_counters(a, (uint32_t)a.ntiles, 0u);     // every tile has read them (it took its ticket afterwards)
         }
+        wipe_records_at_lap_end(a, pc.epoch);                // this tile's look-back ended last: no record is needed any more
     }
 }
 
@@ -454,7 +498,7 @@ __device__ __forceinline__ unsigned int ld_volatile_u32(const unsigned int *p)
 }
 
 // Grid barrier in two halves, so that work which does not depend on the other blocks can run between
-// them.  Every block always arrives, so the host's running count of arrivals stays exact even after a
+// them.  Every block always arrives, so the running count of arrivals stays exact even after a
 // block has given up waiting.
 __device__ __forceinline__ void grid_barrier_arrive(unsigned int *counter)
 {
@@ -519,9 +563,10 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
         return;
     }
     if (refuses_to_plan(a)) return;      // uniform over the grid (the flag only changes between plans): no block waits for another
+    const PlanCounters pc = load_counters(a);
     const int t = tile * MW_TILE + tid;
     const bool active = t < a.T;
-    mw_acc *acc = a.d.acc + (a.epoch & 1u);
+    mw_acc *acc = a.d.acc + (pc.epoch & 1u);
     for (int i = tid; i < a.R * 8; i += MW_TILE) bits[i] = 0;
 
     // ---- phase A: bitmap (Section 4.1: bit r set <=> rank r is a target) and the bitmap table ----
@@ -602,9 +647,9 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             volatile unsigned long long *rec = a.d.tile_state + (size_t)tile * a.NC + c;
             uint32_t excl = 0;
             if (tile == 0) {
-                *rec = pack_state(a.epoch, kFlagPrefix, mine);
+                *rec = pack_state(pc.epoch, kFlagPrefix, mine);
             } else {
-                *rec = pack_state(a.epoch, kFlagAgg, mine);
+                *rec = pack_state(pc.epoch, kFlagAgg, mine);
                 bool done = false;
                 for (int j = tile - 1; j >= 0 && !done; j -= kLookBack) {
                     unsigned long long s[kLookBack];
@@ -617,7 +662,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                         int spins = 0;
                         while (true) {
                             const uint32_t hi = (uint32_t)(s[i] >> 32);
-                            if ((hi >> 2) == (a.wait_epoch & 0x3fffffffu) && (hi & 3u) != 0) break;
+                            if ((hi >> 2) == pc.wait_epoch && (hi & 3u) != 0) break;
                             if (++spins > a.spin_limit) { give_up(a, &acc->status); done = true; break; }
                             __nanosleep(64);
                             s[i] = *(volatile unsigned long long *)(a.d.tile_state + (size_t)(j - i) * a.NC + c);
@@ -627,7 +672,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
                         if (((uint32_t)(s[i] >> 32) & 3u) == kFlagPrefix) done = true;
                     }
                 }
-                *rec = pack_state(a.epoch, kFlagPrefix, excl + mine);
+                *rec = pack_state(pc.epoch, kFlagPrefix, excl + mine);
             }
             base[c] = (int)excl;
         }
@@ -654,7 +699,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
     __syncthreads();
     look_back(0, a.R);
     __syncthreads();
-    bool alive = grid_barrier_wait(a, a.bar_base + (unsigned)a.ntiles, true, &acc->status);
+    bool alive = grid_barrier_wait(a, pc.bar_base + (unsigned)a.ntiles, true, &acc->status);
 
     // ---- phase B2: leaders and group sizes are final; every tile publishes its two totals ----
     int leader = -1, gcount = 0, lead_excl = 0, gc_excl = 0;
@@ -730,7 +775,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             for (; i < a.Kd; ++i) { dr[i] = -1; dp[i] = -1; }
         }
     }
-    alive = grid_barrier_wait(a, a.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
+    alive = grid_barrier_wait(a, pc.bar_base + 2u * (unsigned)a.ntiles, alive, &acc->status);
     if (!alive) {
         if (tid == 0) set_status(&a.d.totals->status, MW_ERR_TIMEOUT);
         return;
@@ -759,9 +804,11 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_fused(PlanArgs a)
             tt.status = plan_status;
             tt.reserved = 0;
             *a.d.totals = tt;
-            mw_acc *next = a.d.acc + ((a.epoch + 1u) & 1u);
+            mw_acc *next = a.d.acc + ((pc.epoch + 1u) & 1u);
             next->valid_slots = 0; next->self_only = 0; next->status = 0;
+            advance_counters(a, 0u, 2u * (uint32_t)a.ntiles);   // every block is past the second barrier: all have read them
         }
+        if (tile == a.ntiles - 1) wipe_records_at_lap_end(a, pc.epoch);      // all look-backs ended before the first barrier
         if (plan_status == MW_ERR_TIMEOUT) return;      // a look-back gave up somewhere: nothing below can be trusted
     }
     // cnt[] now holds the region starts (the tile's own counts are no longer needed); the barriers of the scans
@@ -851,21 +898,12 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     a.ntiles = T > 0 ? (T + MW_TILE - 1) / MW_TILE : 1;
     a.NC = ctx->NC; a.hs_mask = ctx->HS - 1; a.Tm = ctx->cfg.max_tokens;
     a.row_bytes = ctx->cfg.row_bytes;
-    ctx->epoch += 1;
-    a.epoch = ctx->epoch & 0x3fffffffu;
-    if (a.epoch == 0) {
-        // the 30-bit epoch of the look-back records starts a new lap: wipe the records of the lap before
-        if (cudaMemsetAsync(ctx->d.tile_state, 0, sizeof(unsigned long long) * (size_t)ctx->max_tiles * (size_t)ctx->NC, st) != cudaSuccess)
-            return MW_ERR_CUDA;
-    }
-    a.ticket_base = ctx->tickets_used;
+    ctx->epoch += 1;                     // identifies the plan on the host (which plan a slot holds); the kernels count for themselves
     a.d = ctx->d;
-    a.bar_base = ctx->gbar_arrivals;
-    a.wait_epoch = a.epoch;
     a.spin_limit = ctx->spin_limit;
     a.bar_spin_limit = ctx->bar_spin_limit;
-    if (ctx->test_skew & MW_TEST_SKEW_LOOKBACK) a.wait_epoch = (a.epoch + 1u) & 0x3fffffffu;   // records nobody writes
-    if (ctx->test_skew & MW_TEST_SKEW_BARRIER) a.bar_base += 1u;                               // a count nobody reaches
+    a.skew_epoch = (ctx->test_skew & MW_TEST_SKEW_LOOKBACK) ? 1u : 0u;       // records nobody writes
+    a.skew_bar = (ctx->test_skew & MW_TEST_SKEW_BARRIER) ? 1u : 0u;          // a count nobody reaches
     ctx->test_skew &= ~(uint32_t)(MW_TEST_SKEW_LOOKBACK | MW_TEST_SKEW_BARRIER);
     const int blocks = a.ntiles;
     ctx->planned_T = T;
@@ -893,7 +931,6 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
         if (extra > 0 && a.pf_bytes == (int64_t)T * ctx->cfg.row_bytes) ctx->prefetched = rows;     // all of them fit
         const cudaError_t e = mw_launch(fn, dim3(blocks + extra), dim3(MW_TILE), tile_smem_bytes(ctx), st, false, a);
         if (e == cudaSuccess) {
-            ctx->gbar_arrivals += 2u * (uint32_t)blocks;
             ctx->launches += 1;
             return MW_OK;
         }
@@ -902,7 +939,6 @@ int mw_plan_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_t
     }
     k_plan_mask<<<blocks, MW_TILE, 0, st>>>(a);
     k_plan_tile<<<blocks, MW_TILE, tile_smem_bytes(ctx), st>>>(a);
-    ctx->tickets_used += (uint32_t)blocks;
     // one extra thread beyond T so that group_offsets[T] is covered
     k_plan_final<<<(T + 1 + MW_TILE - 1) / MW_TILE, MW_TILE, 0, st>>>(a);
     ctx->launches += 3;

@@ -424,7 +424,7 @@ int mw_small_launch(mw_ctx *ctx, const int32_t *topk_ids, const int32_t *expert_
                     !(ctx->cfg.flags & MW_FLAG_NO_OVERLAP), a);
     ctx->launches += 1;
     ctx->planned_T = T;
-    ctx->epoch += 2;          // a new plan (keeps the parity the tiled plan's double-buffered accumulators rely on)
+    ctx->epoch += 1;          // a new plan (the tiled plan's own counts live on the device and are not touched here)
     ctx->plan_epoch = ctx->epoch;
     ctx->prefetched = nullptr;
     if (e != cudaSuccess) { cudaGetLastError(); return MW_ERR_CUDA; }

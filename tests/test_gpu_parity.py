@@ -307,6 +307,56 @@ def test_one_call_replays_from_a_cuda_graph():
             assert send.guards_intact() and recv.guards_intact()
 
 
+@pytest.mark.parametrize("flags,prefetch", [(0, True), (0, False), (mw.MW_FLAG_PLAN_MULTIPASS, False)])
+def test_three_call_step_replays_from_a_cuda_graph(flags, prefetch):
+    """The tiled plan keeps its running counts (epoch of the look-back records, barrier arrivals, tile tickets) on the
+    device, so a captured plan + pack + deliver can be replayed: one graph, three different batches in the same buffers,
+    ordinary calls in between."""
+    torch = torch_mod()
+    batches = [wl.make_dispatch("dsv3_prefill", seed, T=1500, H=72) for seed in (100, 101, 102)]
+    s = batches[0].shape
+    T, B = 1500, s.row_bytes
+    ids_d = torch.from_numpy(batches[0].topk_ids).cuda()
+    e2r_d = torch.from_numpy(batches[0].expert_to_rank).cuda()
+    x_d = torch.from_numpy(batches[0].x.view(np.int16)).cuda()
+    plans = [mwo.plan(i.topk_ids, i.expert_to_rank, s.R, B) for i in batches]
+    Tn = max(p.totals["T_nonempty"] for p in plans)
+    SD = max(p.totals["total_dest"] for p in plans)
+    send, recv = Guarded(Tn * B), Guarded(SD * B)
+
+    def step(ctx):
+        if prefetch:
+            ctx.mw_plan_prefetch(ids_d, e2r_d, T, x_d)
+        else:
+            ctx.mw_plan(ids_d, e2r_d, T)
+        ctx.mw_pack(x_d, mw.MW_LAYOUT_MULTIWRITE, send.ptr(), Tn)
+        ctx.mw_deliver(mw.MW_LAYOUT_MULTIWRITE, send.ptr(), recv.ptr(), 0, SD)
+
+    with mw.Context(s.R, s.E, s.K, 2000, B, flags=flags) as ctx:
+        step(ctx)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(ctx)
+        for k, (inp, p) in enumerate(zip(batches + batches[:1], plans + plans[:1])):
+            ids_d.copy_(torch.from_numpy(inp.topk_ids))
+            x_d.copy_(torch.from_numpy(inp.x.view(np.int16)))
+            send.body.fill_(SENTINEL)
+            recv.body.fill_(SENTINEL)
+            if k == 2:
+                step(ctx)                     # an ordinary call between two replays
+            graph.replay()
+            graph.replay()                    # twice in a row: the counts advance on the device
+            torch.cuda.synchronize()
+            assert_plan_equal(ctx.plan_arrays(T), p, ctx.mw_get_totals())
+            want_send = mwo.pack_mw(p, inp.x)
+            n_send, n_recv = p.totals["T_nonempty"] * B, p.totals["total_dest"] * B
+            assert np.array_equal(send.host()[:n_send].reshape(-1, B), want_send)
+            assert np.array_equal(recv.host()[:n_recv], mwo.deliver_mw(p, want_send, 0, SENTINEL))
+            assert (send.host()[n_send:] == SENTINEL).all() and (recv.host()[n_recv:] == SENTINEL).all()
+            assert send.guards_intact() and recv.guards_intact()
+
+
 def test_one_call_capacity_overflow_is_reported_and_contained():
     torch = torch_mod()
     inp = wl.make_random_dispatch(21, T=200, K=3, E=32, R=8, H=16, contiguous_map=True)
