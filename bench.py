@@ -626,7 +626,7 @@ def mid_batch_measure(mw, wl, torch) -> list:
     headline workload: mw_plan_dispatch (one launch up to 1024 tokens) replayed from a CUDA graph, against the three
     calls of the headline step launched one by one."""
     out = []
-    for T in (128, 512, 1024, 2048):
+    for T in (128, 512, 1024, 2048, 4096):
         inp = wl.make_dispatch(WORKLOAD, T=T)
         s = inp.shape
         B = s.row_bytes
@@ -662,6 +662,20 @@ def mid_batch_measure(mw, wl, torch) -> list:
             b.record()
             torch.cuda.synchronize()
             row["three_calls_us"] = round(a.elapsed_time(b) * 1e3 / 200, 1)
+            # the same three calls replayed from a CUDA graph (the tiled plan keeps its running counts on the device)
+            graph3 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph3):
+                for i in range(2 * nset):
+                    three(i)
+            for _ in range(3):
+                graph3.replay()
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(20):
+                graph3.replay()
+            b.record()
+            torch.cuda.synchronize()
+            row["three_calls_graph_us"] = round(a.elapsed_time(b) * 1e3 / (40 * nset), 1)
             if T <= 1024:           # the single launch keeps no host-side state and can be replayed
                 one(0)
                 torch.cuda.synchronize()
