@@ -486,7 +486,7 @@ __global__ void __launch_bounds__(MW_TILE) k_plan_final(PlanArgs a)
 }
 
 // ------------------------------------------------------------------------------------------
-// Fused plan: the three phases in one cooperative launch.
+// Fused plan: the three phases in one launch.
 // ------------------------------------------------------------------------------------------
 constexpr int kLookBack = 8;                  // predecessors a look-back reads per round trip (16 measured slower: more records not ready yet)
 
