@@ -98,6 +98,14 @@ def test_random_weights_and_rows_bit_exact(mode, K, pad):
         assert np.array_equal(got, mwo.combine(p, z, weights, stride, precision="f32"))
 
 
+def test_maximum_top_k_bit_exact():
+    inp = workloads.make_random_dispatch(64, T=400, R=128, E=256, K=64, H=264, pad_fraction=0.05)     # up to 64 addends per element
+    rng = np.random.default_rng(64)
+    w = (rng.standard_normal((inp.T, 64)) * 0.7).astype(np.float32)
+    p, got, z, stride = gpu_combine(inp, lambda p, rows, cap: random_bf16(rng, (rows, 264)), w, "strided")
+    assert np.array_equal(got, mwo.combine(p, z, w, stride, precision="f32"))
+
+
 def test_prefill_shape_full_size_bit_exact():
     """The shape the benchmark times (4096 tokens, 64 ranks, 14336-byte rows), random weights and rows."""
     inp = workloads.make_dispatch("dsv3_prefill", payload=False)

@@ -82,6 +82,10 @@ def test_rank_word_boundaries(R, E):
     run_order(wl.make_random_dispatch(R, T=700, K=4, E=E, R=R, H=16))
 
 
+def test_maximum_top_k():
+    run_order(wl.make_random_dispatch(64, T=600, K=64, E=256, R=128, H=16, pad_fraction=0.05))       # 64 destinations per token
+
+
 def test_more_tokens_than_one_resident_grid_holds():
     run_order(wl.make_random_dispatch(17, T=40000, K=4, E=64, R=16, H=16, pad_fraction=0.05))
 

@@ -57,6 +57,16 @@ def test_launch_and_plan_variants_match(flags):
     run_dispatch(wl.make_dispatch("decode", H=64), flags=flags)
 
 
+def test_maximum_top_k():
+    """K = 64 expert slots per token, the largest the library accepts: 64 destinations per token on 128 ranks, and heavy
+    per-rank dedup on 8 ranks; fused and multi-kernel plan, separate calls and the one-pass dispatch."""
+    assert mw.lib() is not None
+    wide = wl.make_random_dispatch(64, T=700, K=64, E=256, R=128, H=24, pad_fraction=0.05)
+    run_dispatch(wide, separate=True)
+    run_dispatch(wide, flags=mw.MW_FLAG_PLAN_MULTIPASS)
+    run_dispatch(wl.make_random_dispatch(65, T=900, K=64, E=64, R=8, H=24, distinct=False), one_call=True)
+
+
 # ---- edge cases ------------------------------------------------------------------------------------
 @pytest.mark.parametrize("R", [1, 2, 63, 64, 65, 128, 129, 256, 1000, 1024])
 def test_rank_word_boundaries(R):

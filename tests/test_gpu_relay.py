@@ -50,7 +50,8 @@ def run_relay(inp, P, src, strided=False, flags=0, max_tokens=None):
 
 @pytest.mark.parametrize("R,P,src,E,K,T", [(16, 8, 0, 64, 8, 1500), (8, 4, 5, 16, 3, 700), (12, 3, 7, 24, 4, 300),
                                            (6, 6, 2, 12, 3, 257), (5, 1, 3, 10, 2, 64), (128, 8, 77, 256, 8, 2000),
-                                           (64, 8, 13, 128, 12, 900), (64, 4, 62, 128, 20, 515)])   # 12 and 20 destinations per token
+                                           (64, 8, 13, 128, 12, 900), (64, 4, 62, 128, 20, 515),    # 12 and 20 destinations per token
+                                           (128, 16, 5, 256, 64, 300)])                             # the largest top-k
 def test_relay_parity_random(R, P, src, E, K, T):
     inp = wl.make_random_dispatch(R + T, T=T, K=K, E=E, R=R, H=40, pad_fraction=0.1, contiguous_map=(E % R == 0))
     run_relay(inp, P, src)
