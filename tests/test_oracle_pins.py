@@ -199,6 +199,17 @@ def check_invariants(p, ids, e2r):
     assert np.array_equal(np.diff(p.rank_offsets), counts) and p.rank_offsets[0] == 0 and p.rank_offsets[R] == SD
     assert np.array_equal(p.token_ndest, onehot.sum(1))
     assert SD == p.token_ndest.sum() and (p.token_ndest <= Kd).all()
+    # the bitmaps, bit by bit (rank r = bit r mod 64 of word r div 64), and nothing beyond rank R - 1
+    bits = ((p.token_mask[:, np.arange(R) // 64] >> (np.arange(R) % 64).astype(np.uint64)) & np.uint64(1)).astype(bool)
+    assert np.array_equal(bits, onehot)
+    assert sum(int(v).bit_count() for v in p.token_mask.reshape(-1)) == SD
+    # a token's destination list: its ranks ascending, then -1
+    want_ranks = np.where(onehot, np.arange(R)[None, :], R + 1)
+    want_ranks.sort(axis=1)
+    want_ranks = np.where(want_ranks[:, :Kd] > R, -1, want_ranks[:, :Kd])
+    assert np.array_equal(p.dest_rank, want_ranks)
+    assert np.array_equal(p.dest_pos < 0, p.dest_rank < 0)
+    assert np.array_equal(p.token_group < 0, p.token_ndest == 0) and np.array_equal(p.token_mw_row < 0, p.token_ndest == 0)
     # offsets monotone, summing to totals
     go = p.group_offsets[:G + 1]
     assert go[0] == 0 and (np.diff(go) >= 1).all() and go[G] == Tn
